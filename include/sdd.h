@@ -1,0 +1,173 @@
+/*
+ * sdd.h — C ABI of the Speculative Diffusion Decoding (SpecDiff) round for NVIDIA B200 (sm_100a).
+ *
+ * One SpecDiff round (Algorithm 1 of "Speculative Diffusion Decoding", arXiv 2408.05636):
+ *   draft   : a masked-diffusion drafter M_q fills gamma [MASK] slots appended to the context in
+ *             T denoising evaluations (non-causal forward, soft-max over the vocabulary, draw);
+ *   verify  : the autoregressive target M_p scores all gamma+1 positions in one causal forward;
+ *   accept  : drafted token j is kept while u_j <= min(1, p_j(x_j)/q_j(x_j)); the first rejected
+ *             position is redrawn from norm(max(0, p - q)); if none is rejected one more token
+ *             is drawn from p_{gamma+1}.
+ *
+ * Conventions
+ *   - Every function returns an int32 status: SDD_OK (0) or a negative SDD_E_* code.  Nothing
+ *     here aborts, throws, traps the device or allocates device memory: the caller owns the
+ *     weights, the prompt, the outputs and one workspace blob whose size the library reports.
+ *     (The library owns only small host-side bookkeeping, including a few pinned host words.)
+ *   - "device" pointers are CUDA device pointers valid on the current device; "host" pointers
+ *     are ordinary host memory.  Pointers are borrowed for the lifetime of the sdd_ctx.
+ *   - All work is enqueued on the caller's stream and is asynchronous; only sdd_sync_status
+ *     blocks.  One sdd_ctx must be driven from one host thread at a time.
+ *   - Both networks are GPT-2-shaped (learned token + position embeddings, pre-LayerNorm blocks
+ *     with fused QKV, tanh-GELU MLP of width 4d, final LayerNorm, LM head tied to the token
+ *     embedding).  The drafter has one extra embedding row, id == vocab, the [MASK] token, and
+ *     uses no attention mask; the target is causal.
+ *   - Randomness: Philox4x32-10 keyed by `seed`; counter = (v >> 2 | 0, slot j, round r,
+ *     purpose << 24 | step k << 16 | sequence b); uniform = ((word >> 9) + 0.5) * 2^-23;
+ *     categorical draws are Gumbel-max over the vocabulary (ties -> lowest id).
+ */
+#ifndef SDD_H_
+#define SDD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  SDD_OK = 0,
+  SDD_E_ARG = -1,        /* null pointer, non-positive size, unsupported option               */
+  SDD_E_SHAPE = -2,      /* model shapes unsupported or inconsistent (vocab, d_model % n_head) */
+  SDD_E_WORKSPACE = -3,  /* workspace too small or misaligned (needs 256-byte alignment)       */
+  SDD_E_CTX_FULL = -4,   /* prompt + max_new + gamma exceeds a model's n_ctx                   */
+  SDD_E_CUDA = -5,       /* a CUDA runtime / driver call failed (see sdd_last_cuda_error)      */
+  SDD_E_TIMEOUT = -6,    /* a bounded device-side wait ran out; the device stays usable        */
+  SDD_E_UNIMPL = -7,     /* option combination not implemented                                 */
+  SDD_E_STATE = -8       /* call order violated (e.g. verify before draft)                     */
+};
+
+enum { SDD_FP32 = 0, SDD_BF16 = 1 };
+
+/* One transformer.  `tensors` is a host array of `n_tensors` device pointers in this order:
+ *   wte [vocab (+1 for the drafter), d], wpe [n_ctx, d],
+ *   then for each layer: ln1_g[d] ln1_b[d] w_qkv[3d,d] b_qkv[3d] w_o[d,d] b_o[d]
+ *                        ln2_g[d] ln2_b[d] w_fc1[4d,d] b_fc1[4d] w_fc2[d,4d] b_fc2[d],
+ *   then lnf_g[d] lnf_b[d].                       (n_tensors = 2 + 12 * n_layer + 2)
+ * Linear weights are [out_features, in_features] row-major (y = x W^T + b).  With dtype ==
+ * SDD_BF16 the matrices (wte, wpe, w_*) are bf16 and the vectors (ln*, b_*) are fp32; with
+ * SDD_FP32 everything is fp32.  All pointers must be 16-byte aligned. */
+typedef struct {
+  int32_t vocab, n_layer, d_model, n_head, n_ctx;
+  int32_t causal; /* 1 = autoregressive target, 0 = masked-diffusion drafter */
+  int32_t dtype;  /* SDD_FP32 or SDD_BF16 */
+  const void* const* tensors;
+  int32_t n_tensors;
+} sdd_model;
+
+typedef struct {
+  int32_t gamma;   /* draft length, 1..256                                                     */
+  int32_t T;       /* denoising evaluations per round, 1..255                                   */
+  int32_t batch;   /* independent sequences, 1..65535                                           */
+  int32_t max_new; /* tokens to generate per sequence; the last round's emission is truncated   */
+  float temp_p;    /* target temperature; 0 = greedy                                            */
+  float temp_q;    /* drafter temperature; 0 = greedy (temp_p and temp_q must both be 0 or > 0) */
+  uint64_t seed;   /* Philox key                                                                */
+  void* stream;    /* cudaStream_t, borrowed                                                    */
+} sdd_params;
+
+typedef struct sdd_ctx sdd_ctx;
+
+/* Bytes of device workspace sdd_create needs for these models and parameters (host call). */
+int32_t sdd_workspace_bytes(const sdd_model* target, const sdd_model* drafter, const sdd_params* params,
+                            uint64_t* out_bytes);
+
+/* Set up one generation (Section "Preliminaries": prefix x_{1:i} in, next n tokens out).
+ *   prompt_ids : device int32 [batch, prompt_stride], row b holds prompt_len[b] ids in [0, vocab)
+ *   prompt_len : host int32 [batch], each >= 1
+ *   workspace  : device memory, 256-byte aligned, >= sdd_workspace_bytes(); zeroed by this call
+ * Also enqueues the target's prefill of x_{0:c-2} into its KV cache.  *out receives the context
+ * (free it with sdd_destroy).  Errors: SDD_E_ARG, SDD_E_SHAPE, SDD_E_WORKSPACE, SDD_E_CTX_FULL,
+ * SDD_E_CUDA. */
+int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_params* params,
+                   const int32_t* prompt_ids, int32_t prompt_stride, const int32_t* prompt_len,
+                   void* workspace, uint64_t workspace_bytes, sdd_ctx** out);
+
+/* Drafting (Algorithm 1, "Take T diffusion steps to generate the draft" and "x ~ q^0"):
+ *   sdd_draft_begin : all gamma slots <- [MASK]
+ *   sdd_draft_step  : one denoising evaluation k = T, T-1, ... : drafter forward over
+ *                     context ∘ slots, LM head on the slot rows, then each still-masked slot is
+ *                     revealed with probability 1/k by a Gumbel-max draw from softmax(l / temp_q);
+ *                     the revealing row's logits and log q(x) are stored for the acceptance test
+ *   sdd_draft       : begin + T steps
+ * SDD_E_STATE if more than T steps are requested in one round. */
+int32_t sdd_draft_begin(sdd_ctx* ctx);
+int32_t sdd_draft_step(sdd_ctx* ctx);
+int32_t sdd_draft(sdd_ctx* ctx);
+
+/* Verification and acceptance (Algorithm 1 from "Run M_p in parallel" to "Return"): one causal,
+ * KV-cached target forward over [last context token, draft_1..draft_gamma], the acceptance test,
+ * the extra token, and the commit of n+1 tokens to every sequence's context.  Requires a finished
+ * draft (SDD_E_STATE otherwise).  If non-null, out_ids (device int32 [batch, gamma+1]) receives
+ * the tokens emitted this round (-1 padded) and n_out (device int32 [batch]) their count per
+ * sequence (0 for a sequence that already has max_new tokens). */
+int32_t sdd_verify_accept(sdd_ctx* ctx, int32_t* out_ids, int32_t* n_out);
+
+/* One whole round = sdd_draft + sdd_verify_accept. */
+int32_t sdd_step(sdd_ctx* ctx, int32_t* out_ids, int32_t* n_out);
+
+/* Non-blocking progress read (host): rounds whose commit has been seen so far, and the smallest
+ * number of generated tokens over the batch at that point.  Either pointer may be null. */
+int32_t sdd_progress(sdd_ctx* ctx, uint64_t* rounds_done, int32_t* min_emitted);
+
+/* Stand-alone acceptance on given logits (the acceptance rule of Section "Preliminaries" and
+ * Algorithm 1's last block, without the networks).  All pointers are device pointers.
+ *   logits_p  fp32 [rows, gamma+1, V]   target logits, row j scores the token after draft[0:j]
+ *   logits_q  fp32 [rows, gamma, V]     drafter logits each draft token was drawn from
+ *   draft_ids int32 [rows, gamma]
+ *   n_accept  int32 [rows]              out: number of accepted draft tokens
+ *   out_ids   int32 [rows, gamma+1]     out: accepted tokens, then the extra token; rest = -1
+ *   accept_prob fp32 [rows, gamma]      out: min(1, p/q) of every row (also past the rejection)
+ *   scratch   device, >= sdd_accept_scratch_bytes(rows, gamma, V) bytes, 16-byte aligned
+ * logits_p and logits_q must be 16-byte aligned.  Row b uses Philox sequence index b and round
+ * index `round`.  rows <= 65535, gamma <= 256, temp_p and temp_q both 0 (greedy) or both > 0. */
+uint64_t sdd_accept_scratch_bytes(int32_t rows, int32_t gamma, int32_t V);
+int32_t sdd_accept_logits(const float* logits_p, const float* logits_q, const int32_t* draft_ids,
+                          int32_t rows, int32_t gamma, int32_t V, float temp_p, float temp_q,
+                          uint64_t seed, uint64_t round, int32_t* n_accept, int32_t* out_ids,
+                          float* accept_prob, void* scratch, void* stream);
+
+/* Read-only device views into the workspace, for inspection and tests. */
+enum {
+  SDD_TAP_TOKENS = 0,      /* int32 [batch, tok_stride] context ids (prompt + emitted);
+                              tok_stride = min(target.n_ctx, drafter.n_ctx)                     */
+  SDD_TAP_CTX_LEN = 1,     /* int32 [batch]                                                     */
+  SDD_TAP_DRAFT_IDS = 2,   /* int32 [batch, gamma]      slot ids (vocab = still [MASK])         */
+  SDD_TAP_STEP_LOGITS = 3, /* fp32  [batch, gamma, V]   drafter logits of the latest evaluation */
+  SDD_TAP_Q_LOGITS = 4,    /* fp32  [batch, gamma, V]   stored rows l / temp_q (raw l if greedy)*/
+  SDD_TAP_LOGQ = 5,        /* fp32  [batch, gamma]      log q_j(x_j)                            */
+  SDD_TAP_REVEAL_STEP = 6, /* int32 [batch, gamma]      k at which slot j was revealed          */
+  SDD_TAP_LOGITS_P = 7,    /* fp32  [batch, gamma+1, V] target logits                           */
+  SDD_TAP_ACCEPT_PROB = 8, /* fp32  [batch, gamma]      min(1, p/q)                             */
+  SDD_TAP_N_ACCEPT = 9,    /* int32 [batch]                                                     */
+  SDD_TAP_EXTRA_TOKEN = 10,/* int32 [batch]                                                     */
+  SDD_TAP_N_EMITTED = 11,  /* int32 [batch]             tokens generated so far                 */
+  SDD_TAP_STATUS = 12      /* int32 [1]                 device status word (0 = ok)             */
+};
+int32_t sdd_tap(sdd_ctx* ctx, int32_t what, const void** dev_ptr, uint64_t* bytes);
+
+/* Host-side counters: rounds enqueued, kernels launched so far by this context. */
+int32_t sdd_counters(sdd_ctx* ctx, uint64_t* rounds, uint64_t* kernel_launches);
+
+/* Synchronise the stream and return the device status word as an SDD_E_* code. */
+int32_t sdd_sync_status(sdd_ctx* ctx);
+
+void sdd_destroy(sdd_ctx* ctx);
+const char* sdd_strerror(int32_t status);
+/* Text of the last CUDA error seen by this thread's calls into the library ("" if none). */
+const char* sdd_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDD_H_ */

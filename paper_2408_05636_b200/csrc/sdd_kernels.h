@@ -1,0 +1,80 @@
+// Internal launcher interface between the round scheduler (sdd_api.cu) and the kernels.
+#pragma once
+
+#include "sdd_common.cuh"
+
+namespace sdd {
+
+// ---- device-resident round state (head of the workspace) ------------------------------------
+struct RoundState {
+  int status;          // DEV_OK or the first device-side error
+  uint32_t round;      // rounds committed so far == Philox round index of the round in flight
+  uint32_t pad[2];
+};
+
+// How a target forward maps its rows to sequence positions.
+//   VERIFY : row j of sequence b is position ctx_len[b] - 1 + j, j = 0..gamma          (all rows valid)
+//   PREFILL: row j of sequence b is position j, valid while j < ctx_len[b] - 1
+enum TargetMode : int { TARGET_VERIFY = 0, TARGET_PREFILL = 1 };
+
+// GEMM epilogues:  C = A W^T (+ bias)
+enum Epilogue : int {
+  EPI_STORE = 0,      // out (activation type) = acc + bias
+  EPI_GELU = 1,       // out (activation type) = gelu_tanh(acc + bias)
+  EPI_RESIDUAL = 2,   // resid (fp32) += acc + bias
+  EPI_STORE_F32 = 3   // out (fp32) = acc            (LM head; ldc may differ from N)
+};
+
+// ---- vocabulary kernels (sdd_sample.cu) -----------------------------------------------------
+int stats_chunks_for(int V);
+cudaError_t launch_row_stats(const float* a, long long rows_a, const float* b, long long rows_b, int V, float inv_tau_a,
+                             float inv_tau_b, float2* partial, cudaStream_t st);
+cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float* q_logits, float* logq, int* reveal_step,
+                                 int batch, int gamma, int V, int k, float inv_tau_q, PhiloxKey key,
+                                 const RoundState* rs, cudaStream_t st);
+cudaError_t launch_accept(const float* logits_p, const float* q_rows, const int* draft_ids, const float* logq_in,
+                          const float2* partial_p, const float2* partial_q, int rows, int gamma, int V, float inv_tau_p,
+                          float inv_tau_q_rows, PhiloxKey key, uint32_t rnd, const RoundState* rs, float* accept_prob,
+                          int* n_accept, int* extra_token, int* out_ids, cudaStream_t st);
+cudaError_t launch_commit(int* tokens, int tok_stride, int* ctx_len, int* n_emitted, const int* slot_ids,
+                          const int* n_accept, const int* extra_token, int batch, int gamma, int max_new, RoundState* rs,
+                          int* out_ids, int* n_out, volatile int* host_mirror, cudaStream_t st);
+cudaError_t launch_reset_slots(int* slot_ids, int* reveal_step, int n, int mask_id, cudaStream_t st);
+
+// ---- glue (sdd_glue.cu) ---------------------------------------------------------------------
+template <typename T>
+cudaError_t launch_embed_drafter(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
+                                 const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st);
+template <typename T>
+cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
+                                const int* slot_ids, int batch, int gamma, int rows_per_seq, int mode, int d, float* h,
+                                cudaStream_t st);
+// LayerNorm of `rows` rows of h (fp32, row stride d) into out (activation type)
+template <typename T>
+cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* out, long long rows, int d, cudaStream_t st);
+// final LayerNorm of the gamma slot rows of every sequence: out[b*gamma + j] = LN(h[b*L_cap + ctx_len[b] + j])
+template <typename T>
+cudaError_t launch_layernorm_slots(const float* h, const float* g, const float* b, T* out, const int* ctx_len, int batch,
+                                   int gamma, int L_cap, int d, cudaStream_t st);
+// copy the K and V thirds of qkv rows into the cache: cache[b][pos][0|1][d]
+template <typename T>
+cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int batch, int rows_per_seq, int mode, int n_ctx,
+                             int d, cudaStream_t st);
+
+// ---- GEMM (sdd_gemm_simt.cu, sdd_gemm_tc.cu) ------------------------------------------------
+// C[M, N] = A[M, K] * W[N, K]^T; A row stride lda, W row stride K, out row stride ldc.
+template <typename T>
+cudaError_t launch_gemm_simt(const T* A, int lda, const T* W, const float* bias, int M, int N, int K, int epi, void* out,
+                             int ldc, cudaStream_t st);
+
+// ---- attention (sdd_attn.cu) ----------------------------------------------------------------
+// drafter: every row of a sequence attends to rows 0 .. ctx_len[b] + gamma - 1 of the same sequence
+template <typename T>
+cudaError_t launch_attn_bidir(const T* qkv, T* out, const int* ctx_len, int batch, int gamma, int L_cap, int n_head,
+                              int d_head, cudaStream_t st);
+// target: row j of sequence b (position p, see TargetMode) attends to cache positions 0 .. p
+template <typename T>
+cudaError_t launch_attn_cached(const T* qkv, const T* cache, T* out, const int* ctx_len, int batch, int rows_per_seq,
+                               int mode, int n_ctx, int n_head, int d_head, cudaStream_t st);
+
+}  // namespace sdd
