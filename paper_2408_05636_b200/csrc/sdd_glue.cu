@@ -1,0 +1,178 @@
+// Small row-wise kernels around the GEMMs: embedding gather, LayerNorm, KV-cache append.
+#include "sdd_kernels.h"
+
+namespace sdd {
+
+// ---------------------------------------------------------------------------------------------
+// embeddings: h = wte[token] + wpe[position]
+// drafter rows: sequence b owns rows b*L_cap .. b*L_cap + L_cap - 1; row i is context token i for
+// i < c, draft slot i - c for c <= i < c + gamma, and zero padding beyond.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_drafter_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
+                                     int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
+                                     int gamma, int L_cap, int d, float* __restrict__ h) {
+  const int i = blockIdx.x, b = blockIdx.y;
+  const int c = ctx_len[b];
+  float* __restrict__ dst = h + ((long long)b * L_cap + i) * d;
+  if (i >= c + gamma) {
+    for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = 0.f;
+    return;
+  }
+  const int tok = i < c ? tokens[(long long)b * tok_stride + i] : slot_ids[(long long)b * gamma + (i - c)];
+  const T* __restrict__ te = wte + (long long)tok * d;
+  const T* __restrict__ pe = wpe + (long long)i * d;
+  for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = to_f32(te[e]) + to_f32(pe[e]);
+}
+
+// target rows: sequence b owns rows b*rows_per_seq ..; VERIFY: row j = [last context token, drafts] at
+// position c-1+j; PREFILL: row j = context token j at position j (valid while j < c-1, else zero).
+template <typename T>
+__global__ void embed_target_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
+                                    int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
+                                    int gamma, int rows_per_seq, int mode, int d, float* __restrict__ h) {
+  const int j = blockIdx.x, b = blockIdx.y;
+  const int c = ctx_len[b];
+  float* __restrict__ dst = h + ((long long)b * rows_per_seq + j) * d;
+  int tok, pos;
+  if (mode == TARGET_VERIFY) {
+    pos = c - 1 + j;
+    tok = j == 0 ? tokens[(long long)b * tok_stride + c - 1] : slot_ids[(long long)b * gamma + j - 1];
+  } else {
+    pos = j;
+    tok = j < c - 1 ? tokens[(long long)b * tok_stride + j] : -1;
+  }
+  if (tok < 0) {
+    for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = 0.f;
+    return;
+  }
+  const T* __restrict__ te = wte + (long long)tok * d;
+  const T* __restrict__ pe = wpe + (long long)pos * d;
+  for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = to_f32(te[e]) + to_f32(pe[e]);
+}
+
+// ---------------------------------------------------------------------------------------------
+// LayerNorm (eps 1e-5): one warp per row, the row held in registers, mean then centred variance
+// ---------------------------------------------------------------------------------------------
+constexpr int LN_MAX_PER_LANE = 64;  // d_model <= 2048
+constexpr float LN_EPS = 1e-5f;
+
+template <typename T>
+__device__ __forceinline__ void layernorm_row(const float* __restrict__ src, const float* __restrict__ g,
+                                              const float* __restrict__ bta, T* __restrict__ dst, int d) {
+  const int lane = threadIdx.x & 31;
+  float x[LN_MAX_PER_LANE];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < LN_MAX_PER_LANE; ++i) {
+    const int e = i * 32 + lane;
+    x[i] = e < d ? src[e] : 0.f;
+    sum += x[i];
+  }
+  const float mu = warp_sum(sum) / (float)d;
+  float var = 0.f;
+#pragma unroll
+  for (int i = 0; i < LN_MAX_PER_LANE; ++i) {
+    const int e = i * 32 + lane;
+    const float c = e < d ? x[i] - mu : 0.f;
+    var += c * c;
+  }
+  const float rstd = rsqrtf(warp_sum(var) / (float)d + LN_EPS);
+#pragma unroll
+  for (int i = 0; i < LN_MAX_PER_LANE; ++i) {
+    const int e = i * 32 + lane;
+    if (e < d) dst[e] = from_f32<T>((x[i] - mu) * rstd * g[e] + bta[e]);
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128)
+layernorm_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
+                 T* __restrict__ out, long long rows, int d) {
+  const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  layernorm_row<T>(h + row * d, g, bta, out + row * d, d);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128)
+layernorm_slots_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
+                       T* __restrict__ out, const int* __restrict__ ctx_len, int batch, int gamma, int L_cap, int d) {
+  const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (r >= batch * gamma) return;
+  const int b = r / gamma, j = r - b * gamma;
+  layernorm_row<T>(h + ((long long)b * L_cap + ctx_len[b] + j) * d, g, bta, out + (long long)r * d, d);
+}
+
+// ---------------------------------------------------------------------------------------------
+// KV append: cache[b][pos][0] = K row, cache[b][pos][1] = V row
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void kv_append_kernel(const T* __restrict__ qkv, T* __restrict__ cache, const int* __restrict__ ctx_len,
+                                 int rows_per_seq, int mode, int n_ctx, int d) {
+  const int j = blockIdx.x, b = blockIdx.y;
+  const int c = ctx_len[b];
+  int pos;
+  if (mode == TARGET_VERIFY) pos = c - 1 + j;
+  else { if (j >= c - 1) return; pos = j; }
+  if (pos >= n_ctx) return;
+  const T* __restrict__ src = qkv + ((long long)b * rows_per_seq + j) * 3 * d + d;  // K then V, contiguous
+  T* __restrict__ dst = cache + ((long long)b * n_ctx + pos) * 2 * d;
+  for (int e = threadIdx.x; e < 2 * d; e += blockDim.x) dst[e] = src[e];
+}
+
+// ---------------------------------------------------------------------------------------------
+// launchers
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+cudaError_t launch_embed_drafter(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
+                                 const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st) {
+  embed_drafter_kernel<T><<<dim3(L_cap, batch), 128, 0, st>>>(wte, wpe, tokens, tok_stride, ctx_len, slot_ids, gamma,
+                                                              L_cap, d, h);
+  return cudaGetLastError();
+}
+template <typename T>
+cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
+                                const int* slot_ids, int batch, int gamma, int rows_per_seq, int mode, int d, float* h,
+                                cudaStream_t st) {
+  if (rows_per_seq <= 0) return cudaSuccess;
+  embed_target_kernel<T><<<dim3(rows_per_seq, batch), 128, 0, st>>>(wte, wpe, tokens, tok_stride, ctx_len, slot_ids, gamma,
+                                                                    rows_per_seq, mode, d, h);
+  return cudaGetLastError();
+}
+template <typename T>
+cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* out, long long rows, int d,
+                             cudaStream_t st) {
+  if (rows <= 0) return cudaSuccess;
+  if (d > LN_MAX_PER_LANE * 32) return cudaErrorInvalidValue;
+  layernorm_kernel<T><<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(h, g, b, out, rows, d);
+  return cudaGetLastError();
+}
+template <typename T>
+cudaError_t launch_layernorm_slots(const float* h, const float* g, const float* b, T* out, const int* ctx_len, int batch,
+                                   int gamma, int L_cap, int d, cudaStream_t st) {
+  if (d > LN_MAX_PER_LANE * 32) return cudaErrorInvalidValue;
+  layernorm_slots_kernel<T><<<(batch * gamma + 3) / 4, 128, 0, st>>>(h, g, b, out, ctx_len, batch, gamma, L_cap, d);
+  return cudaGetLastError();
+}
+template <typename T>
+cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int batch, int rows_per_seq, int mode, int n_ctx,
+                             int d, cudaStream_t st) {
+  if (rows_per_seq <= 0) return cudaSuccess;
+  kv_append_kernel<T><<<dim3(rows_per_seq, batch), 128, 0, st>>>(qkv, cache, ctx_len, rows_per_seq, mode, n_ctx, d);
+  return cudaGetLastError();
+}
+
+#define SDD_INSTANTIATE_GLUE(T)                                                                                          \
+  template cudaError_t launch_embed_drafter<T>(const T*, const T*, const int*, int, const int*, const int*, int, int,   \
+                                               int, int, float*, cudaStream_t);                                         \
+  template cudaError_t launch_embed_target<T>(const T*, const T*, const int*, int, const int*, const int*, int, int,    \
+                                              int, int, int, float*, cudaStream_t);                                     \
+  template cudaError_t launch_layernorm<T>(const float*, const float*, const float*, T*, long long, int, cudaStream_t); \
+  template cudaError_t launch_layernorm_slots<T>(const float*, const float*, const float*, T*, const int*, int, int,    \
+                                                 int, int, cudaStream_t);                                               \
+  template cudaError_t launch_kv_append<T>(const T*, T*, const int*, int, int, int, int, int, cudaStream_t);
+SDD_INSTANTIATE_GLUE(float)
+SDD_INSTANTIATE_GLUE(__nv_bfloat16)
+
+}  // namespace sdd
