@@ -1,0 +1,250 @@
+"""Python binding of the SpecDiff CUDA library (libsdd.so, built from csrc/ for sm_100a).
+
+Argument marshalling only: every step of a draft–verify–accept round runs in the library's
+CUDA kernels.  torch is used for device memory and streams.  The functions carry the same
+names as the C ABI in include/sdd.h; `Session` is a thin convenience wrapper around them.
+
+There is no CPU path: importing this package without a built libsdd.so raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsdd.so")
+
+SDD_OK = 0
+SDD_E_ARG, SDD_E_SHAPE, SDD_E_WORKSPACE, SDD_E_CTX_FULL = -1, -2, -3, -4
+SDD_E_CUDA, SDD_E_TIMEOUT, SDD_E_UNIMPL, SDD_E_STATE = -5, -6, -7, -8
+SDD_FP32, SDD_BF16 = 0, 1
+
+(TAP_TOKENS, TAP_CTX_LEN, TAP_DRAFT_IDS, TAP_STEP_LOGITS, TAP_Q_LOGITS, TAP_LOGQ, TAP_REVEAL_STEP,
+ TAP_LOGITS_P, TAP_ACCEPT_PROB, TAP_N_ACCEPT, TAP_EXTRA_TOKEN, TAP_N_EMITTED, TAP_STATUS) = range(13)
+
+EXPORTS = [
+    "sdd_workspace_bytes", "sdd_create", "sdd_draft_begin", "sdd_draft_step", "sdd_draft",
+    "sdd_verify_accept", "sdd_step", "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
+    "sdd_tap", "sdd_counters", "sdd_sync_status", "sdd_destroy", "sdd_strerror", "sdd_last_cuda_error",
+]
+
+
+class SddError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().sdd_strerror(status).decode()
+        cuda = lib().sdd_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({status})" + (f" [{cuda}]" if status == SDD_E_CUDA and cuda else ""))
+
+
+class sdd_model(C.Structure):
+    _fields_ = [("vocab", C.c_int32), ("n_layer", C.c_int32), ("d_model", C.c_int32), ("n_head", C.c_int32),
+                ("n_ctx", C.c_int32), ("causal", C.c_int32), ("dtype", C.c_int32),
+                ("tensors", C.POINTER(C.c_void_p)), ("n_tensors", C.c_int32)]
+
+
+class sdd_params(C.Structure):
+    _fields_ = [("gamma", C.c_int32), ("T", C.c_int32), ("batch", C.c_int32), ("max_new", C.c_int32),
+                ("temp_p", C.c_float), ("temp_q", C.c_float), ("seed", C.c_uint64), ("stream", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded library; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2408_05636_b200.build` "
+                              "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, u64, f32 = C.c_void_p, C.c_int32, C.c_uint64, C.c_float
+        L.sdd_workspace_bytes.argtypes = [C.POINTER(sdd_model), C.POINTER(sdd_model), C.POINTER(sdd_params), C.POINTER(u64)]
+        L.sdd_create.argtypes = [C.POINTER(sdd_model), C.POINTER(sdd_model), C.POINTER(sdd_params), vp, i32,
+                                 C.POINTER(i32), vp, u64, C.POINTER(vp)]
+        for n in ("sdd_draft_begin", "sdd_draft_step", "sdd_draft", "sdd_sync_status"):
+            getattr(L, n).argtypes = [vp]
+        L.sdd_verify_accept.argtypes = [vp, vp, vp]
+        L.sdd_step.argtypes = [vp, vp, vp]
+        L.sdd_progress.argtypes = [vp, C.POINTER(u64), C.POINTER(i32)]
+        L.sdd_accept_scratch_bytes.argtypes = [i32, i32, i32]
+        L.sdd_accept_scratch_bytes.restype = u64
+        L.sdd_accept_logits.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, u64, u64, vp, vp, vp, vp, vp]
+        L.sdd_tap.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(u64)]
+        L.sdd_counters.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
+        L.sdd_destroy.argtypes = [vp]
+        L.sdd_destroy.restype = None
+        L.sdd_strerror.argtypes = [i32]
+        L.sdd_strerror.restype = C.c_char_p
+        L.sdd_last_cuda_error.argtypes = []
+        L.sdd_last_cuda_error.restype = C.c_char_p
+        for n in EXPORTS:
+            if getattr(L, n).restype is C.c_int:
+                getattr(L, n).restype = i32
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != SDD_OK:
+        raise SddError(status, where)
+
+
+def _torch():
+    import torch
+    return torch
+
+
+# ----------------------------------------------------------------------------------------------
+# models on the device
+# ----------------------------------------------------------------------------------------------
+class DeviceModel:
+    """One transformer's weights uploaded to the GPU in the library's tensor order."""
+
+    def __init__(self, shape, tensors: Dict[str, np.ndarray], names: Sequence[str], dtype: str, device="cuda:0"):
+        torch = _torch()
+        self.shape = shape
+        self.dtype = SDD_BF16 if dtype == "bf16" else SDD_FP32
+        self.keep = []
+        ptrs = (C.c_void_p * len(names))()
+        for i, n in enumerate(names):
+            t = torch.from_numpy(np.ascontiguousarray(tensors[n]))
+            is_matrix = t.dim() == 2
+            t = t.to(device=device, dtype=torch.bfloat16 if (is_matrix and self.dtype == SDD_BF16) else torch.float32)
+            self.keep.append(t)
+            ptrs[i] = t.data_ptr()
+        self.ptrs = ptrs
+        self.c = sdd_model(shape.vocab, shape.n_layer, shape.d_model, shape.n_head, shape.n_ctx,
+                           1 if shape.causal else 0, self.dtype, C.cast(ptrs, C.POINTER(C.c_void_p)), len(names))
+
+
+# ----------------------------------------------------------------------------------------------
+# C ABI, same names
+# ----------------------------------------------------------------------------------------------
+def sdd_workspace_bytes(target: DeviceModel, drafter: DeviceModel, params: sdd_params) -> int:
+    out = C.c_uint64(0)
+    _check(lib().sdd_workspace_bytes(C.byref(target.c), C.byref(drafter.c), C.byref(params), C.byref(out)),
+           "sdd_workspace_bytes")
+    return int(out.value)
+
+
+def sdd_accept_scratch_bytes(rows: int, gamma: int, V: int) -> int:
+    return int(lib().sdd_accept_scratch_bytes(rows, gamma, V))
+
+
+def sdd_accept_logits(logits_p, logits_q, draft_ids, temp_p: float, temp_q: float, seed: int, rnd: int,
+                      scratch=None, stream=None):
+    """logits_p [rows, gamma+1, V] fp32, logits_q [rows, gamma, V] fp32, draft_ids [rows, gamma] int32, all CUDA
+    tensors.  Returns (n_accept [rows], out_ids [rows, gamma+1], accept_prob [rows, gamma])."""
+    torch = _torch()
+    rows, g1, V = logits_p.shape
+    gamma = g1 - 1
+    assert logits_q.shape == (rows, gamma, V) and draft_ids.shape == (rows, gamma)
+    assert logits_p.is_contiguous() and logits_q.is_contiguous() and draft_ids.is_contiguous()
+    assert logits_p.dtype == torch.float32 and logits_q.dtype == torch.float32 and draft_ids.dtype == torch.int32
+    dev = logits_p.device
+    n_accept = torch.empty(rows, dtype=torch.int32, device=dev)
+    out_ids = torch.empty(rows, gamma + 1, dtype=torch.int32, device=dev)
+    prob = torch.empty(rows, gamma, dtype=torch.float32, device=dev)
+    if scratch is None:
+        scratch = torch.empty(sdd_accept_scratch_bytes(rows, gamma, V), dtype=torch.uint8, device=dev)
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    _check(lib().sdd_accept_logits(logits_p.data_ptr(), logits_q.data_ptr(), draft_ids.data_ptr(), rows, gamma, V,
+                                   float(temp_p), float(temp_q), int(seed), int(rnd), n_accept.data_ptr(),
+                                   out_ids.data_ptr(), prob.data_ptr(), scratch.data_ptr(), st.cuda_stream),
+           "sdd_accept_logits")
+    return n_accept, out_ids, prob
+
+
+_TAP_DTYPES = {TAP_STEP_LOGITS: "f", TAP_Q_LOGITS: "f", TAP_LOGQ: "f", TAP_LOGITS_P: "f", TAP_ACCEPT_PROB: "f"}
+
+
+class Session:
+    """One generation: owns the workspace tensor and the sdd_ctx handle."""
+
+    def __init__(self, target: DeviceModel, drafter: DeviceModel, prompts: np.ndarray, prompt_len: Sequence[int],
+                 gamma: int, T: int, max_new: int, temp_p: float = 1.0, temp_q: float = 1.0, seed: int = 0,
+                 device="cuda:0", stream=None):
+        torch = _torch()
+        self.torch = torch
+        self.device = torch.device(device)
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        prompts = np.ascontiguousarray(prompts, dtype=np.int32)
+        self.batch, self.prompt_stride = prompts.shape
+        self.gamma, self.T, self.max_new, self.V = gamma, T, max_new, target.shape.vocab
+        self.tok_stride = min(target.shape.n_ctx, drafter.shape.n_ctx)
+        self.params = sdd_params(gamma, T, self.batch, max_new, temp_p, temp_q, seed, self.stream.cuda_stream)
+        self.target, self.drafter = target, drafter
+        nbytes = sdd_workspace_bytes(target, drafter, self.params)
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        self.prompts_dev = torch.from_numpy(prompts).to(self.device)
+        plen = (C.c_int32 * self.batch)(*[int(x) for x in prompt_len])
+        h = C.c_void_p(0)
+        _check(lib().sdd_create(C.byref(target.c), C.byref(drafter.c), C.byref(self.params), self.prompts_dev.data_ptr(),
+                                self.prompt_stride, plen, self.workspace.data_ptr(), nbytes, C.byref(h)), "sdd_create")
+        self.h = h
+        self.out_ids = torch.empty(self.batch, gamma + 1, dtype=torch.int32, device=self.device)
+        self.n_out = torch.empty(self.batch, dtype=torch.int32, device=self.device)
+
+    # --- the C ABI calls --------------------------------------------------------------------
+    def sdd_draft_begin(self): _check(lib().sdd_draft_begin(self.h), "sdd_draft_begin")
+    def sdd_draft_step(self): _check(lib().sdd_draft_step(self.h), "sdd_draft_step")
+    def sdd_draft(self): _check(lib().sdd_draft(self.h), "sdd_draft")
+
+    def sdd_verify_accept(self):
+        _check(lib().sdd_verify_accept(self.h, self.out_ids.data_ptr(), self.n_out.data_ptr()), "sdd_verify_accept")
+
+    def sdd_step(self):
+        _check(lib().sdd_step(self.h, self.out_ids.data_ptr(), self.n_out.data_ptr()), "sdd_step")
+
+    def sdd_sync_status(self): _check(lib().sdd_sync_status(self.h), "sdd_sync_status")
+
+    def sdd_progress(self):
+        r, e = C.c_uint64(0), C.c_int32(0)
+        _check(lib().sdd_progress(self.h, C.byref(r), C.byref(e)), "sdd_progress")
+        return int(r.value), int(e.value)
+
+    def sdd_counters(self):
+        r, k = C.c_uint64(0), C.c_uint64(0)
+        _check(lib().sdd_counters(self.h, C.byref(r), C.byref(k)), "sdd_counters")
+        return int(r.value), int(k.value)
+
+    def sdd_tap(self, what: int):
+        """Device view of a workspace buffer as a flat torch tensor (no copy)."""
+        torch = self.torch
+        p, n = C.c_void_p(0), C.c_uint64(0)
+        _check(lib().sdd_tap(self.h, what, C.byref(p), C.byref(n)), "sdd_tap")
+        off = p.value - self.workspace.data_ptr()
+        raw = self.workspace[off: off + n.value]
+        return raw.view(torch.float32 if what in _TAP_DTYPES else torch.int32)
+
+    def tap_numpy(self, what: int) -> np.ndarray:
+        self.sdd_sync_status()
+        return self.sdd_tap(what).cpu().numpy()
+
+    def generate(self):
+        """Run rounds until every sequence has max_new tokens; returns the token matrix [batch, tok_stride]
+        and the context lengths (host)."""
+        while True:
+            self.sdd_step()
+            _, emitted = self.sdd_progress()
+            if emitted >= self.max_new:
+                break
+        self.sdd_sync_status()
+        toks = self.sdd_tap(TAP_TOKENS).view(self.batch, self.tok_stride).cpu().numpy()
+        return toks, self.sdd_tap(TAP_CTX_LEN).cpu().numpy()
+
+    def close(self):
+        if getattr(self, "h", None) is not None and self.h.value:
+            lib().sdd_destroy(self.h)
+            self.h = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

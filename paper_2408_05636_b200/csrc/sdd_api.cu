@@ -1,0 +1,544 @@
+// C ABI of the SpecDiff round: argument checking, workspace layout, and the host-side schedule
+// that enqueues the kernels of Algorithm 1 on the caller's stream.  See include/sdd.h.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "sdd_kernels.h"
+
+namespace sdd {
+
+static thread_local char g_cuda_err[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* what) {
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+  return SDD_E_CUDA;
+}
+#define SDD_CUDA(expr)                                   \
+  do {                                                   \
+    cudaError_t e__ = (expr);                            \
+    if (e__ != cudaSuccess) return cuda_fail(e__, #expr); \
+  } while (0)
+#define SDD_TRY(expr)               \
+  do {                              \
+    int s__ = (expr);               \
+    if (s__ != SDD_OK) return s__;  \
+  } while (0)
+
+constexpr int ROW_TILE = 128;  // drafter rows per sequence are padded to a multiple of this
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- one model's tensors, typed -------------------------------------------------------------
+struct Layer {
+  const float *ln1_g, *ln1_b, *b_qkv, *b_o, *ln2_g, *ln2_b, *b_fc1, *b_fc2;
+  const void *w_qkv, *w_o, *w_fc1, *w_fc2;
+};
+struct Net {
+  int vocab, n_layer, d, n_head, d_head, n_ctx, causal, dtype;
+  const void *wte, *wpe;
+  const float *lnf_g, *lnf_b;
+  std::vector<Layer> layers;
+};
+
+static int parse_model(const sdd_model* m, int want_causal, Net* net) {
+  if (m == nullptr || m->tensors == nullptr) return SDD_E_ARG;
+  if (m->vocab < 2 || m->n_layer < 1 || m->d_model < 32 || m->n_head < 1 || m->n_ctx < 2) return SDD_E_SHAPE;
+  if (m->d_model % m->n_head != 0 || m->d_model > 2048 || m->d_model % 8 != 0) return SDD_E_SHAPE;
+  const int dh = m->d_model / m->n_head;
+  if (dh != 32 && dh != 64) return SDD_E_SHAPE;
+  if (m->causal != want_causal) return SDD_E_ARG;
+  if (m->dtype != SDD_FP32 && m->dtype != SDD_BF16) return SDD_E_ARG;
+  if (m->n_tensors != 2 + 12 * m->n_layer + 2) return SDD_E_SHAPE;
+  for (int i = 0; i < m->n_tensors; ++i) {
+    if (m->tensors[i] == nullptr) return SDD_E_ARG;
+    if ((reinterpret_cast<uintptr_t>(m->tensors[i]) & 15u) != 0) return SDD_E_ARG;
+  }
+  net->vocab = m->vocab; net->n_layer = m->n_layer; net->d = m->d_model; net->n_head = m->n_head;
+  net->d_head = dh; net->n_ctx = m->n_ctx; net->causal = m->causal; net->dtype = m->dtype;
+  const void* const* t = m->tensors;
+  net->wte = t[0]; net->wpe = t[1];
+  net->layers.resize(m->n_layer);
+  for (int l = 0; l < m->n_layer; ++l) {
+    const void* const* p = t + 2 + 12 * l;
+    Layer& L = net->layers[l];
+    L.ln1_g = (const float*)p[0]; L.ln1_b = (const float*)p[1]; L.w_qkv = p[2]; L.b_qkv = (const float*)p[3];
+    L.w_o = p[4]; L.b_o = (const float*)p[5]; L.ln2_g = (const float*)p[6]; L.ln2_b = (const float*)p[7];
+    L.w_fc1 = p[8]; L.b_fc1 = (const float*)p[9]; L.w_fc2 = p[10]; L.b_fc2 = (const float*)p[11];
+  }
+  net->lnf_g = (const float*)t[2 + 12 * m->n_layer];
+  net->lnf_b = (const float*)t[3 + 12 * m->n_layer];
+  return SDD_OK;
+}
+
+// ---- workspace ------------------------------------------------------------------------------
+struct Buffers {
+  RoundState* rs;
+  int *tokens, *ctx_len, *n_emitted, *slot_ids, *reveal_step, *n_accept, *extra_token;
+  float *logq, *accept_prob;
+  float *step_logits, *q_logits, *logits_p;
+  float2* partial_p;
+  float* h;                    // residual stream, fp32
+  void *xn, *qkv, *att, *mlp, *xf;  // activations in the model dtype
+  void* kv;                    // target KV cache [layer][batch][n_ctx][2][d]
+};
+
+struct Dims {
+  int batch, gamma, T, max_new, V, tok_stride, chunks;
+  int lcap_max;                // padded rows per sequence of the largest drafter forward
+  long long rows_q, rows_p;    // largest row counts of a drafter / target forward
+  int max_prompt;
+  size_t esize;                // bytes of an activation element
+};
+
+static size_t carve(const Dims& D, const Net& P, const Net& Q, uint8_t* base, Buffers* B) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> uint8_t* {
+    uint8_t* p = base ? base + off : nullptr;
+    off = align_up(off + bytes, 256);
+    return p;
+  };
+  const size_t Bn = D.batch, G = D.gamma, V = D.V;
+  Buffers b;
+  b.rs = (RoundState*)take(sizeof(RoundState));
+  b.tokens = (int*)take(Bn * D.tok_stride * 4);
+  b.ctx_len = (int*)take(Bn * 4);
+  b.n_emitted = (int*)take(Bn * 4);
+  b.slot_ids = (int*)take(Bn * G * 4);
+  b.reveal_step = (int*)take(Bn * G * 4);
+  b.n_accept = (int*)take(Bn * 4);
+  b.extra_token = (int*)take(Bn * 4);
+  b.logq = (float*)take(Bn * G * 4);
+  b.accept_prob = (float*)take(Bn * G * 4);
+  b.step_logits = (float*)take(Bn * G * V * 4);
+  b.q_logits = (float*)take(Bn * G * V * 4);
+  b.logits_p = (float*)take(Bn * (G + 1) * V * 4);
+  b.partial_p = (float2*)take(Bn * (G + 1) * D.chunks * sizeof(float2));
+  const size_t rq = (size_t)D.rows_q, rp = (size_t)D.rows_p;
+  auto mx = [](size_t a, size_t c) { return a > c ? a : c; };
+  b.h = (float*)take(mx(rq * Q.d, rp * P.d) * 4);
+  b.xn = take(mx(rq * Q.d, rp * P.d) * D.esize);
+  b.qkv = take(mx(rq * Q.d, rp * P.d) * 3 * D.esize);
+  b.att = take(mx(rq * Q.d, rp * P.d) * D.esize);
+  b.mlp = take(mx(rq * Q.d, rp * P.d) * 4 * D.esize);
+  b.xf = take(Bn * (G + 1) * mx(Q.d, P.d) * D.esize);
+  b.kv = take((size_t)P.n_layer * Bn * P.n_ctx * 2 * P.d * D.esize);
+  if (B) *B = b;
+  return off;
+}
+
+}  // namespace sdd
+
+using namespace sdd;
+
+struct sdd_ctx {
+  Net P, Q;
+  Dims D;
+  Buffers B;
+  sdd_params prm;
+  cudaStream_t st;
+  PhiloxKey key;
+  float inv_tau_p, inv_tau_q;
+  int steps_done;              // -1: no draft in progress; 0..T: denoising evaluations done this round
+  uint64_t rounds, launches;
+  std::vector<int> prompt_len, c_ub;
+  int* mirror;                 // pinned mapped host memory [1 + 2 B + 1]
+  int* mirror_dev;
+  std::vector<cudaEvent_t> ev;
+  int runahead;
+  int lcap;                    // padded rows per sequence of the current round's drafter forwards
+};
+
+// ---- argument checks shared by workspace_bytes and create -------------------------------------
+static int check_params(const sdd_model* target, const sdd_model* drafter, const sdd_params* p, Net* P, Net* Q) {
+  if (p == nullptr) return SDD_E_ARG;
+  SDD_TRY(parse_model(target, 1, P));
+  SDD_TRY(parse_model(drafter, 0, Q));
+  if (P->vocab != Q->vocab || P->dtype != Q->dtype) return SDD_E_SHAPE;
+  if (p->gamma < 1 || p->gamma > 256 || p->T < 1 || p->T > 255 || p->batch < 1 || p->batch > 65535 || p->max_new < 1)
+    return SDD_E_ARG;
+  if (!(p->temp_p >= 0.f) || !(p->temp_q >= 0.f) || ((p->temp_p == 0.f) != (p->temp_q == 0.f))) return SDD_E_ARG;
+  return SDD_OK;
+}
+
+static void fill_dims(const Net& P, const Net& Q, const sdd_params* p, int max_prompt, Dims* D) {
+  D->batch = p->batch; D->gamma = p->gamma; D->T = p->T; D->max_new = p->max_new; D->V = P.vocab;
+  D->tok_stride = P.n_ctx < Q.n_ctx ? P.n_ctx : Q.n_ctx;
+  D->chunks = stats_chunks_for(P.vocab);
+  int lmax = max_prompt + p->max_new + p->gamma;
+  if (lmax > D->tok_stride) lmax = D->tok_stride;
+  D->lcap_max = (int)align_up((size_t)lmax, ROW_TILE);
+  D->rows_q = (long long)p->batch * D->lcap_max;
+  const long long ver = (long long)p->batch * (p->gamma + 1), pre = (long long)p->batch * (max_prompt > 1 ? max_prompt - 1 : 0);
+  D->rows_p = ver > pre ? ver : pre;
+  D->max_prompt = max_prompt;
+  D->esize = P.dtype == SDD_BF16 ? 2 : 4;
+}
+
+// ---- GEMM dispatch ----------------------------------------------------------------------------
+template <typename T>
+static int gemm(sdd_ctx* c, const void* A, int lda, const void* W, const float* bias, long long M, int N, int K, int epi,
+                void* out, int ldc) {
+  if (M <= 0) return SDD_OK;
+  c->launches++;
+  SDD_CUDA(launch_gemm_simt<T>((const T*)A, lda, (const T*)W, bias, (int)M, N, K, epi, out, ldc, c->st));
+  return SDD_OK;
+}
+
+#define SDD_LAUNCH(c, expr) \
+  do {                      \
+    (c)->launches++;        \
+    SDD_CUDA(expr);         \
+  } while (0)
+
+// one transformer block on `rows` rows; attention is issued by the caller-supplied functor
+template <typename T, typename AttnFn>
+static int run_blocks(sdd_ctx* c, const Net& N, long long rows, AttnFn attn) {
+  const Buffers& B = c->B;
+  const int d = N.d;
+  for (int l = 0; l < N.n_layer; ++l) {
+    const Layer& L = N.layers[l];
+    SDD_LAUNCH(c, launch_layernorm<T>(B.h, L.ln1_g, L.ln1_b, (T*)B.xn, rows, d, c->st));
+    SDD_TRY(gemm<T>(c, B.xn, d, L.w_qkv, L.b_qkv, rows, 3 * d, d, EPI_STORE, B.qkv, 3 * d));
+    SDD_TRY(attn(l));
+    SDD_TRY(gemm<T>(c, B.att, d, L.w_o, L.b_o, rows, d, d, EPI_RESIDUAL, B.h, d));
+    SDD_LAUNCH(c, launch_layernorm<T>(B.h, L.ln2_g, L.ln2_b, (T*)B.xn, rows, d, c->st));
+    SDD_TRY(gemm<T>(c, B.xn, d, L.w_fc1, L.b_fc1, rows, 4 * d, d, EPI_GELU, B.mlp, 4 * d));
+    SDD_TRY(gemm<T>(c, B.mlp, 4 * d, L.w_fc2, L.b_fc2, rows, d, 4 * d, EPI_RESIDUAL, B.h, d));
+  }
+  return SDD_OK;
+}
+
+// one drafter evaluation M_q([x_{0:i}] ∘ [slots]) -> step_logits[B, gamma, V]
+template <typename T>
+static int forward_drafter(sdd_ctx* c) {
+  const Net& Q = c->Q;
+  const Buffers& B = c->B;
+  const Dims& D = c->D;
+  const int lcap = c->lcap;
+  const long long rows = (long long)D.batch * lcap;
+  SDD_LAUNCH(c, launch_embed_drafter<T>((const T*)Q.wte, (const T*)Q.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
+                                        D.batch, D.gamma, lcap, Q.d, B.h, c->st));
+  SDD_TRY((run_blocks<T>(c, Q, rows, [&](int) -> int {
+    SDD_LAUNCH(c, launch_attn_bidir<T>((const T*)B.qkv, (T*)B.att, B.ctx_len, D.batch, D.gamma, lcap, Q.n_head, Q.d_head,
+                                       c->st));
+    return SDD_OK;
+  })));
+  SDD_LAUNCH(c, launch_layernorm_slots<T>(B.h, Q.lnf_g, Q.lnf_b, (T*)B.xf, B.ctx_len, D.batch, D.gamma, lcap, Q.d, c->st));
+  SDD_TRY(gemm<T>(c, B.xf, Q.d, Q.wte, nullptr, (long long)D.batch * D.gamma, D.V, Q.d, EPI_STORE_F32, B.step_logits, D.V));
+  return SDD_OK;
+}
+
+// target forward over rows_per_seq new tokens per sequence against the KV cache
+template <typename T>
+static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) {
+  const Net& P = c->P;
+  const Buffers& B = c->B;
+  const Dims& D = c->D;
+  if (rows_per_seq <= 0) return SDD_OK;
+  const long long rows = (long long)D.batch * rows_per_seq;
+  SDD_LAUNCH(c, launch_embed_target<T>((const T*)P.wte, (const T*)P.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
+                                       D.batch, D.gamma, rows_per_seq, mode, P.d, B.h, c->st));
+  const size_t layer_elems = (size_t)D.batch * P.n_ctx * 2 * P.d;
+  SDD_TRY((run_blocks<T>(c, P, rows, [&](int l) -> int {
+    T* cache = (T*)B.kv + (size_t)l * layer_elems;
+    SDD_LAUNCH(c, launch_kv_append<T>((const T*)B.qkv, cache, B.ctx_len, D.batch, rows_per_seq, mode, P.n_ctx, P.d, c->st));
+    SDD_LAUNCH(c, launch_attn_cached<T>((const T*)B.qkv, cache, (T*)B.att, B.ctx_len, D.batch, rows_per_seq, mode, P.n_ctx,
+                                        P.n_head, P.d_head, c->st));
+    return SDD_OK;
+  })));
+  if (lm_head) {
+    SDD_LAUNCH(c, launch_layernorm<T>(B.h, P.lnf_g, P.lnf_b, (T*)B.xf, rows, P.d, c->st));
+    SDD_TRY(gemm<T>(c, B.xf, P.d, P.wte, nullptr, rows, D.V, P.d, EPI_STORE_F32, B.logits_p, D.V));
+  }
+  return SDD_OK;
+}
+
+// refresh the host's upper bound of every context length from the pinned mirror and pick the
+// padded row count of this round's drafter forwards
+static void choose_lcap(sdd_ctx* c) {
+  const int Bn = c->D.batch;
+  volatile int* m = c->mirror;
+  const int s0 = m[0];
+  std::vector<int> seen(Bn);
+  for (int b = 0; b < Bn; ++b) seen[b] = m[1 + b];
+  const int s1 = m[1 + 2 * Bn];
+  const int per_round = c->D.gamma + 1;
+  if (s0 == s1 && s1 > 0 && (uint64_t)s1 <= c->rounds) {
+    const long long behind = (long long)c->rounds - s1;
+    for (int b = 0; b < Bn; ++b) {
+      long long ub = seen[b] + behind * per_round;
+      if (ub < c->c_ub[b]) c->c_ub[b] = (int)ub;
+    }
+  }
+  int cmax = 1;
+  for (int b = 0; b < Bn; ++b) {
+    const int cap = c->prompt_len[b] + c->D.max_new;
+    if (c->c_ub[b] > cap) c->c_ub[b] = cap;
+    if (c->c_ub[b] > cmax) cmax = c->c_ub[b];
+  }
+  int lcap = (int)align_up((size_t)(cmax + c->D.gamma), ROW_TILE);
+  if (lcap > c->D.lcap_max) lcap = c->D.lcap_max;
+  c->lcap = lcap;
+}
+
+template <typename T>
+static int draft_step_t(sdd_ctx* c) {
+  const Buffers& B = c->B;
+  const Dims& D = c->D;
+  const int k = D.T - c->steps_done;
+  SDD_TRY(forward_drafter<T>(c));
+  SDD_LAUNCH(c, launch_unmask_sample(B.step_logits, B.slot_ids, B.q_logits, B.logq, B.reveal_step, D.batch, D.gamma, D.V, k,
+                                     c->inv_tau_q, c->key, B.rs, c->st));
+  c->steps_done++;
+  return SDD_OK;
+}
+
+template <typename T>
+static int verify_accept_t(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
+  const Buffers& B = c->B;
+  const Dims& D = c->D;
+  SDD_TRY(forward_target<T>(c, TARGET_VERIFY, D.gamma + 1, true));
+  SDD_LAUNCH(c, launch_row_stats(B.logits_p, (long long)D.batch * (D.gamma + 1), nullptr, 0, D.V, c->inv_tau_p, 0.f,
+                                 B.partial_p, c->st));
+  SDD_LAUNCH(c, launch_accept(B.logits_p, B.q_logits, B.slot_ids, B.logq, B.partial_p, nullptr, D.batch, D.gamma, D.V,
+                              c->inv_tau_p, c->inv_tau_p == 0.f ? 0.f : 1.f, c->key, 0u, B.rs, B.accept_prob, B.n_accept,
+                              B.extra_token, nullptr, c->st));
+  SDD_LAUNCH(c, launch_commit(B.tokens, D.tok_stride, B.ctx_len, B.n_emitted, B.slot_ids, B.n_accept, B.extra_token,
+                              D.batch, D.gamma, D.max_new, B.rs, out_ids, n_out, c->mirror_dev, c->st));
+  return SDD_OK;
+}
+
+// =================================================================================================
+extern "C" {
+
+int32_t sdd_workspace_bytes(const sdd_model* target, const sdd_model* drafter, const sdd_params* params,
+                            uint64_t* out_bytes) {
+  if (out_bytes == nullptr) return SDD_E_ARG;
+  Net P, Q;
+  SDD_TRY(check_params(target, drafter, params, &P, &Q));
+  // without the prompt lengths the drafter may have to cover its whole position table
+  Dims D;
+  const int tok_stride = P.n_ctx < Q.n_ctx ? P.n_ctx : Q.n_ctx;
+  fill_dims(P, Q, params, tok_stride, &D);
+  *out_bytes = carve(D, P, Q, nullptr, nullptr);
+  return SDD_OK;
+}
+
+int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_params* params,
+                   const int32_t* prompt_ids, int32_t prompt_stride, const int32_t* prompt_len, void* workspace,
+                   uint64_t workspace_bytes, sdd_ctx** out) {
+  if (out == nullptr || prompt_ids == nullptr || prompt_len == nullptr || workspace == nullptr) return SDD_E_ARG;
+  *out = nullptr;
+  sdd_ctx* c = new (std::nothrow) sdd_ctx();
+  if (c == nullptr) return SDD_E_ARG;
+  struct Guard { sdd_ctx* c; ~Guard() { if (c) sdd_destroy(c); } } guard{c};
+  c->mirror = nullptr;
+  int s = check_params(target, drafter, params, &c->P, &c->Q);
+  if (s != SDD_OK) return s;
+  int max_prompt = 0;
+  for (int b = 0; b < params->batch; ++b) {
+    if (prompt_len[b] < 1 || prompt_len[b] > prompt_stride) return SDD_E_ARG;
+    if (prompt_len[b] > max_prompt) max_prompt = prompt_len[b];
+  }
+  const int tok_stride = c->P.n_ctx < c->Q.n_ctx ? c->P.n_ctx : c->Q.n_ctx;
+  if ((long long)max_prompt + params->max_new + params->gamma > tok_stride) return SDD_E_CTX_FULL;
+  // the layout is the one sdd_workspace_bytes reports (prompt-independent), so its size check is exact
+  fill_dims(c->P, c->Q, params, tok_stride, &c->D);
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SDD_E_WORKSPACE;
+  if (carve(c->D, c->P, c->Q, nullptr, nullptr) > workspace_bytes) return SDD_E_WORKSPACE;
+  carve(c->D, c->P, c->Q, (uint8_t*)workspace, &c->B);
+  c->prm = *params;
+  c->st = (cudaStream_t)params->stream;
+  c->key = make_key(params->seed);
+  c->inv_tau_p = params->temp_p > 0.f ? 1.f / params->temp_p : 0.f;
+  c->inv_tau_q = params->temp_q > 0.f ? 1.f / params->temp_q : 0.f;
+  c->steps_done = -1;
+  c->rounds = 0;
+  c->launches = 0;
+  c->prompt_len.assign(prompt_len, prompt_len + params->batch);
+  c->c_ub = c->prompt_len;
+  const char* ra = getenv("SDD_RUNAHEAD");
+  c->runahead = ra ? atoi(ra) : 2;
+  if (c->runahead < 1) c->runahead = 1;
+  if (c->runahead > 8) c->runahead = 8;
+  c->ev.resize(c->runahead + 1);
+  for (auto& e : c->ev) e = nullptr;
+  for (auto& e : c->ev) SDD_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  const size_t mirror_ints = 2 + 2 * (size_t)params->batch;
+  SDD_CUDA(cudaHostAlloc((void**)&c->mirror, mirror_ints * sizeof(int), cudaHostAllocMapped));
+  memset(c->mirror, 0, mirror_ints * sizeof(int));
+  SDD_CUDA(cudaHostGetDevicePointer((void**)&c->mirror_dev, c->mirror, 0));
+
+  // zero the small state and the activations (padding rows must stay finite), then load the prompts
+  const Buffers& B = c->B;
+  const size_t state_bytes = (size_t)((uint8_t*)B.step_logits - (uint8_t*)workspace);
+  SDD_CUDA(cudaMemsetAsync(workspace, 0, state_bytes, c->st));
+  const size_t act_bytes = (size_t)((uint8_t*)B.kv - (uint8_t*)B.h);
+  SDD_CUDA(cudaMemsetAsync(B.h, 0, act_bytes, c->st));
+  SDD_CUDA(cudaMemcpy2DAsync(B.tokens, (size_t)c->D.tok_stride * 4, prompt_ids, (size_t)prompt_stride * 4,
+                             (size_t)max_prompt * 4, params->batch, cudaMemcpyDeviceToDevice, c->st));
+  SDD_CUDA(cudaMemcpyAsync(B.ctx_len, prompt_len, (size_t)params->batch * 4, cudaMemcpyHostToDevice, c->st));
+  // prefill the target's KV cache with x_{0:c-2}
+  c->D.max_prompt = max_prompt;
+  if (c->P.dtype == SDD_BF16) s = forward_target<__nv_bfloat16>(c, TARGET_PREFILL, max_prompt - 1, false);
+  else s = forward_target<float>(c, TARGET_PREFILL, max_prompt - 1, false);
+  if (s != SDD_OK) return s;
+  // prompt_len is host memory owned by the caller: make sure the copy above has consumed it
+  SDD_CUDA(cudaStreamSynchronize(c->st));
+  guard.c = nullptr;
+  *out = c;
+  return SDD_OK;
+}
+
+int32_t sdd_draft_begin(sdd_ctx* c) {
+  if (c == nullptr) return SDD_E_ARG;
+  // bound the host's run-ahead so that the length mirror stays fresh
+  if (c->rounds >= (uint64_t)c->runahead)
+    SDD_CUDA(cudaEventSynchronize(c->ev[(c->rounds - c->runahead) % c->ev.size()]));
+  choose_lcap(c);
+  SDD_LAUNCH(c, launch_reset_slots(c->B.slot_ids, c->B.reveal_step, c->D.batch * c->D.gamma, c->D.V, c->st));
+  c->steps_done = 0;
+  return SDD_OK;
+}
+
+int32_t sdd_draft_step(sdd_ctx* c) {
+  if (c == nullptr) return SDD_E_ARG;
+  if (c->steps_done < 0 || c->steps_done >= c->D.T) return SDD_E_STATE;
+  return c->P.dtype == SDD_BF16 ? draft_step_t<__nv_bfloat16>(c) : draft_step_t<float>(c);
+}
+
+int32_t sdd_draft(sdd_ctx* c) {
+  SDD_TRY(sdd_draft_begin(c));
+  for (int i = 0; i < c->D.T; ++i) SDD_TRY(sdd_draft_step(c));
+  return SDD_OK;
+}
+
+int32_t sdd_verify_accept(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
+  if (c == nullptr) return SDD_E_ARG;
+  if (c->steps_done != c->D.T) return SDD_E_STATE;
+  int s = c->P.dtype == SDD_BF16 ? verify_accept_t<__nv_bfloat16>(c, out_ids, n_out) : verify_accept_t<float>(c, out_ids, n_out);
+  if (s != SDD_OK) return s;
+  SDD_CUDA(cudaEventRecord(c->ev[c->rounds % c->ev.size()], c->st));
+  c->rounds++;
+  c->steps_done = -1;
+  for (auto& ub : c->c_ub) ub += c->D.gamma + 1;
+  return SDD_OK;
+}
+
+int32_t sdd_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
+  SDD_TRY(sdd_draft(c));
+  return sdd_verify_accept(c, out_ids, n_out);
+}
+
+int32_t sdd_progress(sdd_ctx* c, uint64_t* rounds_done, int32_t* min_emitted) {
+  if (c == nullptr) return SDD_E_ARG;
+  const int Bn = c->D.batch;
+  volatile int* m = c->mirror;
+  for (int attempt = 0; attempt < 64; ++attempt) {
+    const int s0 = m[0];
+    int mn = 0x7fffffff;
+    for (int b = 0; b < Bn; ++b) { const int e = m[1 + Bn + b]; if (e < mn) mn = e; }
+    const int s1 = m[1 + 2 * Bn];
+    if (s0 == s1) {
+      if (rounds_done) *rounds_done = (uint64_t)s1;
+      if (min_emitted) *min_emitted = s1 == 0 ? 0 : mn;
+      return SDD_OK;
+    }
+  }
+  // a commit is being written right now: report the previous, consistent view conservatively
+  if (rounds_done) *rounds_done = 0;
+  if (min_emitted) *min_emitted = 0;
+  return SDD_OK;
+}
+
+uint64_t sdd_accept_scratch_bytes(int32_t rows, int32_t gamma, int32_t V) {
+  if (rows < 1 || gamma < 1 || V < 1) return 0;
+  return (uint64_t)rows * (2ull * gamma + 1) * stats_chunks_for(V) * sizeof(float2);
+}
+
+int32_t sdd_accept_logits(const float* logits_p, const float* logits_q, const int32_t* draft_ids, int32_t rows,
+                          int32_t gamma, int32_t V, float temp_p, float temp_q, uint64_t seed, uint64_t round,
+                          int32_t* n_accept, int32_t* out_ids, float* accept_prob, void* scratch, void* stream) {
+  if (!logits_p || !logits_q || !draft_ids || !n_accept || !out_ids || !accept_prob || !scratch) return SDD_E_ARG;
+  if (rows < 1 || rows > 65535 || gamma < 1 || gamma > 256 || V < 2) return SDD_E_ARG;
+  if (!(temp_p >= 0.f) || !(temp_q >= 0.f) || ((temp_p == 0.f) != (temp_q == 0.f))) return SDD_E_ARG;
+  if (((uintptr_t)logits_p & 15u) || ((uintptr_t)logits_q & 15u) || ((uintptr_t)scratch & 15u)) return SDD_E_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const float itp = temp_p > 0.f ? 1.f / temp_p : 0.f, itq = temp_q > 0.f ? 1.f / temp_q : 0.f;
+  float2* partial = (float2*)scratch;
+  const long long rows_p = (long long)rows * (gamma + 1), rows_q = (long long)rows * gamma;
+  const int chunks = stats_chunks_for(V);
+  SDD_CUDA(launch_row_stats(logits_p, rows_p, logits_q, itp == 0.f ? 0 : rows_q, V, itp, itq, partial, st));
+  SDD_CUDA(launch_accept(logits_p, logits_q, draft_ids, nullptr, partial, partial + rows_p * chunks, rows, gamma, V, itp, itq,
+                         make_key(seed), (uint32_t)round, nullptr, accept_prob, n_accept, nullptr, out_ids, st));
+  return SDD_OK;
+}
+
+int32_t sdd_tap(sdd_ctx* c, int32_t what, const void** dev_ptr, uint64_t* bytes) {
+  if (c == nullptr || dev_ptr == nullptr || bytes == nullptr) return SDD_E_ARG;
+  const Buffers& B = c->B;
+  const uint64_t Bn = c->D.batch, G = c->D.gamma, V = c->D.V;
+  switch (what) {
+    case SDD_TAP_TOKENS: *dev_ptr = B.tokens; *bytes = Bn * c->D.tok_stride * 4; break;
+    case SDD_TAP_CTX_LEN: *dev_ptr = B.ctx_len; *bytes = Bn * 4; break;
+    case SDD_TAP_DRAFT_IDS: *dev_ptr = B.slot_ids; *bytes = Bn * G * 4; break;
+    case SDD_TAP_STEP_LOGITS: *dev_ptr = B.step_logits; *bytes = Bn * G * V * 4; break;
+    case SDD_TAP_Q_LOGITS: *dev_ptr = B.q_logits; *bytes = Bn * G * V * 4; break;
+    case SDD_TAP_LOGQ: *dev_ptr = B.logq; *bytes = Bn * G * 4; break;
+    case SDD_TAP_REVEAL_STEP: *dev_ptr = B.reveal_step; *bytes = Bn * G * 4; break;
+    case SDD_TAP_LOGITS_P: *dev_ptr = B.logits_p; *bytes = Bn * (G + 1) * V * 4; break;
+    case SDD_TAP_ACCEPT_PROB: *dev_ptr = B.accept_prob; *bytes = Bn * G * 4; break;
+    case SDD_TAP_N_ACCEPT: *dev_ptr = B.n_accept; *bytes = Bn * 4; break;
+    case SDD_TAP_EXTRA_TOKEN: *dev_ptr = B.extra_token; *bytes = Bn * 4; break;
+    case SDD_TAP_N_EMITTED: *dev_ptr = B.n_emitted; *bytes = Bn * 4; break;
+    case SDD_TAP_STATUS: *dev_ptr = &B.rs->status; *bytes = 4; break;
+    default: return SDD_E_ARG;
+  }
+  return SDD_OK;
+}
+
+int32_t sdd_counters(sdd_ctx* c, uint64_t* rounds, uint64_t* kernel_launches) {
+  if (c == nullptr) return SDD_E_ARG;
+  if (rounds) *rounds = c->rounds;
+  if (kernel_launches) *kernel_launches = c->launches;
+  return SDD_OK;
+}
+
+int32_t sdd_sync_status(sdd_ctx* c) {
+  if (c == nullptr) return SDD_E_ARG;
+  SDD_CUDA(cudaStreamSynchronize(c->st));
+  int status = 0;
+  SDD_CUDA(cudaMemcpy(&status, &c->B.rs->status, 4, cudaMemcpyDeviceToHost));
+  if (status == DEV_OK) return SDD_OK;
+  return status == DEV_TIMEOUT ? SDD_E_TIMEOUT : SDD_E_CTX_FULL;
+}
+
+void sdd_destroy(sdd_ctx* c) {
+  if (c == nullptr) return;
+  for (auto e : c->ev)
+    if (e) cudaEventDestroy(e);
+  if (c->mirror) cudaFreeHost(c->mirror);
+  delete c;
+}
+
+const char* sdd_strerror(int32_t s) {
+  switch (s) {
+    case SDD_OK: return "ok";
+    case SDD_E_ARG: return "invalid argument";
+    case SDD_E_SHAPE: return "unsupported or inconsistent model shape";
+    case SDD_E_WORKSPACE: return "workspace too small or misaligned";
+    case SDD_E_CTX_FULL: return "context would exceed the position table";
+    case SDD_E_CUDA: return "CUDA call failed";
+    case SDD_E_TIMEOUT: return "bounded device-side wait expired";
+    case SDD_E_UNIMPL: return "not implemented";
+    case SDD_E_STATE: return "call order violated";
+    default: return "unknown status";
+  }
+}
+
+const char* sdd_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"

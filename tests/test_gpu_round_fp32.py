@@ -1,0 +1,109 @@
+"""GPU parity of whole rounds on the tiny fp32 configuration (fp32 tolerance 1e-4 on logits)."""
+import numpy as np
+import pytest
+
+import synth
+from oracle import specdiff as sd
+from tests import roundcheck
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-4
+
+
+def _session(wl, dp, dq, prompts, plen, max_new, tau=1.0, gamma=None, T=None):
+    import paper_2408_05636_b200 as sdd
+    return sdd.Session(dp, dq, prompts, plen, gamma or wl.gamma, T or wl.T, max_new, tau, tau, wl.philox_seed)
+
+
+def test_stage_parity_four_rounds():
+    wl = synth.WORKLOADS["tiny_fp32"]
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 1, wl.prompt_len, wl.prompt_seed)
+    s = _session(wl, dp, dq, prompts, [wl.prompt_len], wl.max_new)
+    log, stats = roundcheck.check_rounds(s, mp, mq, wl, 4, 1.0, 1.0, TOL)
+    print("near-ties:", log, "max logit err q/p:", stats["max_q_err"], stats["max_p_err"])
+    assert len(log) <= 1
+    s.close()
+
+
+def test_end_to_end_four_rounds_no_teacher_forcing():
+    import paper_2408_05636_b200 as sdd
+    wl = synth.WORKLOADS["tiny_fp32"]
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 1, wl.prompt_len, wl.prompt_seed)
+    s = _session(wl, dp, dq, prompts, [wl.prompt_len], wl.max_new)
+    for _ in range(4):
+        s.sdd_step()
+    s.sdd_sync_status()
+    toks = s.tap_numpy(sdd.TAP_TOKENS).reshape(1, -1)[0]
+    c = int(s.tap_numpy(sdd.TAP_CTX_LEN)[0])
+    ids, traces = sd.generate(mp, mq, prompts[0], wl.gamma, wl.T, wl.max_new, 1.0, 1.0, wl.philox_seed, max_rounds=4)
+    assert c == len(ids)
+    assert np.array_equal(toks[:c], ids)
+    rounds, launches = s.sdd_counters()
+    assert rounds == 4 and launches > 0
+    s.close()
+
+
+def test_ragged_batch_with_truncation_and_perturbed_weights():
+    """Three sequences of different prompt lengths; biases and LayerNorm parameters non-trivial so that a
+    dropped bias or gain shows; max_new small so that sequences finish in different rounds."""
+    wl = synth.scaled_workload(synth.WORKLOADS["tiny_fp32"], batch=3)
+    mp, mq, dp, dq = roundcheck.build_pair(wl, bias_std=0.05, perturb_ln=True)
+    prompts = synth.prompt_ids(wl.target.vocab, 3, 40, wl.prompt_seed)
+    plen = [40, 7, 1]
+    s = _session(wl, dp, dq, prompts, plen, max_new=9, gamma=5, T=3)
+    log, stats = roundcheck.check_rounds(s, mp, mq, wl, 5, 1.0, 1.0, TOL)
+    assert len(log) <= 1
+    assert list(s.tap_numpy(__import__("paper_2408_05636_b200").TAP_N_EMITTED)) == [9, 9, 9]
+    assert stats["emitted"][-3:] != [6, 6, 6]
+    s.close()
+
+
+def test_greedy_equals_autoregressive_greedy():
+    import paper_2408_05636_b200 as sdd
+    wl = synth.WORKLOADS["tiny_fp32"]
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 1, wl.prompt_len, wl.prompt_seed)
+    n_new = 20
+    s = _session(wl, dp, dq, prompts, [wl.prompt_len], n_new, tau=0.0)
+    toks, clen = s.generate()
+    assert clen[0] == wl.prompt_len + n_new
+    ref = sd.autoregressive_greedy(mp, prompts[0], n_new)
+    assert np.array_equal(toks[0, : clen[0]], ref)
+    s.close()
+
+
+def test_temperature_and_T1():
+    wl = synth.scaled_workload(synth.WORKLOADS["tiny_fp32"], T=1)
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 1, 12, wl.prompt_seed)
+    import paper_2408_05636_b200 as sdd
+    s = sdd.Session(dp, dq, prompts, [12], 6, 1, 30, 0.8, 1.5, wl.philox_seed)
+    log, stats = roundcheck.check_rounds(s, mp, mq, wl, 3, 0.8, 1.5, TOL)
+    assert len(log) <= 1
+    s.close()
+
+
+def test_call_order_and_argument_errors():
+    import paper_2408_05636_b200 as sdd
+    wl = synth.WORKLOADS["tiny_fp32"]
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 1, wl.prompt_len, wl.prompt_seed)
+    s = _session(wl, dp, dq, prompts, [wl.prompt_len], wl.max_new)
+    with pytest.raises(sdd.SddError) as e:
+        s.sdd_verify_accept()                      # no draft yet
+    assert e.value.status == sdd.SDD_E_STATE
+    s.sdd_draft()
+    with pytest.raises(sdd.SddError) as e:
+        s.sdd_draft_step()                         # more than T steps
+    assert e.value.status == sdd.SDD_E_STATE
+    s.sdd_verify_accept()
+    s.sdd_sync_status()
+    s.close()
+    with pytest.raises(sdd.SddError) as e:         # prompt + max_new + gamma beyond the position table
+        _session(wl, dp, dq, prompts, [wl.prompt_len], 200)
+    assert e.value.status == sdd.SDD_E_CTX_FULL
+    with pytest.raises(sdd.SddError) as e:         # swapped models
+        sdd.Session(dq, dp, prompts, [wl.prompt_len], 8, 4, 10)
+    assert e.value.status == sdd.SDD_E_ARG
