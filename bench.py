@@ -1,0 +1,420 @@
+#!/usr/bin/env python
+"""Benchmark of the SpecDiff draft–verify–accept round on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one whole round (T drafter evaluations, one target verification, acceptance, commit)
+of a batch-1 generation on the GPT-2-small-shaped bf16 pair (12L d768 target and drafter, V = 50257,
+prompt 256 random ids, gamma = 16, T = 8, 256 new tokens).  When a generation reaches its 256 tokens
+a new one (next prompt seed) starts; set-up and prefill are outside the timed segments.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+WORKLOAD = "small_bf16"
+METRIC = "SpecDiff generated tokens/s at bs=1"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "tf_burst": d["bf16_tflops"], "tf_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tf_burst": 1590.0, "tf_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        for r in rows:
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(np.max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------------------------
+# algorithmic work per kernel category of one round (batch 1): (amount, unit-kind)
+# ----------------------------------------------------------------------------------------------
+def round_work(wl, c: int):
+    q, p = wl.drafter, wl.target
+    G, T, V = wl.gamma, wl.T, p.vocab
+    L = c + G
+    w = {}
+    w["gemm_drafter"] = (T * 2.0 * L * 12 * q.d_model ** 2 * q.n_layer, "flop")
+    w["head_drafter"] = (T * 2.0 * G * q.d_model * V, "flop")
+    w["attn_drafter"] = (T * 4.0 * L * L * q.d_model * q.n_layer, "flop")
+    w["gemm_target"] = (12.0 * p.d_model ** 2 * p.n_layer * 2, "byte")              # weights streamed once
+    w["head_target"] = (V * p.d_model * 2.0 + (G + 1) * V * 4.0, "byte")
+    w["attn_target"] = (2.0 * p.n_layer * c * p.d_model * 2, "byte")                # K and V of the cache
+    w["row_stats"] = ((G + 1) * V * 4.0, "byte")
+    w["accept"] = (5.0 * V * 4, "byte")
+    w["sample"] = (2.0 * G * V * 4, "byte")
+    w["layernorm"] = (T * (2 * q.n_layer) * L * q.d_model * 6.0 + 2 * p.n_layer * (G + 1) * p.d_model * 6.0, "byte")
+    w["glue"] = (T * L * q.d_model * 8.0, "byte")
+    w["commit"] = (0.0, "byte")
+    return w
+
+
+def make_models(wl, device):
+    import paper_2408_05636_b200 as sdd
+    wp = synth.model_weights(wl.target, wl.weight_seed, wl.dtype)
+    wq = synth.model_weights(wl.drafter, wl.weight_seed, wl.dtype)
+    dp = sdd.DeviceModel(wl.target, wp, synth.tensor_names(wl.target), wl.dtype, device)
+    dq = sdd.DeviceModel(wl.drafter, wq, synth.tensor_names(wl.drafter), wl.dtype, device)
+    return wp, wq, dp, dq
+
+
+# ----------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import paper_2408_05636_b200 as sdd
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    peaks = load_peaks()
+    wl = synth.WORKLOADS[WORKLOAD]
+    wp, wq, dp, dq = make_models(wl, device)
+    V = wl.target.vocab
+
+    gen_idx = [0]
+
+    def new_session():
+        seed = wl.prompt_seed + 1000 * rank + gen_idx[0]
+        gen_idx[0] += 1
+        prompts = synth.prompt_ids(V, 1, wl.prompt_len, seed)
+        s = sdd.Session(dp, dq, prompts, [wl.prompt_len], wl.gamma, wl.T, wl.max_new, 1.0, 1.0,
+                        wl.philox_seed + gen_idx[0], device)
+        s.sdd_sync_status()
+        return s
+
+    def emitted(s):
+        return int(s.tap_numpy(sdd.TAP_N_EMITTED)[0])
+
+    def run_rounds(n, timed):
+        """Runs n rounds (across generations if needed).  Returns (device ms, tokens, launches)."""
+        nonlocal sess
+        ms_total, tok_total, launch_total, left = 0.0, 0, 0, n
+        while left > 0:
+            e0 = emitted(sess)
+            if e0 >= wl.max_new:
+                sess.close()
+                sess = new_session()
+                e0 = 0
+            # rounds this generation can still take: stop a segment when it completes
+            _, l0 = sess.sdd_counters()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            ev0.record()
+            done = 0
+            while done < left:
+                sess.sdd_step()
+                done += 1
+                _, em = sess.sdd_progress()
+                if em >= wl.max_new:
+                    break
+            ev1.record()
+            torch.cuda.synchronize()
+            sess.sdd_sync_status()
+            _, l1 = sess.sdd_counters()
+            # rounds enqueued after the generation completed emit nothing but still ran: they are counted
+            ms_total += ev0.elapsed_time(ev1)
+            tok_total += emitted(sess) - e0
+            launch_total += l1 - l0
+            left -= done
+        return ms_total, tok_total, launch_total
+
+    sess = new_session()
+    run_rounds(args.warmup, False)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    clocks = ClockSampler(local) if rank == 0 else None
+    ms, toks, launches = run_rounds(args.steps, True)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+        t = torch.tensor([ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        k = torch.tensor([toks], device=device, dtype=torch.float64)
+        dist.all_reduce(k, op=dist.ReduceOp.SUM)
+        toks = int(k.item())
+    # keep the GPU busy a little longer so that the clock sampler sees load (same work, untimed)
+    t_end = time.time() + 1.0
+    while time.time() < t_end:
+        run_rounds(4, False)
+    clock_info = clocks.stop() if clocks else None
+    value = toks / (ms * 1e-3)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- profiled pass: per-category device time of the same rounds ---------------------------
+    sess.close()
+    gen_idx[0] = 0
+    sess = new_session()
+    prof_rounds = min(args.steps, 32)
+    cat_ms = {n: 0.0 for n in sdd.PROF_NAMES}
+    cat_n = {n: 0 for n in sdd.PROF_NAMES}
+    cat_work = {n: 0.0 for n in sdd.PROF_NAMES}
+    kinds = {}
+    for _ in range(prof_rounds):
+        if emitted(sess) >= wl.max_new:
+            sess.close()
+            sess = new_session()
+        c = int(sess.tap_numpy(sdd.TAP_CTX_LEN)[0])
+        sess.sdd_profile_begin()
+        sess.sdd_step()
+        res = sess.sdd_profile_end()
+        work = round_work(wl, c)
+        for n, (m, k) in res.items():
+            cat_ms[n] += m
+            cat_n[n] += k
+            cat_work[n] += work[n][0]
+            kinds[n] = work[n][1]
+    total_ms = sum(cat_ms.values())
+    kernels = {}
+    for n in sdd.PROF_NAMES:
+        if cat_n[n] == 0:
+            continue
+        secs = cat_ms[n] * 1e-3
+        if kinds[n] == "flop":
+            ach, peak, unit, bound = cat_work[n] / secs / 1e12, peaks["tf_sustained"], "TFLOP/s", "tensor"
+        else:
+            ach, peak, unit, bound = cat_work[n] / secs / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+        kernels[n] = {"share": round(cat_ms[n] / total_ms, 4), "launches": cat_n[n],
+                      "avg_us": round(cat_ms[n] * 1e3 / cat_n[n], 2), "bound": bound, "achieved": round(ach, 3),
+                      "peak": peak, "unit": unit, "frac": round(ach / peak, 5)}
+    dom = max(kernels, key=lambda n: kernels[n]["share"])
+    roofline = {"kernel": dom, "bound": kernels[dom]["bound"], "achieved": kernels[dom]["achieved"],
+                "peak": kernels[dom]["peak"], "unit": kernels[dom]["unit"], "frac": kernels[dom]["frac"],
+                "traffic": None, "peak_source": f"of {peaks['source']}",
+                "timing": f"CUDA-event pairs around every launch in a separate pass of {prof_rounds} rounds"}
+    sess.close()
+
+    # ---- stand-alone accept kernel: 64 rows x gamma 32 x V (fp32 logits with a shared component) --
+    rows, g4 = 64, 32
+    gen = torch.Generator(device=device)
+    gen.manual_seed(31)
+    cc = torch.randn(rows, g4 + 1, V, device=device, generator=gen)
+    lp = (cc + 0.5 * torch.randn(rows, g4 + 1, V, device=device, generator=gen)).contiguous()
+    lq = (cc[:, :g4] + 0.5 * torch.randn(rows, g4, V, device=device, generator=gen)).contiguous()
+    del cc
+    ids = torch.distributions.Categorical(logits=lq).sample().to(torch.int32).contiguous()
+    scratch = torch.empty(sdd.sdd_accept_scratch_bytes(rows, g4, V), dtype=torch.uint8, device=device)
+    for i in range(3):
+        sdd.sdd_accept_logits(lp, lq, ids, 1.0, 1.0, 31, i, scratch)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    iters = 20
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(iters):
+        n_acc, _, _ = sdd.sdd_accept_logits(lp, lq, ids, 1.0, 1.0, 31, 10 + i, scratch)
+    e1.record()
+    torch.cuda.synchronize()
+    acc_ms = e0.elapsed_time(e1) / iters
+    acc_bytes = rows * (2 * g4 + 1) * V * 4.0
+    accept_roof = {"bound": "hbm", "achieved": round(acc_bytes / (acc_ms * 1e-3) / 1e9, 1), "peak": peaks["hbm_gbs"],
+                   "unit": "GB/s", "frac": round(acc_bytes / (acc_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                   "traffic": None, "ms": round(acc_ms, 4), "launches_per_call": 2,
+                   "workload": f"{rows} rows x gamma {g4} x V {V} fp32 logits, inputs 0.84 GB > L2",
+                   "mean_accepted": float(n_acc.float().mean().item()), "peak_source": f"of {peaks['source']}"}
+    del lp, lq, ids, scratch
+
+    # ---- end to end through the C ABI with host buffers ----------------------------------------
+    prompts = synth.prompt_ids(V, 1, wl.prompt_len, wl.prompt_seed)
+    pinned_prompt = torch.from_numpy(prompts).pin_memory()
+    host_out = torch.empty(wl.gamma + 2, dtype=torch.int32).pin_memory()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    s = sdd.Session(dp, dq, pinned_prompt.numpy(), [wl.prompt_len], wl.gamma, wl.T, wl.max_new, 1.0, 1.0,
+                    wl.philox_seed, device)
+    rounds = 0
+    got = 0
+    while got < wl.max_new:
+        s.sdd_step()
+        host_out[: wl.gamma + 1].copy_(s.out_ids[0], non_blocking=True)
+        host_out[wl.gamma + 1:].copy_(s.n_out, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        got += int(host_out[wl.gamma + 1])
+        rounds += 1
+    t1 = time.perf_counter()
+    s.close()
+    e2e = {"value": round(got / (t1 - t0), 2), "unit": UNIT,
+           "h2d_bytes_per_step": round(wl.prompt_len * 4 / rounds, 1), "d2h_bytes_per_step": (wl.gamma + 2) * 4,
+           "includes": "sdd_create (prompt H2D, prefill), every round, per-round D2H of emitted ids", "rounds": rounds}
+
+    # ---- the oracle on the host cores, bounded sample -------------------------------------------
+    cpu = time_oracle(wl, wp, wq, budget_s=20.0, max_rounds=3)
+
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "bf16 12L d768 target + 12L d768 masked-diffusion drafter, V=50257, prompt 256, "
+                               "gamma=16, T=8, batch 1, 256 new tokens",
+                   "l2": "no flush: consecutive rounds of one generation; each round streams ~0.5 GB of weights (> 126 MB L2)",
+                   "multi_gpu": "independent replicas, no collective on the data path"},
+        "tokens_per_step": round(toks / args.steps / world, 3),
+        "clocks": clock_info, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline, "roofline_accept_kernel": accept_roof, "kernels": kernels, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------------------------
+def time_oracle(wl, wp, wq, budget_s, max_rounds):
+    from oracle import specdiff as sd
+    from oracle.transformer import Model
+    mp, mq = Model(wl.target, wp), Model(wl.drafter, wq)
+    prompt = synth.prompt_ids(wl.target.vocab, 1, wl.prompt_len, wl.prompt_seed)[0]
+    ids = [int(x) for x in prompt]
+    t0 = time.perf_counter()
+    rounds = 0
+    while rounds < max_rounds and (rounds == 0 or (time.perf_counter() - t0) * (rounds + 1) / rounds < budget_s):
+        tr = sd.specdiff_round(mp, mq, np.array(ids), wl.gamma, wl.T, 1.0, 1.0, wl.philox_seed, rounds)
+        ids += tr.emitted
+        rounds += 1
+    dt = time.perf_counter() - t0
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except Exception:
+        cores = os.cpu_count()
+    return {"value": round((len(ids) - len(prompt)) / dt, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {rounds} round(s) of the same generation (numpy fp64), {dt:.1f} s",
+            "s_per_round": round(dt / rounds, 3)}
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, on the host cores; each step is one oracle round of the same workload.
+    Rounds stop early when a time budget of about three minutes is used up."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import specdiff as sd
+    from oracle.transformer import Model
+    wl = synth.WORKLOADS[WORKLOAD]
+    wp = synth.model_weights(wl.target, wl.weight_seed, wl.dtype)
+    wq = synth.model_weights(wl.drafter, wl.weight_seed, wl.dtype)
+    mp, mq = Model(wl.target, wp), Model(wl.drafter, wq)
+    prompt = synth.prompt_ids(wl.target.vocab, 1, wl.prompt_len, wl.prompt_seed)[0]
+    ids = [int(x) for x in prompt]
+    budget = 180.0
+    t_start = time.perf_counter()
+    rnd = 0
+    for _ in range(args.warmup):
+        if time.perf_counter() - t_start > 0.25 * budget:
+            break
+        ids += sd.specdiff_round(mp, mq, np.array(ids), wl.gamma, wl.T, 1.0, 1.0, wl.philox_seed, rnd).emitted
+        rnd += 1
+    t0 = time.perf_counter()
+    done, toks = 0, 0
+    while done < args.steps:
+        em = sd.specdiff_round(mp, mq, np.array(ids), wl.gamma, wl.T, 1.0, 1.0, wl.philox_seed, rnd).emitted
+        ids += em
+        toks += len(em)
+        rnd += 1
+        done += 1
+        if time.perf_counter() - t_start > budget:
+            break
+    dt = time.perf_counter() - t0
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except Exception:
+        cores = os.cpu_count()
+    value = toks / dt
+    sample = f"{done} oracle round(s) of the same generation (numpy fp64) in {dt:.1f} s"
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": done, "steps_requested": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(dt * 1e3 / done, 2), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "bf16-rounded weights, 12L d768 target + 12L d768 masked-diffusion drafter, V=50257, "
+                                   "prompt 256, gamma=16, T=8, batch 1"},
+            "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 12 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args)
+    else:
+        args.steps = 64 if args.steps is None else args.steps
+        args.warmup = max(3, 8 if args.warmup is None else args.warmup)
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -159,6 +159,19 @@ int32_t sdd_tap(sdd_ctx* ctx, int32_t what, const void** dev_ptr, uint64_t* byte
 /* Host-side counters: rounds enqueued, kernels launched so far by this context. */
 int32_t sdd_counters(sdd_ctx* ctx, uint64_t* rounds, uint64_t* kernel_launches);
 
+/* Optional per-launch timing, for measurement only (it adds two CUDA events around every kernel
+ * launch, so it is not meant to be left on).  sdd_profile_begin starts collecting; sdd_profile_end
+ * synchronises the stream and returns, per kernel category, the summed device time in milliseconds
+ * and the number of launches (arrays of n_categories >= SDD_PROF_COUNT entries). */
+enum {
+  SDD_PROF_GEMM_DRAFTER = 0, SDD_PROF_GEMM_TARGET = 1, SDD_PROF_HEAD_DRAFTER = 2, SDD_PROF_HEAD_TARGET = 3,
+  SDD_PROF_ATTN_DRAFTER = 4, SDD_PROF_ATTN_TARGET = 5, SDD_PROF_LAYERNORM = 6, SDD_PROF_GLUE = 7,
+  SDD_PROF_SAMPLE = 8, SDD_PROF_ROW_STATS = 9, SDD_PROF_ACCEPT = 10, SDD_PROF_COMMIT = 11, SDD_PROF_COUNT = 12
+};
+int32_t sdd_profile_begin(sdd_ctx* ctx);
+int32_t sdd_profile_end(sdd_ctx* ctx, double* ms_per_category, uint64_t* launches_per_category,
+                        int32_t n_categories);
+
 /* Synchronise the stream and return the device status word as an SDD_E_* code. */
 int32_t sdd_sync_status(sdd_ctx* ctx);
 

@@ -25,10 +25,13 @@ SDD_FP32, SDD_BF16 = 0, 1
 (TAP_TOKENS, TAP_CTX_LEN, TAP_DRAFT_IDS, TAP_STEP_LOGITS, TAP_Q_LOGITS, TAP_LOGQ, TAP_REVEAL_STEP,
  TAP_LOGITS_P, TAP_ACCEPT_PROB, TAP_N_ACCEPT, TAP_EXTRA_TOKEN, TAP_N_EMITTED, TAP_STATUS) = range(13)
 
+PROF_NAMES = ["gemm_drafter", "gemm_target", "head_drafter", "head_target", "attn_drafter", "attn_target",
+              "layernorm", "glue", "sample", "row_stats", "accept", "commit"]
+
 EXPORTS = [
     "sdd_workspace_bytes", "sdd_create", "sdd_draft_begin", "sdd_draft_step", "sdd_draft",
     "sdd_verify_accept", "sdd_step", "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
-    "sdd_tap", "sdd_counters", "sdd_sync_status", "sdd_destroy", "sdd_strerror", "sdd_last_cuda_error",
+    "sdd_tap", "sdd_counters", "sdd_profile_begin", "sdd_profile_end", "sdd_sync_status", "sdd_destroy", "sdd_strerror", "sdd_last_cuda_error",
 ]
 
 
@@ -76,6 +79,8 @@ def lib() -> C.CDLL:
         L.sdd_accept_logits.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, u64, u64, vp, vp, vp, vp, vp]
         L.sdd_tap.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(u64)]
         L.sdd_counters.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
+        L.sdd_profile_begin.argtypes = [vp]
+        L.sdd_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u64), i32]
         L.sdd_destroy.argtypes = [vp]
         L.sdd_destroy.restype = None
         L.sdd_strerror.argtypes = [i32]
@@ -212,6 +217,15 @@ class Session:
         r, k = C.c_uint64(0), C.c_uint64(0)
         _check(lib().sdd_counters(self.h, C.byref(r), C.byref(k)), "sdd_counters")
         return int(r.value), int(k.value)
+
+    def sdd_profile_begin(self): _check(lib().sdd_profile_begin(self.h), "sdd_profile_begin")
+
+    def sdd_profile_end(self):
+        """{category name: (milliseconds, launches)} since sdd_profile_begin."""
+        ms = (C.c_double * len(PROF_NAMES))()
+        n = (C.c_uint64 * len(PROF_NAMES))()
+        _check(lib().sdd_profile_end(self.h, ms, n, len(PROF_NAMES)), "sdd_profile_end")
+        return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(PROF_NAMES)}
 
     def sdd_tap(self, what: int):
         """Device view of a workspace buffer as a flat torch tensor (no copy)."""

@@ -29,6 +29,10 @@ static int cuda_fail(cudaError_t e, const char* what) {
 
 constexpr int ROW_TILE = 128;  // drafter rows per sequence are padded to a multiple of this
 
+// kernel categories of the optional per-launch timing (sdd_profile_*)
+enum Cat : int { CAT_GEMM_Q = 0, CAT_GEMM_P, CAT_HEAD_Q, CAT_HEAD_P, CAT_ATTN_Q, CAT_ATTN_P, CAT_LAYERNORM, CAT_GLUE,
+                 CAT_SAMPLE, CAT_STATS, CAT_ACCEPT, CAT_COMMIT, CAT_COUNT };
+
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // ---- one model's tensors, typed -------------------------------------------------------------
@@ -149,6 +153,35 @@ struct sdd_ctx {
   std::vector<cudaEvent_t> ev;
   int runahead;
   int lcap;                    // padded rows per sequence of the current round's drafter forwards
+  // optional per-launch timing
+  bool profiling;
+  std::vector<cudaEvent_t> prof_ev;   // pairs (before, after)
+  std::vector<int> prof_cat;
+  size_t prof_used;
+};
+
+// RAII helper: brackets one launch with events when profiling is on
+struct ProfScope {
+  sdd_ctx* c;
+  bool on;
+  ProfScope(sdd_ctx* c_, int cat) : c(c_), on(false) {
+    if (!c->profiling) return;
+    if (c->prof_used + 2 > c->prof_ev.size()) {
+      for (int i = 0; i < 2; ++i) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) return;
+        c->prof_ev.push_back(e);
+      }
+    }
+    cudaEventRecord(c->prof_ev[c->prof_used], c->st);
+    c->prof_cat.push_back(cat);
+    on = true;
+  }
+  ~ProfScope() {
+    if (!on) return;
+    cudaEventRecord(c->prof_ev[c->prof_used + 1], c->st);
+    c->prof_used += 2;
+  }
 };
 
 // ---- argument checks shared by workspace_bytes and create -------------------------------------
@@ -179,34 +212,36 @@ static void fill_dims(const Net& P, const Net& Q, const sdd_params* p, int max_p
 
 // ---- GEMM dispatch ----------------------------------------------------------------------------
 template <typename T>
-static int gemm(sdd_ctx* c, const void* A, int lda, const void* W, const float* bias, long long M, int N, int K, int epi,
-                void* out, int ldc) {
+static int gemm(sdd_ctx* c, int cat, const void* A, int lda, const void* W, const float* bias, long long M, int N, int K,
+                int epi, void* out, int ldc) {
   if (M <= 0) return SDD_OK;
+  ProfScope prof(c, cat);
   c->launches++;
   SDD_CUDA(launch_gemm_simt<T>((const T*)A, lda, (const T*)W, bias, (int)M, N, K, epi, out, ldc, c->st));
   return SDD_OK;
 }
 
-#define SDD_LAUNCH(c, expr) \
-  do {                      \
-    (c)->launches++;        \
-    SDD_CUDA(expr);         \
+#define SDD_LAUNCH(c, cat, expr) \
+  do {                           \
+    ProfScope prof__((c), (cat)); \
+    (c)->launches++;             \
+    SDD_CUDA(expr);              \
   } while (0)
 
 // one transformer block on `rows` rows; attention is issued by the caller-supplied functor
 template <typename T, typename AttnFn>
-static int run_blocks(sdd_ctx* c, const Net& N, long long rows, AttnFn attn) {
+static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, AttnFn attn) {
   const Buffers& B = c->B;
   const int d = N.d;
   for (int l = 0; l < N.n_layer; ++l) {
     const Layer& L = N.layers[l];
-    SDD_LAUNCH(c, launch_layernorm<T>(B.h, L.ln1_g, L.ln1_b, (T*)B.xn, rows, d, c->st));
-    SDD_TRY(gemm<T>(c, B.xn, d, L.w_qkv, L.b_qkv, rows, 3 * d, d, EPI_STORE, B.qkv, 3 * d));
+    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln1_g, L.ln1_b, (T*)B.xn, rows, d, c->st));
+    SDD_TRY(gemm<T>(c, gcat, B.xn, d, L.w_qkv, L.b_qkv, rows, 3 * d, d, EPI_STORE, B.qkv, 3 * d));
     SDD_TRY(attn(l));
-    SDD_TRY(gemm<T>(c, B.att, d, L.w_o, L.b_o, rows, d, d, EPI_RESIDUAL, B.h, d));
-    SDD_LAUNCH(c, launch_layernorm<T>(B.h, L.ln2_g, L.ln2_b, (T*)B.xn, rows, d, c->st));
-    SDD_TRY(gemm<T>(c, B.xn, d, L.w_fc1, L.b_fc1, rows, 4 * d, d, EPI_GELU, B.mlp, 4 * d));
-    SDD_TRY(gemm<T>(c, B.mlp, 4 * d, L.w_fc2, L.b_fc2, rows, d, 4 * d, EPI_RESIDUAL, B.h, d));
+    SDD_TRY(gemm<T>(c, gcat, B.att, d, L.w_o, L.b_o, rows, d, d, EPI_RESIDUAL, B.h, d));
+    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln2_g, L.ln2_b, (T*)B.xn, rows, d, c->st));
+    SDD_TRY(gemm<T>(c, gcat, B.xn, d, L.w_fc1, L.b_fc1, rows, 4 * d, d, EPI_GELU, B.mlp, 4 * d));
+    SDD_TRY(gemm<T>(c, gcat, B.mlp, 4 * d, L.w_fc2, L.b_fc2, rows, d, 4 * d, EPI_RESIDUAL, B.h, d));
   }
   return SDD_OK;
 }
@@ -219,15 +254,15 @@ static int forward_drafter(sdd_ctx* c) {
   const Dims& D = c->D;
   const int lcap = c->lcap;
   const long long rows = (long long)D.batch * lcap;
-  SDD_LAUNCH(c, launch_embed_drafter<T>((const T*)Q.wte, (const T*)Q.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
+  SDD_LAUNCH(c, CAT_GLUE, launch_embed_drafter<T>((const T*)Q.wte, (const T*)Q.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
                                         D.batch, D.gamma, lcap, Q.d, B.h, c->st));
-  SDD_TRY((run_blocks<T>(c, Q, rows, [&](int) -> int {
-    SDD_LAUNCH(c, launch_attn_bidir<T>((const T*)B.qkv, (T*)B.att, B.ctx_len, D.batch, D.gamma, lcap, Q.n_head, Q.d_head,
+  SDD_TRY((run_blocks<T>(c, Q, rows, CAT_GEMM_Q, [&](int) -> int {
+    SDD_LAUNCH(c, CAT_ATTN_Q, launch_attn_bidir<T>((const T*)B.qkv, (T*)B.att, B.ctx_len, D.batch, D.gamma, lcap, Q.n_head, Q.d_head,
                                        c->st));
     return SDD_OK;
   })));
-  SDD_LAUNCH(c, launch_layernorm_slots<T>(B.h, Q.lnf_g, Q.lnf_b, (T*)B.xf, B.ctx_len, D.batch, D.gamma, lcap, Q.d, c->st));
-  SDD_TRY(gemm<T>(c, B.xf, Q.d, Q.wte, nullptr, (long long)D.batch * D.gamma, D.V, Q.d, EPI_STORE_F32, B.step_logits, D.V));
+  SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm_slots<T>(B.h, Q.lnf_g, Q.lnf_b, (T*)B.xf, B.ctx_len, D.batch, D.gamma, lcap, Q.d, c->st));
+  SDD_TRY(gemm<T>(c, CAT_HEAD_Q, B.xf, Q.d, Q.wte, nullptr, (long long)D.batch * D.gamma, D.V, Q.d, EPI_STORE_F32, B.step_logits, D.V));
   return SDD_OK;
 }
 
@@ -239,19 +274,19 @@ static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) 
   const Dims& D = c->D;
   if (rows_per_seq <= 0) return SDD_OK;
   const long long rows = (long long)D.batch * rows_per_seq;
-  SDD_LAUNCH(c, launch_embed_target<T>((const T*)P.wte, (const T*)P.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
+  SDD_LAUNCH(c, CAT_GLUE, launch_embed_target<T>((const T*)P.wte, (const T*)P.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
                                        D.batch, D.gamma, rows_per_seq, mode, P.d, B.h, c->st));
   const size_t layer_elems = (size_t)D.batch * P.n_ctx * 2 * P.d;
-  SDD_TRY((run_blocks<T>(c, P, rows, [&](int l) -> int {
+  SDD_TRY((run_blocks<T>(c, P, rows, CAT_GEMM_P, [&](int l) -> int {
     T* cache = (T*)B.kv + (size_t)l * layer_elems;
-    SDD_LAUNCH(c, launch_kv_append<T>((const T*)B.qkv, cache, B.ctx_len, D.batch, rows_per_seq, mode, P.n_ctx, P.d, c->st));
-    SDD_LAUNCH(c, launch_attn_cached<T>((const T*)B.qkv, cache, (T*)B.att, B.ctx_len, D.batch, rows_per_seq, mode, P.n_ctx,
+    SDD_LAUNCH(c, CAT_GLUE, launch_kv_append<T>((const T*)B.qkv, cache, B.ctx_len, D.batch, rows_per_seq, mode, P.n_ctx, P.d, c->st));
+    SDD_LAUNCH(c, CAT_ATTN_P, launch_attn_cached<T>((const T*)B.qkv, cache, (T*)B.att, B.ctx_len, D.batch, rows_per_seq, mode, P.n_ctx,
                                         P.n_head, P.d_head, c->st));
     return SDD_OK;
   })));
   if (lm_head) {
-    SDD_LAUNCH(c, launch_layernorm<T>(B.h, P.lnf_g, P.lnf_b, (T*)B.xf, rows, P.d, c->st));
-    SDD_TRY(gemm<T>(c, B.xf, P.d, P.wte, nullptr, rows, D.V, P.d, EPI_STORE_F32, B.logits_p, D.V));
+    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, P.lnf_g, P.lnf_b, (T*)B.xf, rows, P.d, c->st));
+    SDD_TRY(gemm<T>(c, CAT_HEAD_P, B.xf, P.d, P.wte, nullptr, rows, D.V, P.d, EPI_STORE_F32, B.logits_p, D.V));
   }
   return SDD_OK;
 }
@@ -290,7 +325,7 @@ static int draft_step_t(sdd_ctx* c) {
   const Dims& D = c->D;
   const int k = D.T - c->steps_done;
   SDD_TRY(forward_drafter<T>(c));
-  SDD_LAUNCH(c, launch_unmask_sample(B.step_logits, B.slot_ids, B.q_logits, B.logq, B.reveal_step, D.batch, D.gamma, D.V, k,
+  SDD_LAUNCH(c, CAT_SAMPLE, launch_unmask_sample(B.step_logits, B.slot_ids, B.q_logits, B.logq, B.reveal_step, D.batch, D.gamma, D.V, k,
                                      c->inv_tau_q, c->key, B.rs, c->st));
   c->steps_done++;
   return SDD_OK;
@@ -301,12 +336,12 @@ static int verify_accept_t(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
   const Buffers& B = c->B;
   const Dims& D = c->D;
   SDD_TRY(forward_target<T>(c, TARGET_VERIFY, D.gamma + 1, true));
-  SDD_LAUNCH(c, launch_row_stats(B.logits_p, (long long)D.batch * (D.gamma + 1), nullptr, 0, D.V, c->inv_tau_p, 0.f,
+  SDD_LAUNCH(c, CAT_STATS, launch_row_stats(B.logits_p, (long long)D.batch * (D.gamma + 1), nullptr, 0, D.V, c->inv_tau_p, 0.f,
                                  B.partial_p, c->st));
-  SDD_LAUNCH(c, launch_accept(B.logits_p, B.q_logits, B.slot_ids, B.logq, B.partial_p, nullptr, D.batch, D.gamma, D.V,
+  SDD_LAUNCH(c, CAT_ACCEPT, launch_accept(B.logits_p, B.q_logits, B.slot_ids, B.logq, B.partial_p, nullptr, D.batch, D.gamma, D.V,
                               c->inv_tau_p, c->inv_tau_p == 0.f ? 0.f : 1.f, c->key, 0u, B.rs, B.accept_prob, B.n_accept,
                               B.extra_token, nullptr, c->st));
-  SDD_LAUNCH(c, launch_commit(B.tokens, D.tok_stride, B.ctx_len, B.n_emitted, B.slot_ids, B.n_accept, B.extra_token,
+  SDD_LAUNCH(c, CAT_COMMIT, launch_commit(B.tokens, D.tok_stride, B.ctx_len, B.n_emitted, B.slot_ids, B.n_accept, B.extra_token,
                               D.batch, D.gamma, D.max_new, B.rs, out_ids, n_out, c->mirror_dev, c->st));
   return SDD_OK;
 }
@@ -358,6 +393,8 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
   c->steps_done = -1;
   c->rounds = 0;
   c->launches = 0;
+  c->profiling = false;
+  c->prof_used = 0;
   c->prompt_len.assign(prompt_len, prompt_len + params->batch);
   c->c_ub = c->prompt_len;
   const char* ra = getenv("SDD_RUNAHEAD");
@@ -399,7 +436,7 @@ int32_t sdd_draft_begin(sdd_ctx* c) {
   if (c->rounds >= (uint64_t)c->runahead)
     SDD_CUDA(cudaEventSynchronize(c->ev[(c->rounds - c->runahead) % c->ev.size()]));
   choose_lcap(c);
-  SDD_LAUNCH(c, launch_reset_slots(c->B.slot_ids, c->B.reveal_step, c->D.batch * c->D.gamma, c->D.V, c->st));
+  SDD_LAUNCH(c, CAT_GLUE, launch_reset_slots(c->B.slot_ids, c->B.reveal_step, c->D.batch * c->D.gamma, c->D.V, c->st));
   c->steps_done = 0;
   return SDD_OK;
 }
@@ -516,8 +553,35 @@ int32_t sdd_sync_status(sdd_ctx* c) {
   return status == DEV_TIMEOUT ? SDD_E_TIMEOUT : SDD_E_CTX_FULL;
 }
 
+int32_t sdd_profile_begin(sdd_ctx* c) {
+  if (c == nullptr) return SDD_E_ARG;
+  c->profiling = true;
+  c->prof_used = 0;
+  c->prof_cat.clear();
+  return SDD_OK;
+}
+
+int32_t sdd_profile_end(sdd_ctx* c, double* ms_per_category, uint64_t* launches_per_category, int32_t n_categories) {
+  if (c == nullptr || ms_per_category == nullptr || launches_per_category == nullptr) return SDD_E_ARG;
+  if (n_categories < CAT_COUNT) return SDD_E_ARG;
+  c->profiling = false;
+  SDD_CUDA(cudaStreamSynchronize(c->st));
+  for (int i = 0; i < n_categories; ++i) { ms_per_category[i] = 0.0; launches_per_category[i] = 0; }
+  for (size_t i = 0; i + 1 < c->prof_used + 1 && i / 2 < c->prof_cat.size(); i += 2) {
+    float ms = 0.f;
+    SDD_CUDA(cudaEventElapsedTime(&ms, c->prof_ev[i], c->prof_ev[i + 1]));
+    ms_per_category[c->prof_cat[i / 2]] += ms;
+    launches_per_category[c->prof_cat[i / 2]] += 1;
+  }
+  c->prof_used = 0;
+  c->prof_cat.clear();
+  return SDD_OK;
+}
+
 void sdd_destroy(sdd_ctx* c) {
   if (c == nullptr) return;
+  for (auto e : c->prof_ev)
+    if (e) cudaEventDestroy(e);
   for (auto e : c->ev)
     if (e) cudaEventDestroy(e);
   if (c->mirror) cudaFreeHost(c->mirror);
