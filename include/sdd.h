@@ -137,6 +137,29 @@ int32_t sdd_accept_logits(const float* logits_p, const float* logits_q, const in
                           uint64_t seed, uint64_t round, int32_t* n_accept, int32_t* out_ids,
                           float* accept_prob, void* scratch, void* stream);
 
+/* The same acceptance step for callers that cannot allocate device memory: code that runs where
+ * cudaMalloc is off limits (a host whose memory pool was sized and handed out up front, a
+ * real-time loop that must not enter the allocator, a plugin that is given its tensors and
+ * nothing else) still has to place the per-chunk statistics somewhere, so this entry point keeps
+ * them in a fixed array of SDD_ACCEPT_STATIC_SCRATCH_BYTES inside the library's device image.
+ * (This call is a convenience of the library; the paper has no counterpart.)
+ *   - Arguments and results are those of sdd_accept_logits, without `scratch`.
+ *   - Sizes with rows * (2 gamma + 1) * ceil((V + 3) / 8192) * 8 bytes above the fixed size are
+ *     refused with SDD_E_WORKSPACE; use sdd_accept_logits with your own scratch for those.
+ *   - Every GPU that loads the library holds the array until the process exits.
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current, as for every call here); make that first call before any stream capture.
+ *   - All calls share the one array: two calls whose kernels may overlap on the GPU (different
+ *     streams, or different host threads) race on it.  Calls on one stream are safe.  The array
+ *     keeps the previous call's contents; nothing in it needs clearing, because each call writes
+ *     every entry it later reads.
+ *   - It calls no allocation routine of CUDA or of any other library. */
+#define SDD_ACCEPT_STATIC_SCRATCH_BYTES (2u << 20)
+int32_t sdd_accept_logits_static(const float* logits_p, const float* logits_q, const int32_t* draft_ids,
+                                 int32_t rows, int32_t gamma, int32_t V, float temp_p, float temp_q,
+                                 uint64_t seed, uint64_t round, int32_t* n_accept, int32_t* out_ids,
+                                 float* accept_prob, void* stream);
+
 /* Read-only device views into the workspace, for inspection and tests. */
 enum {
   SDD_TAP_TOKENS = 0,      /* int32 [batch, tok_stride] context ids (prompt + emitted);

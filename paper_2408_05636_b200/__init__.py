@@ -31,6 +31,7 @@ PROF_NAMES = ["gemm_drafter", "gemm_target", "head_drafter", "head_target", "att
 EXPORTS = [
     "sdd_workspace_bytes", "sdd_create", "sdd_draft_begin", "sdd_draft_step", "sdd_draft",
     "sdd_verify_accept", "sdd_step", "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
+    "sdd_accept_logits_static",
     "sdd_tap", "sdd_counters", "sdd_profile_begin", "sdd_profile_end", "sdd_sync_status", "sdd_destroy", "sdd_strerror", "sdd_last_cuda_error",
 ]
 
@@ -77,6 +78,7 @@ def lib() -> C.CDLL:
         L.sdd_accept_scratch_bytes.argtypes = [i32, i32, i32]
         L.sdd_accept_scratch_bytes.restype = u64
         L.sdd_accept_logits.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, u64, u64, vp, vp, vp, vp, vp]
+        L.sdd_accept_logits_static.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, u64, u64, vp, vp, vp, vp]
         L.sdd_tap.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(u64)]
         L.sdd_counters.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
         L.sdd_profile_begin.argtypes = [vp]
@@ -163,6 +165,30 @@ def sdd_accept_logits(logits_p, logits_q, draft_ids, temp_p: float, temp_q: floa
                                    out_ids.data_ptr(), prob.data_ptr(), scratch.data_ptr(), st.cuda_stream),
            "sdd_accept_logits")
     return n_accept, out_ids, prob
+
+
+ACCEPT_STATIC_SCRATCH_BYTES = 2 << 20
+
+
+def sdd_accept_logits_static(logits_p, logits_q, draft_ids, n_accept, out_ids, accept_prob, temp_p: float,
+                             temp_q: float, seed: int, rnd: int, stream=None):
+    """sdd_accept_logits for callers that must not allocate on the device: the scratch is a fixed array inside
+    the library, and this wrapper allocates nothing either -- inputs AND outputs are the caller's CUDA tensors
+    (n_accept [rows] int32, out_ids [rows, gamma+1] int32, accept_prob [rows, gamma] fp32).  Problems whose
+    statistics do not fit ACCEPT_STATIC_SCRATCH_BYTES raise SddError(SDD_E_WORKSPACE).  Calls that may overlap on
+    the GPU share the scratch and race; make the first call on a device outside stream capture."""
+    torch = _torch()
+    rows, g1, V = logits_p.shape
+    gamma = g1 - 1
+    assert logits_q.shape == (rows, gamma, V) and draft_ids.shape == (rows, gamma)
+    assert n_accept.shape == (rows,) and out_ids.shape == (rows, gamma + 1) and accept_prob.shape == (rows, gamma)
+    for t in (logits_p, logits_q, draft_ids, n_accept, out_ids, accept_prob):
+        assert t.is_cuda and t.is_contiguous()
+    st = stream if stream is not None else torch.cuda.current_stream(logits_p.device)
+    _check(lib().sdd_accept_logits_static(logits_p.data_ptr(), logits_q.data_ptr(), draft_ids.data_ptr(), rows, gamma,
+                                          V, float(temp_p), float(temp_q), int(seed), int(rnd), n_accept.data_ptr(),
+                                          out_ids.data_ptr(), accept_prob.data_ptr(), st.cuda_stream),
+           "sdd_accept_logits_static")
 
 
 _TAP_DTYPES = {TAP_STEP_LOGITS: "f", TAP_Q_LOGITS: "f", TAP_LOGQ: "f", TAP_LOGITS_P: "f", TAP_ACCEPT_PROB: "f"}
