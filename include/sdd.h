@@ -160,6 +160,20 @@ int32_t sdd_accept_logits_static(const float* logits_p, const float* logits_q, c
                                  uint64_t seed, uint64_t round, int32_t* n_accept, int32_t* out_ids,
                                  float* accept_prob, void* stream);
 
+/* Diagnostic: the library's bf16 GEMM on its own,  C[M, N] = A[M, K] W[N, K]^T  with fp32 accumulation
+ * (the contraction used for the QKV / O / MLP / LM-head products of both networks' forwards).
+ *   A   device bf16, dense [a_rows_capacity, K] of which the first M rows are used
+ *   W   device bf16 [N, K];  bias device fp32 [N] or null
+ *   epilogue 0: out bf16 = acc + bias; 1: out bf16 = gelu_tanh(acc + bias);
+ *            2: out fp32 += acc + bias; 3: out fp32 = acc + bias       (out row stride ldc >= N)
+ *   n_tile   0 = let the library choose, else 32 / 64 / 128 / 256 (only for M > 64)
+ *   use_tensor_cores 1 = tcgen05 kernel, 0 = CUDA-core kernel
+ *   status_word device int32 (may be null): set to 1 if a bounded device-side wait expired
+ * K must be a multiple of 8; A and W 16-byte aligned. */
+int32_t sdd_debug_gemm_bf16(const void* A, int64_t a_rows_capacity, const void* W, const float* bias, int32_t M,
+                            int32_t N, int32_t K, int32_t epilogue, void* out, int32_t ldc, int32_t n_tile,
+                            int32_t use_tensor_cores, int32_t* status_word, void* stream);
+
 /* Read-only device views into the workspace, for inspection and tests. */
 enum {
   SDD_TAP_TOKENS = 0,      /* int32 [batch, tok_stride] context ids (prompt + emitted);

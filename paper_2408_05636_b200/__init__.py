@@ -31,7 +31,7 @@ PROF_NAMES = ["gemm_drafter", "gemm_target", "head_drafter", "head_target", "att
 EXPORTS = [
     "sdd_workspace_bytes", "sdd_create", "sdd_draft_begin", "sdd_draft_step", "sdd_draft",
     "sdd_verify_accept", "sdd_step", "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
-    "sdd_accept_logits_static",
+    "sdd_accept_logits_static", "sdd_debug_gemm_bf16",
     "sdd_tap", "sdd_counters", "sdd_profile_begin", "sdd_profile_end", "sdd_sync_status", "sdd_destroy", "sdd_strerror", "sdd_last_cuda_error",
 ]
 
@@ -79,6 +79,7 @@ def lib() -> C.CDLL:
         L.sdd_accept_scratch_bytes.restype = u64
         L.sdd_accept_logits.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, u64, u64, vp, vp, vp, vp, vp]
         L.sdd_accept_logits_static.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, u64, u64, vp, vp, vp, vp]
+        L.sdd_debug_gemm_bf16.argtypes = [vp, C.c_int64, vp, vp, i32, i32, i32, i32, vp, i32, i32, i32, vp, vp]
         L.sdd_tap.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(u64)]
         L.sdd_counters.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
         L.sdd_profile_begin.argtypes = [vp]
@@ -189,6 +190,19 @@ def sdd_accept_logits_static(logits_p, logits_q, draft_ids, n_accept, out_ids, a
                                           V, float(temp_p), float(temp_q), int(seed), int(rnd), n_accept.data_ptr(),
                                           out_ids.data_ptr(), accept_prob.data_ptr(), st.cuda_stream),
            "sdd_accept_logits_static")
+
+
+def sdd_debug_gemm_bf16(A, W, bias, M: int, epilogue: int, out, n_tile: int = 0, use_tensor_cores: bool = True,
+                        status=None, stream=None):
+    """out = epilogue(A[:M] @ W.T + bias) with the library's bf16 GEMM; A [cap, K], W [N, K] bf16 CUDA tensors."""
+    torch = _torch()
+    cap, K = A.shape
+    N = W.shape[0]
+    st = stream if stream is not None else torch.cuda.current_stream(A.device)
+    _check(lib().sdd_debug_gemm_bf16(A.data_ptr(), cap, W.data_ptr(), bias.data_ptr() if bias is not None else None, M, N,
+                                     K, epilogue, out.data_ptr(), out.stride(0), n_tile, 1 if use_tensor_cores else 0,
+                                     status.data_ptr() if status is not None else None, st.cuda_stream),
+           "sdd_debug_gemm_bf16")
 
 
 _TAP_DTYPES = {TAP_STEP_LOGITS: "f", TAP_Q_LOGITS: "f", TAP_LOGQ: "f", TAP_LOGITS_P: "f", TAP_ACCEPT_PROB: "f"}

@@ -4,6 +4,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <type_traits>
 #include <vector>
 
 #include "sdd_kernels.h"
@@ -153,6 +154,9 @@ struct sdd_ctx {
   std::vector<cudaEvent_t> ev;
   int runahead;
   int lcap;                    // padded rows per sequence of the current round's drafter forwards
+  size_t act_elems, xf_elems;  // capacity (elements) of the xn / att buffers (mlp: 4x) and of xf
+  bool force_simt;             // SDD_GEMM=simt: run bf16 GEMMs on the CUDA-core kernel (cross-check)
+  int bn_hint;                 // SDD_GEMM_BN: N tile of the tensor-core GEMM (0 = choose)
   // optional per-launch timing
   bool profiling;
   std::vector<cudaEvent_t> prof_ev;   // pairs (before, after)
@@ -211,13 +215,19 @@ static void fill_dims(const Net& P, const Net& Q, const sdd_params* p, int max_p
 }
 
 // ---- GEMM dispatch ----------------------------------------------------------------------------
+// `a_elems` is the capacity of the A buffer in elements (the tensor map of an activation buffer covers all of it)
 template <typename T>
-static int gemm(sdd_ctx* c, int cat, const void* A, int lda, const void* W, const float* bias, long long M, int N, int K,
-                int epi, void* out, int ldc) {
+static int gemm(sdd_ctx* c, int cat, const void* A, size_t a_elems, const void* W, const float* bias, long long M, int N,
+                int K, int epi, void* out, int ldc) {
   if (M <= 0) return SDD_OK;
   ProfScope prof(c, cat);
   c->launches++;
-  SDD_CUDA(launch_gemm_simt<T>((const T*)A, lda, (const T*)W, bias, (int)M, N, K, epi, out, ldc, c->st));
+  if (std::is_same<T, __nv_bfloat16>::value && !c->force_simt) {
+    SDD_CUDA(launch_gemm_tc((const __nv_bfloat16*)A, (long long)(a_elems / (size_t)K), (const __nv_bfloat16*)W, bias, (int)M,
+                            N, K, epi, out, ldc, c->bn_hint, &c->B.rs->status, c->st));
+  } else {
+    SDD_CUDA(launch_gemm_simt<T>((const T*)A, K, (const T*)W, bias, (int)M, N, K, epi, out, ldc, c->st));
+  }
   return SDD_OK;
 }
 
@@ -236,12 +246,12 @@ static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, AttnFn
   for (int l = 0; l < N.n_layer; ++l) {
     const Layer& L = N.layers[l];
     SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln1_g, L.ln1_b, (T*)B.xn, rows, d, c->st));
-    SDD_TRY(gemm<T>(c, gcat, B.xn, d, L.w_qkv, L.b_qkv, rows, 3 * d, d, EPI_STORE, B.qkv, 3 * d));
+    SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_qkv, L.b_qkv, rows, 3 * d, d, EPI_STORE, B.qkv, 3 * d));
     SDD_TRY(attn(l));
-    SDD_TRY(gemm<T>(c, gcat, B.att, d, L.w_o, L.b_o, rows, d, d, EPI_RESIDUAL, B.h, d));
+    SDD_TRY(gemm<T>(c, gcat, B.att, c->act_elems, L.w_o, L.b_o, rows, d, d, EPI_RESIDUAL, B.h, d));
     SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln2_g, L.ln2_b, (T*)B.xn, rows, d, c->st));
-    SDD_TRY(gemm<T>(c, gcat, B.xn, d, L.w_fc1, L.b_fc1, rows, 4 * d, d, EPI_GELU, B.mlp, 4 * d));
-    SDD_TRY(gemm<T>(c, gcat, B.mlp, 4 * d, L.w_fc2, L.b_fc2, rows, d, 4 * d, EPI_RESIDUAL, B.h, d));
+    SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_fc1, L.b_fc1, rows, 4 * d, d, EPI_GELU, B.mlp, 4 * d));
+    SDD_TRY(gemm<T>(c, gcat, B.mlp, 4 * c->act_elems, L.w_fc2, L.b_fc2, rows, d, 4 * d, EPI_RESIDUAL, B.h, d));
   }
   return SDD_OK;
 }
@@ -262,7 +272,7 @@ static int forward_drafter(sdd_ctx* c) {
     return SDD_OK;
   })));
   SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm_slots<T>(B.h, Q.lnf_g, Q.lnf_b, (T*)B.xf, B.ctx_len, D.batch, D.gamma, lcap, Q.d, c->st));
-  SDD_TRY(gemm<T>(c, CAT_HEAD_Q, B.xf, Q.d, Q.wte, nullptr, (long long)D.batch * D.gamma, D.V, Q.d, EPI_STORE_F32, B.step_logits, D.V));
+  SDD_TRY(gemm<T>(c, CAT_HEAD_Q, B.xf, c->xf_elems, Q.wte, nullptr, (long long)D.batch * D.gamma, D.V, Q.d, EPI_STORE_F32, B.step_logits, D.V));
   return SDD_OK;
 }
 
@@ -286,7 +296,7 @@ static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) 
   })));
   if (lm_head) {
     SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, P.lnf_g, P.lnf_b, (T*)B.xf, rows, P.d, c->st));
-    SDD_TRY(gemm<T>(c, CAT_HEAD_P, B.xf, P.d, P.wte, nullptr, rows, D.V, P.d, EPI_STORE_F32, B.logits_p, D.V));
+    SDD_TRY(gemm<T>(c, CAT_HEAD_P, B.xf, c->xf_elems, P.wte, nullptr, rows, D.V, P.d, EPI_STORE_F32, B.logits_p, D.V));
   }
   return SDD_OK;
 }
@@ -395,6 +405,16 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
   c->launches = 0;
   c->profiling = false;
   c->prof_used = 0;
+  {
+    const size_t rq = (size_t)c->D.rows_q, rp = (size_t)c->D.rows_p;
+    const size_t a = rq * c->Q.d, b = rp * c->P.d;
+    c->act_elems = a > b ? a : b;
+    c->xf_elems = (size_t)params->batch * (params->gamma + 1) * (c->Q.d > c->P.d ? c->Q.d : c->P.d);
+    const char* g = getenv("SDD_GEMM");
+    c->force_simt = g != nullptr && strcmp(g, "simt") == 0;
+    const char* bn = getenv("SDD_GEMM_BN");
+    c->bn_hint = bn ? atoi(bn) : 0;
+  }
   c->prompt_len.assign(prompt_len, prompt_len + params->batch);
   c->c_ub = c->prompt_len;
   const char* ra = getenv("SDD_RUNAHEAD");
@@ -511,6 +531,21 @@ int32_t sdd_accept_logits(const float* logits_p, const float* logits_q, const in
   SDD_CUDA(launch_row_stats(logits_p, rows_p, logits_q, itp == 0.f ? 0 : rows_q, V, itp, itq, partial, st));
   SDD_CUDA(launch_accept(logits_p, logits_q, draft_ids, nullptr, partial, partial + rows_p * chunks, rows, gamma, V, itp, itq,
                          make_key(seed), (uint32_t)round, nullptr, accept_prob, n_accept, nullptr, out_ids, st));
+  return SDD_OK;
+}
+
+int32_t sdd_debug_gemm_bf16(const void* A, int64_t a_rows_capacity, const void* W, const float* bias, int32_t M, int32_t N,
+                            int32_t K, int32_t epilogue, void* out, int32_t ldc, int32_t n_tile, int32_t use_tensor_cores,
+                            int32_t* status_word, void* stream) {
+  if (!A || !W || !out || M < 1 || N < 1 || K < 8 || (K % 8) != 0 || epilogue < 0 || epilogue > 3) return SDD_E_ARG;
+  if (a_rows_capacity < M || ldc < N) return SDD_E_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (use_tensor_cores)
+    SDD_CUDA(launch_gemm_tc((const __nv_bfloat16*)A, a_rows_capacity, (const __nv_bfloat16*)W, bias, M, N, K, epilogue, out,
+                            ldc, n_tile, status_word, st));
+  else
+    SDD_CUDA(launch_gemm_simt<__nv_bfloat16>((const __nv_bfloat16*)A, K, (const __nv_bfloat16*)W, bias, M, N, K, epilogue,
+                                             out, ldc, st));
   return SDD_OK;
 }
 

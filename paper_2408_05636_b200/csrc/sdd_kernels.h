@@ -67,6 +67,11 @@ template <typename T>
 cudaError_t launch_gemm_simt(const T* A, int lda, const T* W, const float* bias, int M, int N, int K, int epi, void* out,
                              int ldc, cudaStream_t st);
 
+// bf16 tensor-core GEMM (tcgen05 / TMEM / TMA).  A is a dense [a_cap, K] buffer of which M rows are used;
+// bn_hint selects the N tile (0 = choose); a bounded wait that expires sets *status = DEV_TIMEOUT.
+cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_bfloat16* W, const float* bias, int M, int N,
+                           int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st);
+
 // ---- attention (sdd_attn.cu) ----------------------------------------------------------------
 // drafter: every row of a sequence attends to rows 0 .. ctx_len[b] + gamma - 1 of the same sequence
 template <typename T>

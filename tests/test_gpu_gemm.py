@@ -1,0 +1,74 @@
+"""The bf16 tensor-core GEMM (tcgen05 / TMEM / TMA) against a plain fp32 matmul of the same bf16 inputs:
+all tile widths, both orientations (normal and swapped for few rows), ragged M / N, every epilogue."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+def _ref(A, W, bias, M, epi, out0):
+    acc = A[:M].float() @ W.float().t()
+    if bias is not None:
+        acc = acc + bias
+    if epi == 0:
+        return acc
+    if epi == 1:
+        return torch.nn.functional.gelu(acc, approximate="tanh")
+    if epi == 2:
+        return out0 + acc
+    return acc
+
+
+CASES = [
+    # M, N, K, n_tile
+    (128, 128, 64, 128), (128, 256, 128, 256), (300, 200, 192, 64), (257, 96, 768, 32), (384, 2304, 768, 0),
+    (400, 768, 3072, 0), (130, 50257, 128, 128),
+    # swapped orientation: M <= 64 rows
+    (1, 128, 64, 0), (17, 2304, 768, 0), (33, 1600, 1600, 0), (64, 777, 256, 0), (17, 50257, 768, 0),
+]
+
+
+@pytest.mark.parametrize("M,N,K,n_tile", CASES)
+def test_tc_gemm_matches_fp32_matmul(M, N, K, n_tile):
+    import paper_2408_05636_b200 as sdd
+    g = torch.Generator(device="cuda").manual_seed(M * 7 + N)
+    cap = M + 37
+    A = torch.randn(cap, K, device="cuda", generator=g).to(torch.bfloat16)
+    W = (torch.randn(N, K, device="cuda", generator=g) * 0.05).to(torch.bfloat16)
+    bias = torch.randn(N, device="cuda", generator=g)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    epis = (0, 1, 2, 3) if N < 10000 else (3,)
+    for epi in epis:
+        for b in (bias, None):
+            ldc = N + (8 if epi in (0, 1) else 3)
+            if epi in (0, 1):
+                out = torch.full((M, ldc), 7.0, device="cuda", dtype=torch.bfloat16)
+            else:
+                out = torch.randn(M, ldc, device="cuda", generator=g)
+            out0 = out[:, :N].float().clone()
+            sdd.sdd_debug_gemm_bf16(A, W, b, M, epi, out, n_tile, True, status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            ref = _ref(A, W, b, M, epi, out0)
+            got = out[:, :N].float()
+            tol = 2e-2 if epi in (0, 1) else 2e-3      # bf16 output rounding / fp32 accumulation order
+            err = (got - ref).abs().max().item()
+            scale = ref.abs().max().item()
+            assert err <= tol * max(1.0, scale), (epi, err, scale)
+            pad = out[:, N:].float()
+            if epi in (0, 1):
+                assert torch.all(pad == 7.0)            # nothing written past column N
+
+
+def test_simt_and_tc_agree():
+    import paper_2408_05636_b200 as sdd
+    g = torch.Generator(device="cuda").manual_seed(3)
+    A = torch.randn(200, 256, device="cuda", generator=g).to(torch.bfloat16)
+    W = (torch.randn(300, 256, device="cuda", generator=g) * 0.05).to(torch.bfloat16)
+    o1 = torch.zeros(200, 300, device="cuda")
+    o2 = torch.zeros(200, 300, device="cuda")
+    sdd.sdd_debug_gemm_bf16(A, W, None, 200, 3, o1, 0, True)
+    sdd.sdd_debug_gemm_bf16(A, W, None, 200, 3, o2, 0, False)
+    torch.cuda.synchronize()
+    assert (o1 - o2).abs().max().item() < 1e-3
