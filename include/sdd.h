@@ -174,6 +174,24 @@ int32_t sdd_debug_gemm_bf16(const void* A, int64_t a_rows_capacity, const void* 
                             int32_t N, int32_t K, int32_t epilogue, void* out, int32_t ldc, int32_t n_tile,
                             int32_t use_tensor_cores, int32_t* status_word, void* stream);
 
+/* Diagnostic: the library's bf16 tensor-core attention on its own (d_head = 64), as used inside both
+ * networks' blocks: out = softmax(Q K^T / 8 [+ mask]) V per head.
+ *   q   device bf16 [q_rows_total, q_ld]; head h occupies columns q_col0 + 64 h .. ; sequence b owns rows
+ *       b * q_rows_per_seq ..
+ *   k   device bf16 [k_rows_total, k_ld], heads from column k_col0, sequence b owns rows b * k_rows_per_seq ..
+ *   vt  device bf16 [batch * 64 n_head, vt_ld]: V transposed, row b * d + feature, column = key position
+ *       (entries past the valid keys must be finite)
+ *   out device bf16 [batch * q_rows_per_seq, ld_out]
+ *   mode 0: no mask, rows and keys 0 .. ctx_len[b] + gamma - 1 (the drafter);
+ *        1: row i is position ctx_len[b] - 1 + i and sees keys 0 .. that position (target verification);
+ *        2: row i is position i, valid while i < ctx_len[b] - 1 (target prefill).
+ * q_ld, k_ld, vt_ld, ld_out multiples of 8; all pointers 16-byte aligned. */
+int32_t sdd_debug_attention_bf16(const void* q, int64_t q_rows_total, int32_t q_ld, int32_t q_col0, const void* k,
+                                 int64_t k_rows_total, int32_t k_ld, int32_t k_col0, int32_t k_rows_per_seq,
+                                 const void* vt, int32_t vt_ld, void* out, int32_t ld_out, const int32_t* ctx_len,
+                                 int32_t batch, int32_t n_head, int32_t gamma, int32_t mode, int32_t q_rows_per_seq,
+                                 int32_t* status_word, void* stream);
+
 /* Read-only device views into the workspace, for inspection and tests. */
 enum {
   SDD_TAP_TOKENS = 0,      /* int32 [batch, tok_stride] context ids (prompt + emitted);

@@ -31,7 +31,7 @@ PROF_NAMES = ["gemm_drafter", "gemm_target", "head_drafter", "head_target", "att
 EXPORTS = [
     "sdd_workspace_bytes", "sdd_create", "sdd_draft_begin", "sdd_draft_step", "sdd_draft",
     "sdd_verify_accept", "sdd_step", "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
-    "sdd_accept_logits_static", "sdd_debug_gemm_bf16",
+    "sdd_accept_logits_static", "sdd_debug_gemm_bf16", "sdd_debug_attention_bf16",
     "sdd_tap", "sdd_counters", "sdd_profile_begin", "sdd_profile_end", "sdd_sync_status", "sdd_destroy", "sdd_strerror", "sdd_last_cuda_error",
 ]
 
@@ -80,6 +80,8 @@ def lib() -> C.CDLL:
         L.sdd_accept_logits.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, u64, u64, vp, vp, vp, vp, vp]
         L.sdd_accept_logits_static.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, u64, u64, vp, vp, vp, vp]
         L.sdd_debug_gemm_bf16.argtypes = [vp, C.c_int64, vp, vp, i32, i32, i32, i32, vp, i32, i32, i32, vp, vp]
+        L.sdd_debug_attention_bf16.argtypes = [vp, C.c_int64, i32, i32, vp, C.c_int64, i32, i32, i32, vp, i32, vp, i32, vp,
+                                               i32, i32, i32, i32, i32, vp, vp]
         L.sdd_tap.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(u64)]
         L.sdd_counters.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
         L.sdd_profile_begin.argtypes = [vp]
@@ -203,6 +205,18 @@ def sdd_debug_gemm_bf16(A, W, bias, M: int, epilogue: int, out, n_tile: int = 0,
                                      K, epilogue, out.data_ptr(), out.stride(0), n_tile, 1 if use_tensor_cores else 0,
                                      status.data_ptr() if status is not None else None, st.cuda_stream),
            "sdd_debug_gemm_bf16")
+
+
+def sdd_debug_attention_bf16(q, q_col0, k, k_col0, k_rows_per_seq, vt, out, ctx_len, batch, n_head, gamma, mode,
+                             q_rows_per_seq, status=None, stream=None):
+    """The library's tensor-core attention on caller tensors (see include/sdd.h for the layouts)."""
+    torch = _torch()
+    st = stream if stream is not None else torch.cuda.current_stream(q.device)
+    _check(lib().sdd_debug_attention_bf16(q.data_ptr(), q.shape[0], q.stride(0), q_col0, k.data_ptr(), k.shape[0],
+                                          k.stride(0), k_col0, k_rows_per_seq, vt.data_ptr(), vt.stride(0),
+                                          out.data_ptr(), out.stride(0), ctx_len.data_ptr(), batch, n_head, gamma, mode,
+                                          q_rows_per_seq, status.data_ptr() if status is not None else None,
+                                          st.cuda_stream), "sdd_debug_attention_bf16")
 
 
 _TAP_DTYPES = {TAP_STEP_LOGITS: "f", TAP_Q_LOGITS: "f", TAP_LOGQ: "f", TAP_LOGITS_P: "f", TAP_ACCEPT_PROB: "f"}

@@ -87,6 +87,7 @@ struct Buffers {
   float2* partial_p;
   float* h;                    // residual stream, fp32
   void *xn, *qkv, *att, *mlp, *xf;  // activations in the model dtype
+  void* vt;                    // drafter V transposed [batch][d_q][lcap_max] (tensor-core path)
   void* kv;                    // target KV cache [layer][batch][n_ctx][2][d]
 };
 
@@ -129,6 +130,7 @@ static size_t carve(const Dims& D, const Net& P, const Net& Q, uint8_t* base, Bu
   b.att = take(mx(rq * Q.d, rp * P.d) * D.esize);
   b.mlp = take(mx(rq * Q.d, rp * P.d) * 4 * D.esize);
   b.xf = take(Bn * (G + 1) * mx(Q.d, P.d) * D.esize);
+  b.vt = take(Bn * (size_t)Q.d * D.lcap_max * D.esize);
   b.kv = take((size_t)P.n_layer * Bn * P.n_ctx * 2 * P.d * D.esize);
   if (B) *B = b;
   return off;
@@ -218,17 +220,23 @@ static void fill_dims(const Net& P, const Net& Q, const sdd_params* p, int max_p
 // `a_elems` is the capacity of the A buffer in elements (the tensor map of an activation buffer covers all of it)
 template <typename T>
 static int gemm(sdd_ctx* c, int cat, const void* A, size_t a_elems, const void* W, const float* bias, long long M, int N,
-                int K, int epi, void* out, int ldc) {
+                int K, int epi, void* out, int ldc, const QkvDst* qd = nullptr) {
   if (M <= 0) return SDD_OK;
   ProfScope prof(c, cat);
   c->launches++;
   if (std::is_same<T, __nv_bfloat16>::value && !c->force_simt) {
     SDD_CUDA(launch_gemm_tc((const __nv_bfloat16*)A, (long long)(a_elems / (size_t)K), (const __nv_bfloat16*)W, bias, (int)M,
-                            N, K, epi, out, ldc, c->bn_hint, &c->B.rs->status, c->st));
+                            N, K, epi, out, ldc, c->bn_hint, &c->B.rs->status, c->st, qd));
   } else {
     SDD_CUDA(launch_gemm_simt<T>((const T*)A, K, (const T*)W, bias, (int)M, N, K, epi, out, ldc, c->st));
   }
   return SDD_OK;
+}
+
+// the tensor-core path (tcgen05 GEMMs with the fused QKV epilogue + tensor-core attention) needs bf16 and d_head 64
+template <typename T>
+static bool use_tc(const sdd_ctx* c, const Net& N) {
+  return std::is_same<T, __nv_bfloat16>::value && !c->force_simt && N.d_head == 64;
 }
 
 #define SDD_LAUNCH(c, cat, expr) \
@@ -239,14 +247,17 @@ static int gemm(sdd_ctx* c, int cat, const void* A, size_t a_elems, const void* 
   } while (0)
 
 // one transformer block on `rows` rows; attention is issued by the caller-supplied functor
-template <typename T, typename AttnFn>
-static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, AttnFn attn) {
+template <typename T, typename QkvFn, typename AttnFn>
+static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, QkvFn qkv_dst, AttnFn attn) {
   const Buffers& B = c->B;
   const int d = N.d;
   for (int l = 0; l < N.n_layer; ++l) {
     const Layer& L = N.layers[l];
     SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln1_g, L.ln1_b, (T*)B.xn, rows, d, c->st));
-    SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_qkv, L.b_qkv, rows, 3 * d, d, EPI_STORE, B.qkv, 3 * d));
+    QkvDst qd = {};
+    const bool fused = qkv_dst(l, &qd);
+    SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_qkv, L.b_qkv, rows, 3 * d, d, fused ? EPI_QKV : EPI_STORE, B.qkv,
+                    3 * d, fused ? &qd : nullptr));
     SDD_TRY(attn(l));
     SDD_TRY(gemm<T>(c, gcat, B.att, c->act_elems, L.w_o, L.b_o, rows, d, d, EPI_RESIDUAL, B.h, d));
     SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln2_g, L.ln2_b, (T*)B.xn, rows, d, c->st));
@@ -266,11 +277,27 @@ static int forward_drafter(sdd_ctx* c) {
   const long long rows = (long long)D.batch * lcap;
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_drafter<T>((const T*)Q.wte, (const T*)Q.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
                                         D.batch, D.gamma, lcap, Q.d, B.h, c->st));
-  SDD_TRY((run_blocks<T>(c, Q, rows, CAT_GEMM_Q, [&](int) -> int {
-    SDD_LAUNCH(c, CAT_ATTN_Q, launch_attn_bidir<T>((const T*)B.qkv, (T*)B.att, B.ctx_len, D.batch, D.gamma, lcap, Q.n_head, Q.d_head,
-                                       c->st));
-    return SDD_OK;
-  })));
+  const bool tc = use_tc<T>(c, Q);
+  SDD_TRY((run_blocks<T>(c, Q, rows, CAT_GEMM_Q,
+    [&](int, QkvDst* qd) -> bool {
+      if (!tc) return false;
+      qd->k_dst = nullptr; qd->vt_dst = (__nv_bfloat16*)B.vt; qd->ctx_len = B.ctx_len; qd->rows_per_seq = lcap;
+      qd->mode = 0; qd->d = Q.d; qd->k_seq_rows = 0; qd->vt_ld = D.lcap_max;
+      return true;
+    },
+    [&](int) -> int {
+      if (tc) {
+        const __nv_bfloat16* qkv = (const __nv_bfloat16*)B.qkv;
+        SDD_LAUNCH(c, CAT_ATTN_Q, launch_attn_tc(qkv, (long long)(c->act_elems / Q.d), 3 * Q.d, 0, qkv,
+                                                 (long long)(c->act_elems / Q.d), 3 * Q.d, Q.d, lcap,
+                                                 (const __nv_bfloat16*)B.vt, D.lcap_max, (__nv_bfloat16*)B.att, Q.d, B.ctx_len,
+                                                 D.batch, Q.n_head, Q.d, D.gamma, 0, lcap, &B.rs->status, c->st));
+      } else {
+        SDD_LAUNCH(c, CAT_ATTN_Q, launch_attn_bidir<T>((const T*)B.qkv, (T*)B.att, B.ctx_len, D.batch, D.gamma, lcap, Q.n_head,
+                                                       Q.d_head, c->st));
+      }
+      return SDD_OK;
+    })));
   SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm_slots<T>(B.h, Q.lnf_g, Q.lnf_b, (T*)B.xf, B.ctx_len, D.batch, D.gamma, lcap, Q.d, c->st));
   SDD_TRY(gemm<T>(c, CAT_HEAD_Q, B.xf, c->xf_elems, Q.wte, nullptr, (long long)D.batch * D.gamma, D.V, Q.d, EPI_STORE_F32, B.step_logits, D.V));
   return SDD_OK;
@@ -287,13 +314,33 @@ static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) 
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_target<T>((const T*)P.wte, (const T*)P.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
                                        D.batch, D.gamma, rows_per_seq, mode, P.d, B.h, c->st));
   const size_t layer_elems = (size_t)D.batch * P.n_ctx * 2 * P.d;
-  SDD_TRY((run_blocks<T>(c, P, rows, CAT_GEMM_P, [&](int l) -> int {
-    T* cache = (T*)B.kv + (size_t)l * layer_elems;
-    SDD_LAUNCH(c, CAT_GLUE, launch_kv_append<T>((const T*)B.qkv, cache, B.ctx_len, D.batch, rows_per_seq, mode, P.n_ctx, P.d, c->st));
-    SDD_LAUNCH(c, CAT_ATTN_P, launch_attn_cached<T>((const T*)B.qkv, cache, (T*)B.att, B.ctx_len, D.batch, rows_per_seq, mode, P.n_ctx,
-                                        P.n_head, P.d_head, c->st));
-    return SDD_OK;
-  })));
+  const bool tc = use_tc<T>(c, P);
+  // tensor-core path: per layer the cache is K [B][n_ctx][d] followed by V^T [B][d][n_ctx];
+  // CUDA-core path: [B][n_ctx][K|V][d]
+  SDD_TRY((run_blocks<T>(c, P, rows, CAT_GEMM_P,
+    [&](int l, QkvDst* qd) -> bool {
+      if (!tc) return false;
+      __nv_bfloat16* kc = (__nv_bfloat16*)B.kv + (size_t)l * layer_elems;
+      qd->k_dst = kc; qd->vt_dst = kc + layer_elems / 2; qd->ctx_len = B.ctx_len; qd->rows_per_seq = rows_per_seq;
+      qd->mode = mode == TARGET_VERIFY ? 1 : 2; qd->d = P.d; qd->k_seq_rows = P.n_ctx; qd->vt_ld = P.n_ctx;
+      return true;
+    },
+    [&](int l) -> int {
+      T* cache = (T*)B.kv + (size_t)l * layer_elems;
+      if (tc) {
+        const __nv_bfloat16* kc = (const __nv_bfloat16*)cache;
+        SDD_LAUNCH(c, CAT_ATTN_P, launch_attn_tc((const __nv_bfloat16*)B.qkv, (long long)(c->act_elems / P.d), 3 * P.d, 0, kc,
+                                                 (long long)D.batch * P.n_ctx, P.d, 0, P.n_ctx, kc + layer_elems / 2, P.n_ctx,
+                                                 (__nv_bfloat16*)B.att, P.d, B.ctx_len, D.batch, P.n_head, P.d, D.gamma,
+                                                 mode == TARGET_VERIFY ? 1 : 2, rows_per_seq, &B.rs->status, c->st));
+      } else {
+        SDD_LAUNCH(c, CAT_GLUE, launch_kv_append<T>((const T*)B.qkv, cache, B.ctx_len, D.batch, rows_per_seq, mode, P.n_ctx, P.d,
+                                                    c->st));
+        SDD_LAUNCH(c, CAT_ATTN_P, launch_attn_cached<T>((const T*)B.qkv, cache, (T*)B.att, B.ctx_len, D.batch, rows_per_seq, mode,
+                                                        P.n_ctx, P.n_head, P.d_head, c->st));
+      }
+      return SDD_OK;
+    })));
   if (lm_head) {
     SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, P.lnf_g, P.lnf_b, (T*)B.xf, rows, P.d, c->st));
     SDD_TRY(gemm<T>(c, CAT_HEAD_P, B.xf, c->xf_elems, P.wte, nullptr, rows, D.V, P.d, EPI_STORE_F32, B.logits_p, D.V));
@@ -435,6 +482,9 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
   SDD_CUDA(cudaMemsetAsync(workspace, 0, state_bytes, c->st));
   const size_t act_bytes = (size_t)((uint8_t*)B.kv - (uint8_t*)B.h);
   SDD_CUDA(cudaMemsetAsync(B.h, 0, act_bytes, c->st));
+  // the tensor-core attention multiplies masked probabilities (exact zeros) with whatever the V^T cache holds
+  // past the valid positions, so that memory must be finite
+  SDD_CUDA(cudaMemsetAsync(B.kv, 0, (size_t)c->P.n_layer * params->batch * c->P.n_ctx * 2 * c->P.d * c->D.esize, c->st));
   SDD_CUDA(cudaMemcpy2DAsync(B.tokens, (size_t)c->D.tok_stride * 4, prompt_ids, (size_t)prompt_stride * 4,
                              (size_t)max_prompt * 4, params->batch, cudaMemcpyDeviceToDevice, c->st));
   SDD_CUDA(cudaMemcpyAsync(B.ctx_len, prompt_len, (size_t)params->batch * 4, cudaMemcpyHostToDevice, c->st));
@@ -546,6 +596,18 @@ int32_t sdd_debug_gemm_bf16(const void* A, int64_t a_rows_capacity, const void* 
   else
     SDD_CUDA(launch_gemm_simt<__nv_bfloat16>((const __nv_bfloat16*)A, K, (const __nv_bfloat16*)W, bias, M, N, K, epilogue,
                                              out, ldc, st));
+  return SDD_OK;
+}
+
+int32_t sdd_debug_attention_bf16(const void* q, int64_t q_rows_total, int32_t q_ld, int32_t q_col0, const void* k,
+                                 int64_t k_rows_total, int32_t k_ld, int32_t k_col0, int32_t k_rows_per_seq, const void* vt,
+                                 int32_t vt_ld, void* out, int32_t ld_out, const int32_t* ctx_len, int32_t batch,
+                                 int32_t n_head, int32_t gamma, int32_t mode, int32_t q_rows_per_seq, int32_t* status_word,
+                                 void* stream) {
+  if (!q || !k || !vt || !out || !ctx_len || batch < 1 || n_head < 1 || mode < 0 || mode > 2) return SDD_E_ARG;
+  SDD_CUDA(launch_attn_tc((const __nv_bfloat16*)q, q_rows_total, q_ld, q_col0, (const __nv_bfloat16*)k, k_rows_total, k_ld,
+                          k_col0, k_rows_per_seq, (const __nv_bfloat16*)vt, vt_ld, (__nv_bfloat16*)out, ld_out, ctx_len, batch,
+                          n_head, n_head * 64, gamma, mode, q_rows_per_seq, status_word, (cudaStream_t)stream));
   return SDD_OK;
 }
 

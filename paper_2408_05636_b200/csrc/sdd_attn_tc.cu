@@ -1,0 +1,268 @@
+// Tensor-core attention for sm_100a (bf16 in, fp32 soft-max state), d_head = 64.
+//
+// One CTA owns 128 query rows of one head of one sequence and walks over the keys in tiles of 128:
+//   S  = Q K^T          tcgen05.mma, 128 x 128 fp32 accumulator in TMEM (Q, K tiles via TMA, K-major)
+//   P  = exp2(S - max)  four soft-max warps, one thread per query row (tcgen05.ld gives a thread its row);
+//                       P is written as bf16 into shared memory in the 128-byte-swizzled K-major layout
+//   PV = P V            tcgen05.mma with V^T tiles ([d_head, keys], keys contiguous) as the second operand,
+//                       64-column fp32 accumulator in TMEM, folded into the per-thread output row with the
+//                       usual online-soft-max correction.
+// The same kernel serves the drafter (no mask: every row sees every row of its sequence) and the target
+// (row at position p sees cache positions 0..p).  V is consumed transposed, which the QKV GEMM's epilogue
+// produces for free; that keeps both MMAs on K-major operands.
+// Waits are bounded exactly as in the GEMM kernel.
+#include "sdd_kernels.h"
+#include "sdd_tc.cuh"
+
+namespace sdd {
+namespace tc {
+
+constexpr int AT_THREADS = 192;
+constexpr int AT_DH = 64;
+constexpr int AT_Q_BYTES = 128 * 64 * 2;            // 16 KB
+constexpr int AT_P_BYTES = 2 * 128 * 64 * 2;        // two k-blocks of 64 keys: 32 KB
+constexpr int AT_K_BYTES = 128 * 64 * 2;            // 16 KB
+constexpr int AT_VT_BYTES = 2 * 64 * 64 * 2;        // two boxes [64 d_head rows x 64 keys]: 16 KB
+constexpr int AT_STAGE_BYTES = AT_K_BYTES + AT_VT_BYTES;
+constexpr int AT_KV_STAGES = 2;
+constexpr int AT_BAR_OFF = AT_Q_BYTES + AT_P_BYTES + AT_KV_STAGES * AT_STAGE_BYTES;   // 112 KB
+constexpr int AT_SMEM = AT_BAR_OFF + 1024 + 256;
+constexpr uint32_t AT_TMEM_COLS = 256;              // S: columns 0..127, PV: columns 128..191
+
+struct AttnParams {
+  __nv_bfloat16* out;
+  int ld_out;
+  const int* ctx_len;
+  int mode;             // 0: drafter, no mask; 1: target verify (position c-1+i); 2: target prefill (position i)
+  int gamma;
+  int q_rows_per_seq;   // rows of one sequence in the Q tensor and in out
+  int k_rows_per_seq;   // rows of one sequence in the K tensor
+  int q_col0, k_col0;   // column of head 0 in the Q / K tensors
+  int d;                // model width = rows of one sequence in the V^T tensor
+  int* status;
+};
+
+__global__ void __launch_bounds__(AT_THREADS)
+attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+               const __grid_constant__ CUtensorMap map_vt, const AttnParams prm) {
+  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int c = prm.ctx_len[b];
+  const int q0 = qt * 128;
+  int n_valid_q;
+  if (prm.mode == 0) n_valid_q = c + prm.gamma;
+  else if (prm.mode == 1) n_valid_q = prm.q_rows_per_seq;
+  else n_valid_q = c - 1;
+  if (n_valid_q > prm.q_rows_per_seq) n_valid_q = prm.q_rows_per_seq;
+  if (q0 >= n_valid_q) return;                       // padding tile (uniform for the CTA)
+  const int last_valid = (n_valid_q < q0 + 128 ? n_valid_q : q0 + 128) - 1;
+  int n_keys_cta;
+  if (prm.mode == 0) n_keys_cta = c + prm.gamma;
+  else if (prm.mode == 1) n_keys_cta = c - 1 + last_valid + 1;
+  else n_keys_cta = last_valid + 1;
+  if (n_keys_cta > prm.k_rows_per_seq) n_keys_cta = prm.k_rows_per_seq;
+  const int num_kt = (n_keys_cta + 127) / 128;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t sQ = base, sP = base + AT_Q_BYTES;
+  auto sK = [&](int s) { return base + AT_Q_BYTES + AT_P_BYTES + s * AT_STAGE_BYTES; };
+  auto sVT = [&](int s) { return sK(s) + AT_K_BYTES; };
+  const uint32_t bars = base + AT_BAR_OFF;
+  const uint32_t q_full = bars, s_full = bars + 8, p_ready = bars + 16, pv_full = bars + 24;
+  auto kv_full = [&](int s) { return bars + 32 + 8u * s; };
+  auto kv_empty = [&](int s) { return bars + 48 + 8u * s; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + AT_BAR_OFF + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + AT_BAR_OFF + 72);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1); mbar_init(s_full, 1); mbar_init(p_ready, 128); mbar_init(pv_full, 1);
+    for (int s = 0; s < AT_KV_STAGES; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, AT_TMEM_COLS);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(q_full, AT_Q_BYTES);
+      tma_load_2d(sQ, &map_q, q_full, prm.q_col0 + h * AT_DH, b * prm.q_rows_per_seq + q0);
+      int issued = 0;
+      for (int t = 0; t < num_kt; ++t) {
+        const int s = t & 1;
+        if (!mbar_wait(kv_empty(s), ((uint32_t)(t >> 1) & 1u) ^ 1u, abort_flag, prm.status)) break;
+        mbar_expect_tx(kv_full(s), AT_STAGE_BYTES);
+        tma_load_2d(sK(s), &map_k, kv_full(s), prm.k_col0 + h * AT_DH, b * prm.k_rows_per_seq + t * 128);
+        tma_load_2d(sVT(s), &map_vt, kv_full(s), t * 128, b * prm.d + h * AT_DH);
+        tma_load_2d(sVT(s) + 64 * 64 * 2, &map_vt, kv_full(s), t * 128 + 64, b * prm.d + h * AT_DH);
+        issued = t + 1;
+      }
+      if (*abort_flag) {   // do not leave while copies into this CTA's shared memory may be in flight
+        long long t0 = clock64();
+        while (!mbar_try(q_full, 0u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        for (int t = issued > AT_KV_STAGES ? issued - AT_KV_STAGES : 0; t < issued; ++t) {
+          t0 = clock64();
+          while (!mbar_try(kv_full(t & 1), (uint32_t)(t >> 1) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc<128>();
+      constexpr uint32_t idesc_pv = make_idesc<64>();
+      bool ok = mbar_wait(q_full, 0u, abort_flag, prm.status);
+      const uint64_t dq = make_smem_desc(sQ);
+      for (int t = 0; t < num_kt && ok; ++t) {
+        const int s = t & 1;
+        ok = mbar_wait(kv_full(s), (uint32_t)(t >> 1) & 1u, abort_flag, prm.status);
+        if (!ok) break;
+        fence_after_sync();
+        const uint64_t dk = make_smem_desc(sK(s));
+#pragma unroll
+        for (int k = 0; k < 4; ++k) umma(tmem_base, dq + 2u * k, dk + 2u * k, idesc_s, k > 0 ? 1u : 0u);
+        umma_commit(s_full);
+        ok = mbar_wait(p_ready, (uint32_t)t & 1u, abort_flag, prm.status);
+        if (!ok) break;
+        fence_after_sync();
+#pragma unroll
+        for (int kb = 0; kb < 2; ++kb) {
+          const uint64_t dp = make_smem_desc(sP + kb * (128 * 64 * 2));
+          const uint64_t dv = make_smem_desc(sVT(s) + kb * (64 * 64 * 2));
+#pragma unroll
+          for (int k = 0; k < 4; ++k) umma(tmem_base + 128u, dp + 2u * k, dv + 2u * k, idesc_pv, (kb | k) ? 1u : 0u);
+        }
+        umma_commit(pv_full);
+        umma_commit(kv_empty(s));
+      }
+    }
+  } else {
+    const int r = (warp & 3) * 32 + lane;
+    const int i = q0 + r;
+    const bool valid = i < n_valid_q;
+    int key_limit;                                     // keys [0, key_limit) are visible to this row
+    if (prm.mode == 0) key_limit = n_keys_cta;
+    else if (prm.mode == 1) key_limit = c - 1 + i + 1;
+    else key_limit = i + 1;
+    if (key_limit > n_keys_cta) key_limit = n_keys_cta;
+    if (!valid) key_limit = 0;
+    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const float scale = 0.125f * 1.4426950408889634f;  // 1/sqrt(64) * log2(e)
+    float m = -INFINITY, l = 0.f;
+    float o[AT_DH];
+#pragma unroll
+    for (int j = 0; j < AT_DH; ++j) o[j] = 0.f;
+    uint8_t* p_row = gbase + AT_Q_BYTES + r * 128;
+    const int sw = r & 7;
+    bool ok = true;
+    for (int t = 0; t < num_kt; ++t) {
+      ok = __all_sync(0xffffffffu, mbar_wait(s_full, (uint32_t)t & 1u, abort_flag, prm.status));
+      if (!ok) break;
+      fence_after_sync();
+      const int key0 = t * 128;
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t v[32];
+        tmem_ld32(t_lane + (uint32_t)(cc * 32), v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (key0 + cc * 32 + j < key_limit) mx = fmaxf(mx, __uint_as_float(v[j]));
+      }
+      const float m_new = fmaxf(m, mx * scale);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;
+      const float corr = m == -INFINITY ? 0.f : exp2f(m - m_use);
+      float sum = 0.f;
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t v[32];
+        tmem_ld32(t_lane + (uint32_t)(cc * 32), v);
+        uint8_t* blk = p_row + (cc >> 1) * (128 * 64 * 2);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int j0 = g * 8 + 2 * e;
+            const float p0 = (key0 + cc * 32 + j0 < key_limit) ? exp2f(fmaf(__uint_as_float(v[j0]), scale, -m_use)) : 0.f;
+            const float p1 = (key0 + cc * 32 + j0 + 1 < key_limit) ? exp2f(fmaf(__uint_as_float(v[j0 + 1]), scale, -m_use)) : 0.f;
+            sum += p0 + p1;
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+          }
+          const int chunk = (cc & 1) * 4 + g;           // 16-byte chunk of this row inside the 64-key block
+          *reinterpret_cast<uint4*>(blk + ((chunk ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+      }
+      l = l * corr + sum;
+      m = m_new;
+      fence_async_smem();
+      mbar_arrive(p_ready);
+      ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)t & 1u, abort_flag, prm.status));
+      if (!ok) break;
+      fence_after_sync();
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        uint32_t v[32];
+        tmem_ld32(t_lane + 128u + (uint32_t)(cc * 32), v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) o[cc * 32 + j] = fmaf(o[cc * 32 + j], corr, __uint_as_float(v[j]));
+      }
+    }
+    if (ok && valid) {
+      const float inv = 1.f / l;
+      __nv_bfloat16* dst = prm.out + ((long long)b * prm.q_rows_per_seq + i) * prm.ld_out + h * AT_DH;
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __nv_bfloat162 h2 = __floats2bfloat162_rn(o[g * 8 + 2 * e] * inv, o[g * 8 + 2 * e + 1] * inv);
+          pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+        }
+        *reinterpret_cast<uint4*>(dst + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      }
+    }
+  }
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    fence_after_sync();
+    tmem_dealloc(tmem_base, AT_TMEM_COLS);
+  }
+}
+
+}  // namespace tc
+
+cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q_ld, int q_col0, const __nv_bfloat16* k,
+                           long long k_rows_total, int k_ld, int k_col0, int k_rows_per_seq, const __nv_bfloat16* vt,
+                           int vt_ld, __nv_bfloat16* out, int ld_out, const int* ctx_len, int batch, int n_head, int d,
+                           int gamma, int mode, int q_rows_per_seq, int* status, cudaStream_t st) {
+  using namespace tc;
+  if (q_rows_per_seq <= 0) return cudaSuccess;
+  if (d != n_head * AT_DH || (ld_out & 7) != 0) return cudaErrorInvalidValue;
+  CUtensorMap mq, mk, mv;
+  cudaError_t e;
+  if ((e = get_tensor_map(q, q_rows_total, q_ld, q_ld, 128, 64, &mq)) != cudaSuccess) return e;
+  if ((e = get_tensor_map(k, k_rows_total, k_ld, k_ld, 128, 64, &mk)) != cudaSuccess) return e;
+  if ((e = get_tensor_map(vt, (long long)batch * d, vt_ld, vt_ld, 64, 64, &mv)) != cudaSuccess) return e;
+  static bool attr_set = false;
+  if (!attr_set) {
+    e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  AttnParams p;
+  p.out = out; p.ld_out = ld_out; p.ctx_len = ctx_len; p.mode = mode; p.gamma = gamma;
+  p.q_rows_per_seq = q_rows_per_seq; p.k_rows_per_seq = k_rows_per_seq; p.q_col0 = q_col0; p.k_col0 = k_col0;
+  p.d = d; p.status = status;
+  dim3 grid((q_rows_per_seq + 127) / 128, n_head, batch);
+  attn_tc_kernel<<<grid, AT_THREADS, AT_SMEM, st>>>(mq, mk, mv, p);
+  return cudaGetLastError();
+}
+
+}  // namespace sdd

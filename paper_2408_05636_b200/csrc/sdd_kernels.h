@@ -22,7 +22,19 @@ enum Epilogue : int {
   EPI_STORE = 0,      // out (activation type) = acc + bias
   EPI_GELU = 1,       // out (activation type) = gelu_tanh(acc + bias)
   EPI_RESIDUAL = 2,   // resid (fp32) += acc + bias
-  EPI_STORE_F32 = 3   // out (fp32) = acc            (LM head; ldc may differ from N)
+  EPI_STORE_F32 = 3,  // out (fp32) = acc            (LM head; ldc may differ from N)
+  EPI_QKV = 4         // fused-QKV projection of the tensor-core path: Q (and the drafter's K) to `out`,
+                      // the target's K to its cache, V transposed ([feature][position]) -- see QkvDst
+};
+
+// Destinations of the EPI_QKV epilogue.  Token row tr belongs to sequence b = tr / rows_per_seq at local
+// index i = tr % rows_per_seq; its position is i (mode 0 drafter, mode 2 prefill, valid while i < c - 1)
+// or c - 1 + i (mode 1 verify), with c = ctx_len[b].
+struct QkvDst {
+  __nv_bfloat16* k_dst;   // null: K is stored to `out` next to Q; else K cache [B][k_seq_rows][d]
+  __nv_bfloat16* vt_dst;  // V^T [B][d][vt_ld]
+  const int* ctx_len;
+  int rows_per_seq, mode, d, k_seq_rows, vt_ld;
 };
 
 // ---- vocabulary kernels (sdd_sample.cu) -----------------------------------------------------
@@ -70,7 +82,16 @@ cudaError_t launch_gemm_simt(const T* A, int lda, const T* W, const float* bias,
 // bf16 tensor-core GEMM (tcgen05 / TMEM / TMA).  A is a dense [a_cap, K] buffer of which M rows are used;
 // bn_hint selects the N tile (0 = choose); a bounded wait that expires sets *status = DEV_TIMEOUT.
 cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_bfloat16* W, const float* bias, int M, int N,
-                           int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st);
+                           int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st,
+                           const QkvDst* qkv = nullptr);
+
+// bf16 tensor-core attention, d_head = 64 (sdd_attn_tc.cu).  q / k are row-major tensors with the heads side by
+// side starting at column q_col0 / k_col0; vt is V transposed: [batch * d rows, vt_ld positions].
+// mode 0: drafter (no mask, ctx_len[b] + gamma rows and keys); 1: target verify; 2: target prefill.
+cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q_ld, int q_col0, const __nv_bfloat16* k,
+                           long long k_rows_total, int k_ld, int k_col0, int k_rows_per_seq, const __nv_bfloat16* vt,
+                           int vt_ld, __nv_bfloat16* out, int ld_out, const int* ctx_len, int batch, int n_head, int d,
+                           int gamma, int mode, int q_rows_per_seq, int* status, cudaStream_t st);
 
 // ---- attention (sdd_attn.cu) ----------------------------------------------------------------
 // drafter: every row of a sequence attends to rows 0 .. ctx_len[b] + gamma - 1 of the same sequence
