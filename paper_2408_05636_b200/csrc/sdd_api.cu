@@ -3,7 +3,9 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <new>
+#include <tuple>
 #include <type_traits>
 #include <vector>
 
@@ -159,6 +161,9 @@ struct sdd_ctx {
   size_t act_elems, xf_elems;  // capacity (elements) of the xn / att buffers (mlp: 4x) and of xf
   bool force_simt;             // SDD_GEMM=simt: run bf16 GEMMs on the CUDA-core kernel (cross-check)
   int bn_hint;                 // SDD_GEMM_BN: N tile of the tensor-core GEMM (0 = choose)
+  bool use_graph;              // SDD_GRAPH != 0: sdd_step replays a captured graph per row-count bucket
+  struct GraphEntry { cudaGraphExec_t exec; uint64_t launches; };
+  std::map<std::tuple<int, void*, void*>, GraphEntry> graphs;
   // optional per-launch timing
   bool profiling;
   std::vector<cudaEvent_t> prof_ev;   // pairs (before, after)
@@ -461,6 +466,8 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
     c->force_simt = g != nullptr && strcmp(g, "simt") == 0;
     const char* bn = getenv("SDD_GEMM_BN");
     c->bn_hint = bn ? atoi(bn) : 0;
+    const char* gr = getenv("SDD_GRAPH");
+    c->use_graph = gr == nullptr || atoi(gr) != 0;
   }
   c->prompt_len.assign(prompt_len, prompt_len + params->batch);
   c->c_ub = c->prompt_len;
@@ -476,6 +483,10 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
   memset(c->mirror, 0, mirror_ints * sizeof(int));
   SDD_CUDA(cudaHostGetDevicePointer((void**)&c->mirror_dev, c->mirror, 0));
 
+  if (c->P.dtype == SDD_BF16) {   // before anything can be captured into a graph
+    SDD_CUDA(tc_prepare_gemm());
+    SDD_CUDA(tc_prepare_attn());
+  }
   // zero the small state and the activations (padding rows must stay finite), then load the prompts
   const Buffers& B = c->B;
   const size_t state_bytes = (size_t)((uint8_t*)B.step_logits - (uint8_t*)workspace);
@@ -500,21 +511,43 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
   return SDD_OK;
 }
 
-int32_t sdd_draft_begin(sdd_ctx* c) {
-  if (c == nullptr) return SDD_E_ARG;
+// ---- round pieces: host bookkeeping outside, stream work inside (the latter can be captured in a graph) ----
+static int round_prologue(sdd_ctx* c) {
   // bound the host's run-ahead so that the length mirror stays fresh
   if (c->rounds >= (uint64_t)c->runahead)
     SDD_CUDA(cudaEventSynchronize(c->ev[(c->rounds - c->runahead) % c->ev.size()]));
   choose_lcap(c);
+  return SDD_OK;
+}
+static int enqueue_draft_begin(sdd_ctx* c) {
   SDD_LAUNCH(c, CAT_GLUE, launch_reset_slots(c->B.slot_ids, c->B.reveal_step, c->D.batch * c->D.gamma, c->D.V, c->st));
   c->steps_done = 0;
   return SDD_OK;
+}
+static int enqueue_draft_step(sdd_ctx* c) {
+  return c->P.dtype == SDD_BF16 ? draft_step_t<__nv_bfloat16>(c) : draft_step_t<float>(c);
+}
+static int enqueue_verify_accept(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
+  return c->P.dtype == SDD_BF16 ? verify_accept_t<__nv_bfloat16>(c, out_ids, n_out) : verify_accept_t<float>(c, out_ids, n_out);
+}
+static int round_epilogue(sdd_ctx* c) {
+  SDD_CUDA(cudaEventRecord(c->ev[c->rounds % c->ev.size()], c->st));
+  c->rounds++;
+  c->steps_done = -1;
+  for (auto& ub : c->c_ub) ub += c->D.gamma + 1;
+  return SDD_OK;
+}
+
+int32_t sdd_draft_begin(sdd_ctx* c) {
+  if (c == nullptr) return SDD_E_ARG;
+  SDD_TRY(round_prologue(c));
+  return enqueue_draft_begin(c);
 }
 
 int32_t sdd_draft_step(sdd_ctx* c) {
   if (c == nullptr) return SDD_E_ARG;
   if (c->steps_done < 0 || c->steps_done >= c->D.T) return SDD_E_STATE;
-  return c->P.dtype == SDD_BF16 ? draft_step_t<__nv_bfloat16>(c) : draft_step_t<float>(c);
+  return enqueue_draft_step(c);
 }
 
 int32_t sdd_draft(sdd_ctx* c) {
@@ -526,18 +559,46 @@ int32_t sdd_draft(sdd_ctx* c) {
 int32_t sdd_verify_accept(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
   if (c == nullptr) return SDD_E_ARG;
   if (c->steps_done != c->D.T) return SDD_E_STATE;
-  int s = c->P.dtype == SDD_BF16 ? verify_accept_t<__nv_bfloat16>(c, out_ids, n_out) : verify_accept_t<float>(c, out_ids, n_out);
-  if (s != SDD_OK) return s;
-  SDD_CUDA(cudaEventRecord(c->ev[c->rounds % c->ev.size()], c->st));
-  c->rounds++;
-  c->steps_done = -1;
-  for (auto& ub : c->c_ub) ub += c->D.gamma + 1;
-  return SDD_OK;
+  SDD_TRY(enqueue_verify_accept(c, out_ids, n_out));
+  return round_epilogue(c);
 }
 
+// One whole round.  Every launch parameter of a round is fixed for a given padded row count (all lengths,
+// the round index and the RNG state live on the device), so the round is captured once per row-count bucket
+// and replayed as a CUDA graph; SDD_GRAPH=0 (or per-launch timing) enqueues the kernels one by one instead.
 int32_t sdd_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
-  SDD_TRY(sdd_draft(c));
-  return sdd_verify_accept(c, out_ids, n_out);
+  if (c == nullptr) return SDD_E_ARG;
+  if (c->steps_done != -1) return SDD_E_STATE;
+  if (!c->use_graph || c->profiling) {
+    SDD_TRY(sdd_draft(c));
+    return sdd_verify_accept(c, out_ids, n_out);
+  }
+  SDD_TRY(round_prologue(c));
+  const auto key = std::make_tuple(c->lcap, (void*)out_ids, (void*)n_out);
+  auto it = c->graphs.find(key);
+  if (it == c->graphs.end()) {
+    const uint64_t l0 = c->launches;
+    SDD_CUDA(cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal));
+    int s = enqueue_draft_begin(c);
+    for (int i = 0; i < c->D.T && s == SDD_OK; ++i) s = enqueue_draft_step(c);
+    if (s == SDD_OK) s = enqueue_verify_accept(c, out_ids, n_out);
+    cudaGraph_t g = nullptr;
+    cudaError_t e = cudaStreamEndCapture(c->st, &g);
+    c->steps_done = -1;
+    if (s != SDD_OK) { if (g) cudaGraphDestroy(g); return s; }
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamEndCapture");
+    sdd_ctx::GraphEntry ge;
+    ge.exec = nullptr;
+    ge.launches = c->launches - l0;
+    c->launches = l0;
+    e = cudaGraphInstantiate(&ge.exec, g, 0);
+    cudaGraphDestroy(g);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGraphInstantiate");
+    it = c->graphs.emplace(key, ge).first;
+  }
+  SDD_CUDA(cudaGraphLaunch(it->second.exec, c->st));
+  c->launches += it->second.launches;
+  return round_epilogue(c);
 }
 
 int32_t sdd_progress(sdd_ctx* c, uint64_t* rounds_done, int32_t* min_emitted) {
@@ -679,6 +740,8 @@ void sdd_destroy(sdd_ctx* c) {
   if (c == nullptr) return;
   for (auto e : c->prof_ev)
     if (e) cudaEventDestroy(e);
+  for (auto& g : c->graphs)
+    if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
   for (auto e : c->ev)
     if (e) cudaEventDestroy(e);
   if (c->mirror) cudaFreeHost(c->mirror);

@@ -11,6 +11,8 @@
 // (row at position p sees cache positions 0..p).  V is consumed transposed, which the QKV GEMM's epilogue
 // produces for free; that keeps both MMAs on K-major operands.
 // Waits are bounded exactly as in the GEMM kernel.
+#include <mutex>
+
 #include "sdd_kernels.h"
 #include "sdd_tc.cuh"
 
@@ -238,6 +240,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
 }  // namespace tc
 
+cudaError_t tc_prepare_attn() {
+  return cudaFuncSetAttribute(tc::attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AT_SMEM);
+}
+
 cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q_ld, int q_col0, const __nv_bfloat16* k,
                            long long k_rows_total, int k_ld, int k_col0, int k_rows_per_seq, const __nv_bfloat16* vt,
                            int vt_ld, __nv_bfloat16* out, int ld_out, const int* ctx_len, int batch, int n_head, int d,
@@ -250,12 +256,10 @@ cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q
   if ((e = get_tensor_map(q, q_rows_total, q_ld, q_ld, 128, 64, &mq)) != cudaSuccess) return e;
   if ((e = get_tensor_map(k, k_rows_total, k_ld, k_ld, 128, 64, &mk)) != cudaSuccess) return e;
   if ((e = get_tensor_map(vt, (long long)batch * d, vt_ld, vt_ld, 64, 64, &mv)) != cudaSuccess) return e;
-  static bool attr_set = false;
-  if (!attr_set) {
-    e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::once_flag once;
+  static cudaError_t prep = cudaSuccess;
+  std::call_once(once, [] { prep = tc_prepare_attn(); });
+  if (prep != cudaSuccess) return prep;
   AttnParams p;
   p.out = out; p.ld_out = ld_out; p.ctx_len = ctx_len; p.mode = mode; p.gamma = gamma;
   p.q_rows_per_seq = q_rows_per_seq; p.k_rows_per_seq = k_rows_per_seq; p.q_col0 = q_col0; p.k_col0 = k_col0;

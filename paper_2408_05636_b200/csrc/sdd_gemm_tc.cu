@@ -237,18 +237,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 template <int BN, bool SWAP>
 static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, int rows_a, int rows_b, int K, int epi,
                               const float* bias, void* out, int ldc, int* status, cudaStream_t st, const QkvDst& qd) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<BN>());
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
   dim3 grid((rows_b + BN - 1) / BN, (rows_a + BM - 1) / BM);
   gemm_tc_kernel<BN, SWAP><<<grid, THREADS, smem_bytes<BN>(), st>>>(ma, mb, rows_a, rows_b, K, epi, bias, out, ldc, status, qd);
   return cudaGetLastError();
 }
 
+template <int BN, bool SWAP>
+static cudaError_t prepare_one() {
+  return cudaFuncSetAttribute(gemm_tc_kernel<BN, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<BN>());
+}
+
 }  // namespace tc
+
+// raise the dynamic shared-memory limit of every kernel variant (once per device, outside any stream capture)
+cudaError_t tc_prepare_gemm() {
+  using namespace tc;
+  cudaError_t e;
+  if ((e = prepare_one<32, false>()) != cudaSuccess) return e;
+  if ((e = prepare_one<64, false>()) != cudaSuccess) return e;
+  if ((e = prepare_one<128, false>()) != cudaSuccess) return e;
+  if ((e = prepare_one<256, false>()) != cudaSuccess) return e;
+  if ((e = prepare_one<32, true>()) != cudaSuccess) return e;
+  return prepare_one<64, true>();
+}
 
 static PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 static std::mutex g_map_mu;
@@ -289,6 +300,10 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
                            int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st, const QkvDst* qkv) {
   using namespace tc;
   if (M <= 0 || N <= 0) return cudaSuccess;
+  static std::once_flag once;
+  static cudaError_t prep = cudaSuccess;
+  std::call_once(once, [] { prep = tc_prepare_gemm(); });
+  if (prep != cudaSuccess) return prep;
   QkvDst qd = {};
   if (epi == EPI_QKV) {
     if (qkv == nullptr || (qkv->d & 63) != 0) return cudaErrorInvalidValue;

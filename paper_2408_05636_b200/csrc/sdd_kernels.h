@@ -85,6 +85,10 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
                            int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st,
                            const QkvDst* qkv = nullptr);
 
+// one-time set-up of the tensor-core kernels (dynamic shared-memory limits); also done lazily on first launch
+cudaError_t tc_prepare_gemm();
+cudaError_t tc_prepare_attn();
+
 // bf16 tensor-core attention, d_head = 64 (sdd_attn_tc.cu).  q / k are row-major tensors with the heads side by
 // side starting at column q_col0 / k_col0; vt is V transposed: [batch * d rows, vt_ld positions].
 // mode 0: drafter (no mask, ctx_len[b] + gamma rows and keys); 1: target verify; 2: target prefill.
