@@ -231,7 +231,9 @@ class Session:
         torch = _torch()
         self.torch = torch
         self.device = torch.device(device)
-        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        # a stream of its own by default: the library replays whole rounds as CUDA graphs, which the legacy
+        # default stream cannot capture.  Results are read after sdd_sync_status(), or on this stream.
+        self.stream = stream if stream is not None else torch.cuda.Stream(self.device)
         prompts = np.ascontiguousarray(prompts, dtype=np.int32)
         self.batch, self.prompt_stride = prompts.shape
         self.gamma, self.T, self.max_new, self.V = gamma, T, max_new, target.shape.vocab

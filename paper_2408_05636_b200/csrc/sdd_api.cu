@@ -467,7 +467,8 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
     const char* bn = getenv("SDD_GEMM_BN");
     c->bn_hint = bn ? atoi(bn) : 0;
     const char* gr = getenv("SDD_GRAPH");
-    c->use_graph = gr == nullptr || atoi(gr) != 0;
+    // the legacy default stream cannot be captured: rounds are then enqueued kernel by kernel
+    c->use_graph = (gr == nullptr || atoi(gr) != 0) && c->st != nullptr && c->st != cudaStreamLegacy;
   }
   c->prompt_len.assign(prompt_len, prompt_len + params->batch);
   c->c_ub = c->prompt_len;
