@@ -13,7 +13,15 @@
 
 namespace sdd {
 
-static thread_local char g_cuda_err[256] = "";
+static thread_local char g_cuda_err[512] = "";
+
+bool pdl_enabled() {
+  static const bool on = [] {
+    const char* e = getenv("SDD_PDL");
+    return e == nullptr || atoi(e) != 0;
+  }();
+  return on;
+}
 
 static int cuda_fail(cudaError_t e, const char* what) {
   snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));

@@ -55,6 +55,7 @@ template <typename T, int DH>
 __global__ void __launch_bounds__(128)
 attn_bidir_kernel(const T* __restrict__ qkv, T* __restrict__ out, const int* __restrict__ ctx_len, int gamma, int L_cap,
                   int n_head) {
+  pdl_wait();
   const int i = blockIdx.x * 4 + (threadIdx.x >> 5), h = blockIdx.y, b = blockIdx.z;
   if (i >= L_cap) return;
   const int d = n_head * DH;
@@ -73,6 +74,7 @@ template <typename T, int DH>
 __global__ void __launch_bounds__(128)
 attn_cached_kernel(const T* __restrict__ qkv, const T* __restrict__ cache, T* __restrict__ out,
                    const int* __restrict__ ctx_len, int rows_per_seq, int mode, int n_ctx, int n_head) {
+  pdl_wait();
   const int j = blockIdx.x * 4 + (threadIdx.x >> 5), h = blockIdx.y, b = blockIdx.z;
   if (j >= rows_per_seq) return;
   const int d = n_head * DH;
@@ -95,8 +97,8 @@ template <typename T>
 cudaError_t launch_attn_bidir(const T* qkv, T* out, const int* ctx_len, int batch, int gamma, int L_cap, int n_head,
                               int d_head, cudaStream_t st) {
   dim3 grid((L_cap + 3) / 4, n_head, batch);
-  if (d_head == 64) attn_bidir_kernel<T, 64><<<grid, 128, 0, st>>>(qkv, out, ctx_len, gamma, L_cap, n_head);
-  else if (d_head == 32) attn_bidir_kernel<T, 32><<<grid, 128, 0, st>>>(qkv, out, ctx_len, gamma, L_cap, n_head);
+  if (d_head == 64) launch_k(attn_bidir_kernel<T, 64>, dim3(grid), dim3(128), 0, st, qkv, out, ctx_len, gamma, L_cap, n_head);
+  else if (d_head == 32) launch_k(attn_bidir_kernel<T, 32>, dim3(grid), dim3(128), 0, st, qkv, out, ctx_len, gamma, L_cap, n_head);
   else return cudaErrorInvalidValue;
   return cudaGetLastError();
 }
@@ -107,9 +109,9 @@ cudaError_t launch_attn_cached(const T* qkv, const T* cache, T* out, const int* 
   if (rows_per_seq <= 0) return cudaSuccess;
   dim3 grid((rows_per_seq + 3) / 4, n_head, batch);
   if (d_head == 64)
-    attn_cached_kernel<T, 64><<<grid, 128, 0, st>>>(qkv, cache, out, ctx_len, rows_per_seq, mode, n_ctx, n_head);
+    launch_k(attn_cached_kernel<T, 64>, dim3(grid), dim3(128), 0, st, qkv, cache, out, ctx_len, rows_per_seq, mode, n_ctx, n_head);
   else if (d_head == 32)
-    attn_cached_kernel<T, 32><<<grid, 128, 0, st>>>(qkv, cache, out, ctx_len, rows_per_seq, mode, n_ctx, n_head);
+    launch_k(attn_cached_kernel<T, 32>, dim3(grid), dim3(128), 0, st, qkv, cache, out, ctx_len, rows_per_seq, mode, n_ctx, n_head);
   else return cudaErrorInvalidValue;
   return cudaGetLastError();
 }

@@ -48,6 +48,7 @@ __global__ void __launch_bounds__(AT_THREADS)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_vt, const AttnParams prm) {
   const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  pdl_wait();   // ctx_len and Q / K / V^T come from earlier kernels
   const int c = prm.ctx_len[b];
   const int q0 = qt * 128;
   int n_valid_q;
@@ -265,7 +266,7 @@ cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q
   p.q_rows_per_seq = q_rows_per_seq; p.k_rows_per_seq = k_rows_per_seq; p.q_col0 = q_col0; p.k_col0 = k_col0;
   p.d = d; p.status = status;
   dim3 grid((q_rows_per_seq + 127) / 128, n_head, batch);
-  attn_tc_kernel<<<grid, AT_THREADS, AT_SMEM, st>>>(mq, mk, mv, p);
+  launch_k(attn_tc_kernel, dim3(grid), dim3(AT_THREADS), AT_SMEM, st, mq, mk, mv, p);
   return cudaGetLastError();
 }
 

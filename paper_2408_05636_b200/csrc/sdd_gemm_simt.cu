@@ -11,6 +11,7 @@ template <typename T>
 __global__ void __launch_bounds__(SG_THREADS)
 gemm_simt_kernel(const T* __restrict__ A, int lda, const T* __restrict__ W, const float* __restrict__ bias, int M, int N,
                  int K, int epi, void* __restrict__ out, int ldc) {
+  pdl_wait();
   __shared__ float As[SG_BK][SG_BM + 4];
   __shared__ float Ws[SG_BK][SG_BN + 4];
   const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
@@ -61,7 +62,7 @@ cudaError_t launch_gemm_simt(const T* A, int lda, const T* W, const float* bias,
                              int ldc, cudaStream_t st) {
   if (M <= 0 || N <= 0) return cudaSuccess;
   dim3 grid((N + SG_BN - 1) / SG_BN, (M + SG_BM - 1) / SG_BM);
-  gemm_simt_kernel<T><<<grid, SG_THREADS, 0, st>>>(A, lda, W, bias, M, N, K, epi, out, ldc);
+  launch_k(gemm_simt_kernel<T>, dim3(grid), dim3(SG_THREADS), 0, st, A, lda, W, bias, M, N, K, epi, out, ldc);
   return cudaGetLastError();
 }
 

@@ -29,19 +29,25 @@ namespace tc {
 constexpr int BM = 128;          // MMA M
 constexpr int BK = 64;           // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int STAGES = 4;
 constexpr int THREADS = 192;     // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
 
 template <int BN>
 constexpr int stage_bytes() { return BM * BK * 2 + BN * BK * 2; }
+// shared-memory ring depth per N tile: as deep as one CTA per SM allows (about 190 KB), so that a short K loop
+// has all of its tiles in flight at once
 template <int BN>
-constexpr int smem_bytes() { return STAGES * stage_bytes<BN>() + 1024 /*alignment slack*/ + 256 /*barriers*/; }
+constexpr int ring_stages() { return BN <= 64 ? 8 : (BN == 128 ? 6 : 4); }
+template <int BN>
+constexpr int smem_bytes() { return ring_stages<BN>() * stage_bytes<BN>() + 1024 /*alignment slack*/ + 256 /*barriers*/; }
 
+// grid = (N tiles, M tiles, K splits).  With more than one K split every CTA accumulates its share of the K
+// range and adds it to the fp32 output with atomics (EPI_RESIDUAL only; the bias is added by split 0).
 template <int BN, bool SWAP>
 __global__ void __launch_bounds__(THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int rows_a,
                int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out, int ldc, int* status,
                const QkvDst qd) {
+  constexpr int STAGES = ring_stages<BN>();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bar_base = base + STAGES * stage_bytes<BN>();
@@ -56,7 +62,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.y * BM;      // offset along the A operand's rows (MMA M axis)
   const int n0 = blockIdx.x * BN;      // offset along the B operand's rows (MMA N axis)
-  const int num_kb = (K + BK - 1) / BK;
+  const int total_kb = (K + BK - 1) / BK;
+  const int kb_per = (total_kb + (int)gridDim.z - 1) / (int)gridDim.z;
+  const int kb0 = (int)blockIdx.z * kb_per;
+  const int num_kb = min(kb_per, total_kb - kb0);     // host guarantees >= 1
+  const bool split = gridDim.z > 1;
+  if (split && blockIdx.z != 0) bias = nullptr;
   constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
 
   if (threadIdx.x == 0) {
@@ -72,6 +83,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  // everything above touched only shared / tensor memory; global inputs may still be in production
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -82,8 +96,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, status)) break;
         mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes<BN>());
         const uint32_t sa = base + s * stage_bytes<BN>();
-        tma_load_2d(sa, &map_a, full_bar(s), kb * BK, m0);
-        tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), kb * BK, n0);
+        tma_load_2d(sa, &map_a, full_bar(s), (kb0 + kb) * BK, m0);
+        tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), (kb0 + kb) * BK, n0);
         issued = kb + 1;
       }
       if (*abort_flag) {
@@ -180,10 +194,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               }
             } else {
               float* o = reinterpret_cast<float*>(out) + (long long)r * ldc + c0;
-              for (int j = 0; j < 32; ++j) {
-                if (c0 + j < rows_b) {
-                  const float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
-                  if (epi == EPI_RESIDUAL) o[j] += x; else o[j] = x;
+              if (epi == EPI_RESIDUAL && !split && c0 + 32 <= rows_b && (ldc & 3) == 0) {
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                  float4 h4 = *reinterpret_cast<float4*>(o + g * 4);
+                  h4.x += __uint_as_float(v[g * 4 + 0]) + (bias ? bias[c0 + g * 4 + 0] : 0.f);
+                  h4.y += __uint_as_float(v[g * 4 + 1]) + (bias ? bias[c0 + g * 4 + 1] : 0.f);
+                  h4.z += __uint_as_float(v[g * 4 + 2]) + (bias ? bias[c0 + g * 4 + 2] : 0.f);
+                  h4.w += __uint_as_float(v[g * 4 + 3]) + (bias ? bias[c0 + g * 4 + 3] : 0.f);
+                  *reinterpret_cast<float4*>(o + g * 4) = h4;
+                }
+              } else {
+                for (int j = 0; j < 32; ++j) {
+                  if (c0 + j < rows_b) {
+                    const float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
+                    if (epi == EPI_RESIDUAL) { if (split) atomicAdd(o + j, x); else o[j] += x; }
+                    else o[j] = x;
+                  }
                 }
               }
             }
@@ -215,7 +242,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
               } else if (epi == EPI_STORE) reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(x);
               else if (epi == EPI_GELU) reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(gelu_tanh(x));
-              else if (epi == EPI_RESIDUAL) reinterpret_cast<float*>(out)[o] += x;
+              else if (epi == EPI_RESIDUAL) { if (split) atomicAdd(reinterpret_cast<float*>(out) + o, x); else reinterpret_cast<float*>(out)[o] += x; }
               else reinterpret_cast<float*>(out)[o] = x;
             }
           }
@@ -236,9 +263,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 template <int BN, bool SWAP>
 static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, int rows_a, int rows_b, int K, int epi,
-                              const float* bias, void* out, int ldc, int* status, cudaStream_t st, const QkvDst& qd) {
-  dim3 grid((rows_b + BN - 1) / BN, (rows_a + BM - 1) / BM);
-  gemm_tc_kernel<BN, SWAP><<<grid, THREADS, smem_bytes<BN>(), st>>>(ma, mb, rows_a, rows_b, K, epi, bias, out, ldc, status, qd);
+                              const float* bias, void* out, int ldc, int* status, cudaStream_t st, const QkvDst& qd,
+                              int splits) {
+  dim3 grid((rows_b + BN - 1) / BN, (rows_a + BM - 1) / BM, splits);
+  launch_k(gemm_tc_kernel<BN, SWAP>, dim3(grid), dim3(THREADS), smem_bytes<BN>(), st, ma, mb, rows_a, rows_b, K, epi, bias, out, ldc, status, qd);
   return cudaGetLastError();
 }
 
@@ -311,29 +339,44 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
   }
   CUtensorMap ma, mb;
   cudaError_t e;
+  const int total_kb = (K + BK - 1) / BK;
+  constexpr int SMS = 148;
+  // K splits fill idle SMs of a single-wave grid; only the residual epilogue can add partial sums
+  auto pick_splits = [&](long long ctas, int min_kb) {
+    if (epi != EPI_RESIDUAL || ctas >= SMS) return 1;
+    long long s = SMS / ctas;
+    if (s > total_kb / min_kb) s = total_kb / min_kb;
+    if (s < 1) s = 1;
+    // no empty split: ceil(total_kb / s) * (s - 1) < total_kb
+    while (s > 1 && ((total_kb + s - 1) / s) * (s - 1) >= total_kb) --s;
+    return (int)s;
+  };
   if (M <= 64) {
     // SWAP: A operand = weights (box 128 rows), B operand = tokens (box BN rows)
     const int bn = M <= 32 ? 32 : 64;
+    const int splits = pick_splits((N + BM - 1) / BM, 2);
     if ((e = get_tensor_map(W, N, K, K, BM, BK, &ma)) != cudaSuccess) return e;
     if ((e = get_tensor_map(A, a_cap, K, K, bn, BK, &mb)) != cudaSuccess) return e;
-    if (bn == 32) return launch_cfg<32, true>(ma, mb, N, M, K, epi, bias, out, ldc, status, st, qd);
-    return launch_cfg<64, true>(ma, mb, N, M, K, epi, bias, out, ldc, status, st, qd);
+    if (bn == 32) return launch_cfg<32, true>(ma, mb, N, M, K, epi, bias, out, ldc, status, st, qd, splits);
+    return launch_cfg<64, true>(ma, mb, N, M, K, epi, bias, out, ldc, status, st, qd, splits);
   }
   int bn = bn_hint;
+  const long long mt = (M + BM - 1) / BM;
   if (bn != 32 && bn != 64 && bn != 128 && bn != 256) {
-    const long long mt = (M + BM - 1) / BM;
-    bn = 32;
-    for (int cand : {256, 128, 64}) {
-      if (mt * ((N + cand - 1) / cand) >= 120) { bn = cand; break; }
+    // the narrowest N tile whose grid still fits one wave (most CTAs without a second wave); 256 beyond that
+    bn = 256;
+    for (int cand : {32, 64, 128}) {
+      if (mt * ((N + cand - 1) / cand) <= SMS) { bn = cand; break; }
     }
   }
+  const int splits = pick_splits(mt * ((N + bn - 1) / bn), 4);
   if ((e = get_tensor_map(A, a_cap, K, K, BM, BK, &ma)) != cudaSuccess) return e;
   if ((e = get_tensor_map(W, N, K, K, bn, BK, &mb)) != cudaSuccess) return e;
   switch (bn) {
-    case 256: return launch_cfg<256, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd);
-    case 128: return launch_cfg<128, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd);
-    case 64: return launch_cfg<64, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd);
-    default: return launch_cfg<32, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd);
+    case 256: return launch_cfg<256, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
+    case 128: return launch_cfg<128, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
+    case 64: return launch_cfg<64, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
+    default: return launch_cfg<32, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
   }
 }
 

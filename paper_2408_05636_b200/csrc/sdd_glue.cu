@@ -12,6 +12,7 @@ template <typename T>
 __global__ void embed_drafter_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
                                      int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
                                      int gamma, int L_cap, int d, float* __restrict__ h) {
+  pdl_wait();
   const int i = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
   float* __restrict__ dst = h + ((long long)b * L_cap + i) * d;
@@ -31,6 +32,7 @@ template <typename T>
 __global__ void embed_target_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
                                     int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
                                     int gamma, int rows_per_seq, int mode, int d, float* __restrict__ h) {
+  pdl_wait();
   const int j = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
   float* __restrict__ dst = h + ((long long)b * rows_per_seq + j) * d;
@@ -89,6 +91,7 @@ template <typename T>
 __global__ void __launch_bounds__(128)
 layernorm_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
                  T* __restrict__ out, long long rows, int d) {
+  pdl_wait();
   const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
   if (row >= rows) return;
   layernorm_row<T>(h + row * d, g, bta, out + row * d, d);
@@ -98,6 +101,7 @@ template <typename T>
 __global__ void __launch_bounds__(128)
 layernorm_slots_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
                        T* __restrict__ out, const int* __restrict__ ctx_len, int batch, int gamma, int L_cap, int d) {
+  pdl_wait();
   const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
   if (r >= batch * gamma) return;
   const int b = r / gamma, j = r - b * gamma;
@@ -110,6 +114,7 @@ layernorm_slots_kernel(const float* __restrict__ h, const float* __restrict__ g,
 template <typename T>
 __global__ void kv_append_kernel(const T* __restrict__ qkv, T* __restrict__ cache, const int* __restrict__ ctx_len,
                                  int rows_per_seq, int mode, int n_ctx, int d) {
+  pdl_wait();
   const int j = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
   int pos;
@@ -127,7 +132,7 @@ __global__ void kv_append_kernel(const T* __restrict__ qkv, T* __restrict__ cach
 template <typename T>
 cudaError_t launch_embed_drafter(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                  const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st) {
-  embed_drafter_kernel<T><<<dim3(L_cap, batch), 128, 0, st>>>(wte, wpe, tokens, tok_stride, ctx_len, slot_ids, gamma,
+  launch_k(embed_drafter_kernel<T>, dim3(dim3(L_cap, batch)), dim3(128), 0, st, wte, wpe, tokens, tok_stride, ctx_len, slot_ids, gamma,
                                                               L_cap, d, h);
   return cudaGetLastError();
 }
@@ -136,7 +141,7 @@ cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, i
                                 const int* slot_ids, int batch, int gamma, int rows_per_seq, int mode, int d, float* h,
                                 cudaStream_t st) {
   if (rows_per_seq <= 0) return cudaSuccess;
-  embed_target_kernel<T><<<dim3(rows_per_seq, batch), 128, 0, st>>>(wte, wpe, tokens, tok_stride, ctx_len, slot_ids, gamma,
+  launch_k(embed_target_kernel<T>, dim3(dim3(rows_per_seq, batch)), dim3(128), 0, st, wte, wpe, tokens, tok_stride, ctx_len, slot_ids, gamma,
                                                                     rows_per_seq, mode, d, h);
   return cudaGetLastError();
 }
@@ -145,21 +150,21 @@ cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* 
                              cudaStream_t st) {
   if (rows <= 0) return cudaSuccess;
   if (d > LN_MAX_PER_LANE * 32) return cudaErrorInvalidValue;
-  layernorm_kernel<T><<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(h, g, b, out, rows, d);
+  launch_k(layernorm_kernel<T>, dim3((unsigned)((rows + 3) / 4)), dim3(128), 0, st, h, g, b, out, rows, d);
   return cudaGetLastError();
 }
 template <typename T>
 cudaError_t launch_layernorm_slots(const float* h, const float* g, const float* b, T* out, const int* ctx_len, int batch,
                                    int gamma, int L_cap, int d, cudaStream_t st) {
   if (d > LN_MAX_PER_LANE * 32) return cudaErrorInvalidValue;
-  layernorm_slots_kernel<T><<<(batch * gamma + 3) / 4, 128, 0, st>>>(h, g, b, out, ctx_len, batch, gamma, L_cap, d);
+  launch_k(layernorm_slots_kernel<T>, dim3((batch * gamma + 3) / 4), dim3(128), 0, st, h, g, b, out, ctx_len, batch, gamma, L_cap, d);
   return cudaGetLastError();
 }
 template <typename T>
 cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int batch, int rows_per_seq, int mode, int n_ctx,
                              int d, cudaStream_t st) {
   if (rows_per_seq <= 0) return cudaSuccess;
-  kv_append_kernel<T><<<dim3(rows_per_seq, batch), 128, 0, st>>>(qkv, cache, ctx_len, rows_per_seq, mode, n_ctx, d);
+  launch_k(kv_append_kernel<T>, dim3(dim3(rows_per_seq, batch)), dim3(128), 0, st, qkv, cache, ctx_len, rows_per_seq, mode, n_ctx, d);
   return cudaGetLastError();
 }
 

@@ -3,6 +3,8 @@
 //   unmask_sample_kernel  one denoising step's reveal test + Gumbel-max draw + stored q row
 //   accept_kernel         u <= min(1, p/q) scan, residual norm(max(0, p - q)) or bonus draw
 //   commit_kernel         append the emitted tokens to each sequence
+#include <cooperative_groups.h>
+
 #include "sdd_kernels.h"
 
 namespace sdd {
@@ -28,6 +30,7 @@ template <bool GREEDY>
 __global__ void __launch_bounds__(STATS_THREADS)
 row_stats_kernel(const float* __restrict__ buf_a, long long rows_a, const float* __restrict__ buf_b, long long rows_b,
                  int V, int chunks, float inv_tau_a, float inv_tau_b, float2* __restrict__ partial) {
+  pdl_wait();
   const long long row = blockIdx.x / chunks;
   const int chunk = blockIdx.x - (int)(row * chunks);
   const bool is_a = row < rows_a;
@@ -182,20 +185,82 @@ __device__ __forceinline__ void maxsum_push(MaxSum& ms, float z) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// denoising step k: reveal test, Gumbel-max draw, stored q row            grid = (gamma, batch)
+// The two vocabulary-wide draws below give one logit row to a thread-block cluster of VC CTAs: each
+// CTA scans an interleaved 1/VC of the row, reduces inside the block, publishes its partial result
+// in its own shared memory, and after a cluster barrier the partials are merged through distributed
+// shared memory.  A single CTA per row would leave the row's latency chain (Philox, two logs, the
+// scan over 50 k entries) on one SM.
+// ---------------------------------------------------------------------------------------------
+namespace cg = cooperative_groups;
+constexpr int VC = 8;
+
+struct RowPartial {
+  float arg_s; int arg_i;      // Gumbel arg-max of this CTA's share
+  float fb_s; int fb_i;        // fall-back arg-max (draw from p itself)
+  float m, s;                  // online soft-max pair of this CTA's share
+};
+
+__device__ __forceinline__ ArgMax cluster_merge_argmax(cg::cluster_group& cl, RowPartial* mine, bool fallback) {
+  ArgMax a;
+  a.s = -INFINITY;
+  a.i = 0x7fffffff;
+  for (int r = 0; r < VC; ++r) {
+    const RowPartial* o = cl.map_shared_rank(mine, r);
+    ArgMax b;
+    b.s = fallback ? o->fb_s : o->arg_s;
+    b.i = fallback ? o->fb_i : o->arg_i;
+    a = argmax_better(a, b);
+  }
+  return a;
+}
+__device__ __forceinline__ float cluster_merge_lse(cg::cluster_group& cl, RowPartial* mine) {
+  MaxSum t;
+  t.m = -INFINITY;
+  t.s = 0.f;
+  for (int r = 0; r < VC; ++r) {
+    const RowPartial* o = cl.map_shared_rank(mine, r);
+    MaxSum b;
+    b.m = o->m; b.s = o->s;
+    t = maxsum_merge(t, b);
+  }
+  return t.m + logf(t.s);
+}
+
+// block-wide online soft-max pair; result valid in thread 0
+template <int THREADS>
+__device__ __forceinline__ MaxSum block_maxsum(MaxSum ms, float* s_m, float* s_s) {
+  ms = warp_maxsum(ms);
+  if ((threadIdx.x & 31) == 0) { s_m[threadIdx.x >> 5] = ms.m; s_s[threadIdx.x >> 5] = ms.s; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < THREADS / 32; ++w) {
+      MaxSum o;
+      o.m = s_m[w]; o.s = s_s[w];
+      ms = maxsum_merge(ms, o);
+    }
+  }
+  return ms;
+}
+
+// ---------------------------------------------------------------------------------------------
+// denoising step k: reveal test, Gumbel-max draw, stored q row     grid = (VC * gamma, batch), cluster VC
 // ---------------------------------------------------------------------------------------------
 constexpr int SAMPLE_THREADS = 512;
 
-__global__ void __launch_bounds__(SAMPLE_THREADS)
+__global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(SAMPLE_THREADS)
 unmask_sample_kernel(const float* __restrict__ step_logits,  // [B, gamma, V]
                      int* __restrict__ slot_ids,             // [B, gamma]  (V = masked)
                      float* __restrict__ q_logits,           // [B, gamma, V]
                      float* __restrict__ logq,               // [B, gamma]
                      int* __restrict__ reveal_step,          // [B, gamma]
                      int gamma, int V, int k, float inv_tau_q, PhiloxKey key, const RoundState* __restrict__ rs) {
-  const int j = blockIdx.x, b = blockIdx.y;
+  pdl_wait();
+  cg::cluster_group cl = cg::this_cluster();
+  const int rank = (int)cl.block_rank();
+  const int j = blockIdx.x / VC, b = blockIdx.y;
   const uint32_t rnd = rs->round;
   const long long row = (long long)b * gamma + j;
+  // every CTA of the cluster takes the same decision from the same inputs, before anyone writes the slot
   if (slot_ids[row] != V) return;  // already revealed: carried over unchanged
   // reveal with probability 1/k: u = m * 2^-24 with m odd, so u < 1/k  <=>  m * k < 2^24 (exact, k <= 255)
   const uint32_t wu = philox4x32_10(0u, (uint32_t)j, rnd, rng_c3(RNG_UNMASK, (uint32_t)k, (uint32_t)b), key).x;
@@ -214,7 +279,7 @@ unmask_sample_kernel(const float* __restrict__ step_logits,  // [B, gamma, V]
   best.s = -INFINITY;
   best.i = 0x7fffffff;
   const int nblk = (V + 3) >> 2;
-  for (int blk = threadIdx.x; blk < nblk; blk += SAMPLE_THREADS) {
+  for (int blk = rank * SAMPLE_THREADS + threadIdx.x; blk < nblk; blk += VC * SAMPLE_THREADS) {
     uint4 w = make_uint4(0, 0, 0, 0);
     if (!greedy) w = philox4x32_10((uint32_t)blk, (uint32_t)j, rnd, c3, key);
     const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
@@ -236,33 +301,43 @@ unmask_sample_kernel(const float* __restrict__ step_logits,  // [B, gamma, V]
   __shared__ float s_val[SAMPLE_THREADS / 32];
   __shared__ int s_idx[SAMPLE_THREADS / 32];
   __shared__ float s_m[SAMPLE_THREADS / 32], s_s[SAMPLE_THREADS / 32];
-  __shared__ float s_lse;
+  __shared__ RowPartial part;
   best = block_argmax<SAMPLE_THREADS>(best, s_val, s_idx);
-  const float lse = block_lse<SAMPLE_THREADS>(ms, s_m, s_s, &s_lse);
+  ms = block_maxsum<SAMPLE_THREADS>(ms, s_m, s_s);
   if (threadIdx.x == 0) {
-    slot_ids[row] = best.i;
-    logq[row] = greedy ? 0.f : src[best.i] * inv_tau_q - lse;
+    part.arg_s = best.s; part.arg_i = best.i; part.m = ms.m; part.s = ms.s;
+  }
+  cl.sync();
+  if (rank == 0 && threadIdx.x == 0) {
+    const ArgMax win = cluster_merge_argmax(cl, &part, false);
+    const float lse = greedy ? 0.f : cluster_merge_lse(cl, &part);
+    slot_ids[row] = win.i;
+    logq[row] = greedy ? 0.f : src[win.i] * inv_tau_q - lse;
     reveal_step[row] = k;
   }
+  cl.sync();   // partials stay alive until rank 0 has read them
 }
 
 // ---------------------------------------------------------------------------------------------
-// acceptance scan + extra token                                               grid = (rows)
+// acceptance scan + extra token                                  grid = (VC * rows), cluster VC per row
 //
 // logits_p [rows, gamma+1, V]; q rows [rows, gamma, V] hold z_q = l * inv_tau_q_rows (inv_tau_q_rows
 // = 1 when the rows were stored already divided by the temperature).  log q(x) comes either from
 // `logq_in` (round pipeline) or from the q-row partial statistics (stand-alone call).
 // ---------------------------------------------------------------------------------------------
-constexpr int ACCEPT_THREADS = 1024;
+constexpr int ACCEPT_THREADS = 512;
 
-__global__ void __launch_bounds__(ACCEPT_THREADS)
+__global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(ACCEPT_THREADS)
 accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_rows, const int* __restrict__ draft_ids,
               const float* __restrict__ logq_in, const float2* __restrict__ partial_p,
               const float2* __restrict__ partial_q, int chunks, int gamma, int V, float inv_tau_p,
               float inv_tau_q_rows, PhiloxKey key, uint32_t rnd_arg, const RoundState* __restrict__ rs,
               float* __restrict__ accept_prob, int* __restrict__ n_accept, int* __restrict__ extra_token,
               int* __restrict__ out_ids) {
-  const int b = blockIdx.x;
+  pdl_wait();
+  cg::cluster_group cl = cg::this_cluster();
+  const int rank = (int)cl.block_rank();
+  const int b = blockIdx.x / VC;
   const uint32_t rnd = rs != nullptr ? rs->round : rnd_arg;
   const bool greedy = inv_tau_p == 0.f;
   extern __shared__ float s_dyn[];           // [gamma+1] lse_p (or arg-max bits), [gamma] lse_q
@@ -274,6 +349,7 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
   __shared__ int s_idx[ACCEPT_THREADS / 32];
   __shared__ float s_m2[ACCEPT_THREADS / 32], s_s2[ACCEPT_THREADS / 32];
   __shared__ float s_lse2;
+  __shared__ RowPartial part;
 
   const float2* pp = partial_p + (long long)b * (gamma + 1) * chunks;
   for (int j = threadIdx.x; j <= gamma; j += ACCEPT_THREADS) {
@@ -286,7 +362,7 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
   }
   __syncthreads();
 
-  // first rejected position (the host guarantees gamma <= ACCEPT_THREADS)
+  // first rejected position, computed identically by every CTA of the cluster (gamma <= ACCEPT_THREADS)
   int rej = gamma;
   if ((int)threadIdx.x < gamma) {
     const int j = threadIdx.x;
@@ -301,7 +377,7 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
       ratio = expf(fminf(0.f, logp - lq));
     }
     const float u = scalar_uniform(key, RNG_ACCEPT, rnd, 0u, (uint32_t)j, (uint32_t)b);
-    accept_prob[(long long)b * gamma + j] = ratio;
+    if (rank == 0) accept_prob[(long long)b * gamma + j] = ratio;
     if (!(u <= ratio)) rej = j;
   }
 #pragma unroll
@@ -318,32 +394,35 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
 
   // extra token: residual of row n (n < gamma) or the bonus draw from row gamma
   const float* __restrict__ prow = logits_p + ((long long)b * (gamma + 1) + n) * V;
-  ArgMax best;
+  const bool resid = n < gamma;
+  ArgMax best, fallback;
   best.s = -INFINITY;
   best.i = 0x7fffffff;
-  if (greedy) {
-    best.s = 0.f;
-    best.i = __float_as_int(s_lsep[n]);   // arg-max of the target row, in both branches
-  } else {
-    const bool resid = n < gamma;
+  fallback = best;
+  if (!greedy) {
     const float* __restrict__ qrow = q_rows + ((long long)b * gamma + (resid ? n : 0)) * V;
     const float lsep = s_lsep[n];
     float lseq = 0.f;
     if (resid) {
       if (partial_q != nullptr) lseq = s_lseq[n];
       else {
-        // round pipeline: q row statistics are not kept; recompute the row's log-sum-exp here
+        // round pipeline: q row statistics are not kept; the cluster recomputes the row's log-sum-exp
         MaxSum ms;
         ms.m = -INFINITY;
         ms.s = 0.f;
-        for (int v = threadIdx.x; v < V; v += ACCEPT_THREADS) maxsum_push(ms, qrow[v] * inv_tau_q_rows);
-        lseq = block_lse<ACCEPT_THREADS>(ms, s_m2, s_s2, &s_lse2);
+        for (int v = rank * ACCEPT_THREADS + threadIdx.x; v < V; v += VC * ACCEPT_THREADS)
+          maxsum_push(ms, qrow[v] * inv_tau_q_rows);
+        ms = block_maxsum<ACCEPT_THREADS>(ms, s_m2, s_s2);
+        if (threadIdx.x == 0) { part.m = ms.m; part.s = ms.s; }
+        cl.sync();
+        if (threadIdx.x == 0) s_lse2 = cluster_merge_lse(cl, &part);
+        __syncthreads();
+        lseq = s_lse2;
       }
     }
     const uint32_t c3 = rng_c3(resid ? RNG_RESID : RNG_BONUS, 0u, (uint32_t)b);
     const int nblk = (V + 3) >> 2;
-    ArgMax fallback = best;   // a draw from p itself, used only if max(0, p - q) is identically zero
-    for (int blk = threadIdx.x; blk < nblk; blk += ACCEPT_THREADS) {
+    for (int blk = rank * ACCEPT_THREADS + threadIdx.x; blk < nblk; blk += VC * ACCEPT_THREADS) {
       const uint4 w = philox4x32_10((uint32_t)blk, (uint32_t)n, rnd, c3, key);
       const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
@@ -356,7 +435,7 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
           cand.i = v;
           cand.s = zp + g;
           if (resid) {
-            fallback = argmax_better(fallback, cand);
+            fallback = argmax_better(fallback, cand);    // a draw from p itself, if max(0, p - q) == 0 everywhere
             const float zq = qrow[v] * inv_tau_q_rows - lseq;
             const float wv = expf(zp) - expf(zq);
             if (wv > 0.f) {
@@ -370,20 +449,30 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
       }
     }
     best = block_argmax<ACCEPT_THREADS>(best, s_val, s_idx);
-    if (resid) {
-      __syncthreads();
-      fallback = block_argmax<ACCEPT_THREADS>(fallback, s_val, s_idx);
-      if (threadIdx.x == 0 && best.i == 0x7fffffff) best = fallback;
-    }
+    __syncthreads();
+    fallback = block_argmax<ACCEPT_THREADS>(fallback, s_val, s_idx);
   }
   if (threadIdx.x == 0) {
+    part.arg_s = best.s; part.arg_i = best.i; part.fb_s = fallback.s; part.fb_i = fallback.i;
+  }
+  cl.sync();
+  if (rank == 0 && threadIdx.x == 0) {
+    int t;
+    if (greedy) {
+      t = __float_as_int(s_lsep[n]);   // arg-max of the target row, in both branches
+    } else {
+      ArgMax win = cluster_merge_argmax(cl, &part, false);
+      if (win.i == 0x7fffffff) win = cluster_merge_argmax(cl, &part, true);
+      t = win.i;
+    }
     n_accept[b] = n;
-    if (extra_token != nullptr) extra_token[b] = best.i;
+    if (extra_token != nullptr) extra_token[b] = t;
     if (out_ids != nullptr) {
       for (int j = 0; j <= gamma; ++j)
-        out_ids[(long long)b * (gamma + 1) + j] = j < n ? draft_ids[(long long)b * gamma + j] : (j == n ? best.i : -1);
+        out_ids[(long long)b * (gamma + 1) + j] = j < n ? draft_ids[(long long)b * gamma + j] : (j == n ? t : -1);
     }
   }
+  cl.sync();   // partials stay alive until rank 0 has read them
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -395,6 +484,7 @@ __global__ void commit_kernel(int* __restrict__ tokens, int tok_stride, int* __r
                               const int* __restrict__ n_accept, const int* __restrict__ extra_token, int batch, int gamma,
                               int max_new, RoundState* rs, int* __restrict__ out_ids, int* __restrict__ n_out,
                               volatile int* host_mirror) {
+  pdl_wait();
   const uint32_t stamp = rs->round + 1u;
   if (host_mirror != nullptr && threadIdx.x == 0) {
     host_mirror[0] = (int)stamp;
@@ -438,6 +528,7 @@ __global__ void commit_kernel(int* __restrict__ tokens, int tok_stride, int* __r
 }
 
 __global__ void reset_slots_kernel(int* __restrict__ slot_ids, int* __restrict__ reveal_step, int n, int mask_id) {
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) {
     slot_ids[i] = mask_id;
@@ -458,17 +549,17 @@ cudaError_t launch_row_stats(const float* a, long long rows_a, const float* b, l
   if (rows * chunks > 0x7fffffffll) return cudaErrorInvalidValue;
   const unsigned grid = (unsigned)(rows * chunks);
   if (inv_tau_a == 0.f)
-    row_stats_kernel<true><<<grid, STATS_THREADS, 0, st>>>(a, rows_a, b, rows_b, V, chunks, inv_tau_a, inv_tau_b, partial);
+    launch_k(row_stats_kernel<true>, dim3(grid), dim3(STATS_THREADS), 0, st, a, rows_a, b, rows_b, V, chunks, inv_tau_a, inv_tau_b, partial);
   else
-    row_stats_kernel<false><<<grid, STATS_THREADS, 0, st>>>(a, rows_a, b, rows_b, V, chunks, inv_tau_a, inv_tau_b, partial);
+    launch_k(row_stats_kernel<false>, dim3(grid), dim3(STATS_THREADS), 0, st, a, rows_a, b, rows_b, V, chunks, inv_tau_a, inv_tau_b, partial);
   return cudaGetLastError();
 }
 
 cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float* q_logits, float* logq, int* reveal_step,
                                  int batch, int gamma, int V, int k, float inv_tau_q, PhiloxKey key,
                                  const RoundState* rs, cudaStream_t st) {
-  dim3 grid(gamma, batch);
-  unmask_sample_kernel<<<grid, SAMPLE_THREADS, 0, st>>>(step_logits, slot_ids, q_logits, logq, reveal_step, gamma, V, k,
+  dim3 grid(VC * gamma, batch);
+  launch_k(unmask_sample_kernel, dim3(grid), dim3(SAMPLE_THREADS), 0, st, step_logits, slot_ids, q_logits, logq, reveal_step, gamma, V, k,
                                                        inv_tau_q, key, rs);
   return cudaGetLastError();
 }
@@ -478,7 +569,7 @@ cudaError_t launch_accept(const float* logits_p, const float* q_rows, const int*
                           float inv_tau_q_rows, PhiloxKey key, uint32_t rnd, const RoundState* rs, float* accept_prob,
                           int* n_accept, int* extra_token, int* out_ids, cudaStream_t st) {
   const size_t smem = (size_t)(2 * gamma + 1) * sizeof(float);
-  accept_kernel<<<rows, ACCEPT_THREADS, smem, st>>>(logits_p, q_rows, draft_ids, logq_in, partial_p, partial_q,
+  launch_k(accept_kernel, dim3(VC * rows), dim3(ACCEPT_THREADS), smem, st, logits_p, q_rows, draft_ids, logq_in, partial_p, partial_q,
                                                     stats_chunks(V), gamma, V, inv_tau_p, inv_tau_q_rows, key, rnd, rs,
                                                     accept_prob, n_accept, extra_token, out_ids);
   return cudaGetLastError();
@@ -487,13 +578,13 @@ cudaError_t launch_accept(const float* logits_p, const float* q_rows, const int*
 cudaError_t launch_commit(int* tokens, int tok_stride, int* ctx_len, int* n_emitted, const int* slot_ids,
                           const int* n_accept, const int* extra_token, int batch, int gamma, int max_new, RoundState* rs,
                           int* out_ids, int* n_out, volatile int* host_mirror, cudaStream_t st) {
-  commit_kernel<<<1, 256, 0, st>>>(tokens, tok_stride, ctx_len, n_emitted, slot_ids, n_accept, extra_token, batch, gamma,
+  launch_k(commit_kernel, dim3(1), dim3(256), 0, st, tokens, tok_stride, ctx_len, n_emitted, slot_ids, n_accept, extra_token, batch, gamma,
                                    max_new, rs, out_ids, n_out, host_mirror);
   return cudaGetLastError();
 }
 
 cudaError_t launch_reset_slots(int* slot_ids, int* reveal_step, int n, int mask_id, cudaStream_t st) {
-  reset_slots_kernel<<<(n + 255) / 256, 256, 0, st>>>(slot_ids, reveal_step, n, mask_id);
+  launch_k(reset_slots_kernel, dim3((n + 255) / 256), dim3(256), 0, st, slot_ids, reveal_step, n, mask_id);
   return cudaGetLastError();
 }
 
