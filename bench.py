@@ -258,34 +258,20 @@ def run_ours(args):
                 "timing": f"CUDA-event pairs around every launch in a separate pass of {prof_rounds} rounds"}
     sess.close()
 
-    # ---- stand-alone accept kernel: 64 rows x gamma 32 x V (fp32 logits with a shared component) --
+    # ---- stand-alone kernels (paper_2408_05636_b200.microbench) --------------------------------
+    from paper_2408_05636_b200 import microbench
     rows, g4 = 64, 32
-    gen = torch.Generator(device=device)
-    gen.manual_seed(31)
-    cc = torch.randn(rows, g4 + 1, V, device=device, generator=gen)
-    lp = (cc + 0.5 * torch.randn(rows, g4 + 1, V, device=device, generator=gen)).contiguous()
-    lq = (cc[:, :g4] + 0.5 * torch.randn(rows, g4, V, device=device, generator=gen)).contiguous()
-    del cc
-    ids = torch.distributions.Categorical(logits=lq).sample().to(torch.int32).contiguous()
-    scratch = torch.empty(sdd.sdd_accept_scratch_bytes(rows, g4, V), dtype=torch.uint8, device=device)
-    for i in range(3):
-        sdd.sdd_accept_logits(lp, lq, ids, 1.0, 1.0, 31, i, scratch)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    iters = 20
-    torch.cuda.synchronize()
-    e0.record()
-    for i in range(iters):
-        n_acc, _, _ = sdd.sdd_accept_logits(lp, lq, ids, 1.0, 1.0, 31, 10 + i, scratch)
-    e1.record()
-    torch.cuda.synchronize()
-    acc_ms = e0.elapsed_time(e1) / iters
-    acc_bytes = rows * (2 * g4 + 1) * V * 4.0
-    accept_roof = {"bound": "hbm", "achieved": round(acc_bytes / (acc_ms * 1e-3) / 1e9, 1), "peak": peaks["hbm_gbs"],
-                   "unit": "GB/s", "frac": round(acc_bytes / (acc_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
-                   "traffic": None, "ms": round(acc_ms, 4), "launches_per_call": 2,
+    acc = microbench.accept(rows, g4, V, 0.5, iters=20, warmup=3)
+    accept_roof = {"bound": "hbm", "achieved": round(acc["gbs"], 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                   "frac": round(acc["gbs"] / peaks["hbm_gbs"], 4), "traffic": None, "ms": round(acc["us"] * 1e-3, 4),
+                   "launches_per_call": 2,
                    "workload": f"{rows} rows x gamma {g4} x V {V} fp32 logits, inputs 0.84 GB > L2",
-                   "mean_accepted": float(n_acc.float().mean().item()), "peak_source": f"of {peaks['source']}"}
-    del lp, lq, ids, scratch
+                   "mean_accepted": acc["mean_accepted"], "peak_source": f"of {peaks['source']}"}
+    gm = microbench.gemm(16384, 4096, 1024, epilogue=1, iters=20, warmup=3)
+    gemm_roof = {"bound": "tensor", "achieved": round(gm["tflops"], 1), "peak": peaks["tf_burst"], "unit": "TFLOP/s",
+                 "frac": round(gm["tflops"] / peaks["tf_burst"], 4), "traffic": None, "us": round(gm["us"], 2),
+                 "workload": "bf16 GEMM 16384 x 4096 x 1024 with bias + GELU epilogue (drafter FC1 at batch 16), timed alone",
+                 "peak_source": f"of {peaks['source']} (burst)"}
 
     # ---- end to end through the C ABI with host buffers ----------------------------------------
     prompts = synth.prompt_ids(V, 1, wl.prompt_len, wl.prompt_seed)
@@ -324,7 +310,8 @@ def run_ours(args):
                    "multi_gpu": "independent replicas, no collective on the data path"},
         "tokens_per_step": round(toks / args.steps / world, 3),
         "clocks": clock_info, "e2e": e2e, "gpu_launches": int(launches),
-        "roofline": roofline, "roofline_accept_kernel": accept_roof, "kernels": kernels, "cpu_baseline": cpu,
+        "roofline": roofline, "roofline_accept_kernel": accept_roof, "roofline_gemm_kernel": gemm_roof,
+        "kernels": kernels, "cpu_baseline": cpu,
     }
     print(json.dumps(line))
     if dist is not None:
