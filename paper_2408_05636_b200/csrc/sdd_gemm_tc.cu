@@ -177,7 +177,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   for (int e = 0; e < 4; ++e) {
                     float x0 = __uint_as_float(v[g * 8 + 2 * e]) + (bias ? bias[c0 + g * 8 + 2 * e] : 0.f);
                     float x1 = __uint_as_float(v[g * 8 + 2 * e + 1]) + (bias ? bias[c0 + g * 8 + 2 * e + 1] : 0.f);
-                    if (epi == EPI_GELU) { x0 = gelu_tanh(x0); x1 = gelu_tanh(x1); }
+                    if (epi == EPI_GELU) { x0 = gelu_tanh_fast(x0); x1 = gelu_tanh_fast(x1); }
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
                     pk[e] = *reinterpret_cast<uint32_t*>(&h2);
                   }
@@ -187,7 +187,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 for (int j = 0; j < 32; ++j) {
                   if (c0 + j < rows_b) {
                     float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
-                    if (epi == EPI_GELU) x = gelu_tanh(x);
+                    if (epi == EPI_GELU) x = gelu_tanh_fast(x);
                     o[j] = __float2bfloat16_rn(x);
                   }
                 }
@@ -241,7 +241,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   }
                 }
               } else if (epi == EPI_STORE) reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(x);
-              else if (epi == EPI_GELU) reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(gelu_tanh(x));
+              else if (epi == EPI_GELU) reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(gelu_tanh_fast(x));
               else if (epi == EPI_RESIDUAL) { if (split) atomicAdd(reinterpret_cast<float*>(out) + o, x); else reinterpret_cast<float*>(out)[o] += x; }
               else reinterpret_cast<float*>(out)[o] = x;
             }
