@@ -172,6 +172,7 @@ struct sdd_ctx {
   bool use_graph;              // SDD_GRAPH != 0: sdd_step replays a captured graph per row-count bucket
   struct GraphEntry { cudaGraphExec_t exec; uint64_t launches; };
   std::map<std::tuple<int, void*, void*>, GraphEntry> graphs;
+  std::vector<std::tuple<int, void*, void*>> prof_graphs;   // one-off graphs of the current timing pass
   // optional per-launch timing
   bool profiling;
   std::vector<cudaEvent_t> prof_ev;   // pairs (before, after)
@@ -578,12 +579,15 @@ int32_t sdd_verify_accept(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
 int32_t sdd_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
   if (c == nullptr) return SDD_E_ARG;
   if (c->steps_done != -1) return SDD_E_STATE;
-  if (!c->use_graph || c->profiling) {
+  if (!c->use_graph) {
     SDD_TRY(sdd_draft(c));
     return sdd_verify_accept(c, out_ids, n_out);
   }
   SDD_TRY(round_prologue(c));
-  const auto key = std::make_tuple(c->lcap, (void*)out_ids, (void*)n_out);
+  // per-launch timing: the event pairs are captured into a one-off graph, so the stamps are taken on the device
+  // timeline without host launch gaps in between
+  const auto key = std::make_tuple(c->profiling ? -c->lcap - (int)c->prof_graphs.size() - 1 : c->lcap, (void*)out_ids,
+                                   (void*)n_out);
   auto it = c->graphs.find(key);
   if (it == c->graphs.end()) {
     const uint64_t l0 = c->launches;
@@ -604,6 +608,7 @@ int32_t sdd_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
     cudaGraphDestroy(g);
     if (e != cudaSuccess) return cuda_fail(e, "cudaGraphInstantiate");
     it = c->graphs.emplace(key, ge).first;
+    if (c->profiling) c->prof_graphs.push_back(key);
   }
   SDD_CUDA(cudaGraphLaunch(it->second.exec, c->st));
   c->launches += it->second.launches;
@@ -742,6 +747,14 @@ int32_t sdd_profile_end(sdd_ctx* c, double* ms_per_category, uint64_t* launches_
   }
   c->prof_used = 0;
   c->prof_cat.clear();
+  for (auto& k : c->prof_graphs) {
+    auto it = c->graphs.find(k);
+    if (it != c->graphs.end()) {
+      if (it->second.exec) cudaGraphExecDestroy(it->second.exec);
+      c->graphs.erase(it);
+    }
+  }
+  c->prof_graphs.clear();
   return SDD_OK;
 }
 
