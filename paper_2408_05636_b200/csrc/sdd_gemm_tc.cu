@@ -44,9 +44,9 @@ constexpr int smem_bytes() { return ring_stages<BN>() * stage_bytes<BN>() + 1024
 // range and adds it to the fp32 output with atomics (EPI_RESIDUAL only; the bias is added by split 0).
 template <int BN, bool SWAP>
 __global__ void __launch_bounds__(THREADS)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int rows_a,
-               int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out, int ldc, int* status,
-               const QkvDst qd) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_out, int tma_out, int rows_a, int rows_b, int K, int epi,
+               const float* __restrict__ bias, void* __restrict__ out, int ldc, int* status, const QkvDst qd) {
   constexpr int STAGES = ring_stages<BN>();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -133,9 +133,75 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // epilogue warps 2..5 own TMEM lane quarters (warp id % 4)
     const int q = warp & 3;
     // every lane waits; the outcome is made warp-uniform because tcgen05.ld is a warp-wide instruction
-    const bool ready = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar, 0u, abort_flag, status));
+    // (and uniform over the four epilogue warps, which meet at named barriers in the TMA-store path)
+    const bool ready = named_bar_and(1, 128, mbar_wait(tmem_full_bar, 0u, abort_flag, status));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ready) {
+    if (ready && !SWAP && tma_out) {
+      // Output through shared memory and TMA: every thread writes its row's 128-byte piece of the tile into a
+      // staging buffer (128-byte swizzle, so that the 32 rows of a warp spread over all banks), one thread issues a
+      // tile store (bf16 outputs) or an add-reduce (fp32 residual stream; also correct under K splits).  The operand
+      // ring is free by now: tmem_full completes only after every MMA has read its stage.
+      const int rl = q * 32 + lane;               // row inside the tile
+      const int sw = rl & 7;
+      const bool is_issuer = threadIdx.x == 64;
+      const bool f32 = epi == EPI_RESIDUAL;
+      constexpr int CHUNKS = BN / 32;
+      int n_store = 0;
+#pragma unroll 1
+      for (int cc = 0; cc < CHUNKS; ++cc) {
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
+        const int c0 = n0 + cc * 32;
+        // fp32: one 32-column chunk fills a 128-byte row; bf16: two chunks do
+        const int buf = f32 ? (cc & 1) : ((cc >> 1) & 1);
+        const bool first_of_buf = f32 || (cc & 1) == 0;
+        const bool last_of_buf = f32 || (cc & 1) == 1 || cc == CHUNKS - 1;
+        if (first_of_buf) {
+          if (is_issuer && n_store >= 2) tma_wait_group_read<1>();   // the store that last used this buffer has read it
+          named_bar_sync(2, 128);
+        }
+        uint8_t* row = generic_base + buf * (128 * 128) + rl * 128;
+        if (f32) {
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            float4 x;
+            x.x = __uint_as_float(v[g * 4 + 0]) + ((bias && c0 + g * 4 + 0 < rows_b) ? bias[c0 + g * 4 + 0] : 0.f);
+            x.y = __uint_as_float(v[g * 4 + 1]) + ((bias && c0 + g * 4 + 1 < rows_b) ? bias[c0 + g * 4 + 1] : 0.f);
+            x.z = __uint_as_float(v[g * 4 + 2]) + ((bias && c0 + g * 4 + 2 < rows_b) ? bias[c0 + g * 4 + 2] : 0.f);
+            x.w = __uint_as_float(v[g * 4 + 3]) + ((bias && c0 + g * 4 + 3 < rows_b) ? bias[c0 + g * 4 + 3] : 0.f);
+            *reinterpret_cast<float4*>(row + ((g ^ sw) << 4)) = x;
+          }
+        } else {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int j0 = g * 8 + 2 * e;
+              float x0 = __uint_as_float(v[j0]) + ((bias && c0 + j0 < rows_b) ? bias[c0 + j0] : 0.f);
+              float x1 = __uint_as_float(v[j0 + 1]) + ((bias && c0 + j0 + 1 < rows_b) ? bias[c0 + j0 + 1] : 0.f);
+              if (epi == EPI_GELU) { x0 = gelu_tanh_fast(x0); x1 = gelu_tanh_fast(x1); }
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+              pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            const int chunk = (cc & 1) * 4 + g;
+            *reinterpret_cast<uint4*>(row + ((chunk ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
+        }
+        if (last_of_buf) {
+          fence_async_smem();
+          named_bar_sync(2, 128);
+          if (is_issuer) {
+            const uint32_t src = base + buf * (128 * 128);
+            if (f32) tma_reduce_add_2d(&map_out, src, c0, m0);
+            else tma_store_2d(&map_out, src, n0 + (cc & ~1) * 32, m0);
+            tma_commit_group();
+          }
+          ++n_store;
+        }
+      }
+      if (is_issuer) tma_wait_group_read<0>();      // shared memory stays valid until the copies have read it
+    } else if (ready) {
       const int r = m0 + q * 32 + lane;          // index along the A operand's rows
       const bool r_ok = r < rows_a;
 #pragma unroll 1
@@ -262,11 +328,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // host side: tensor maps (cached per pointer / shape / box) and launch
 // ---------------------------------------------------------------------------------------------
 template <int BN, bool SWAP>
-static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, int rows_a, int rows_b, int K, int epi,
+static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, int tma_out, int rows_a,
+                              int rows_b, int K, int epi,
                               const float* bias, void* out, int ldc, int* status, cudaStream_t st, const QkvDst& qd,
                               int splits) {
   dim3 grid((rows_b + BN - 1) / BN, (rows_a + BM - 1) / BM, splits);
-  launch_k(gemm_tc_kernel<BN, SWAP>, dim3(grid), dim3(THREADS), smem_bytes<BN>(), st, ma, mb, rows_a, rows_b, K, epi, bias, out, ldc, status, qd);
+  launch_k(gemm_tc_kernel<BN, SWAP>, dim3(grid), dim3(THREADS), smem_bytes<BN>(), st, ma, mb, mo, tma_out, rows_a, rows_b, K, epi, bias, out, ldc, status, qd);
   return cudaGetLastError();
 }
 
@@ -294,7 +361,7 @@ static std::mutex g_map_mu;
 static std::map<std::tuple<const void*, long long, long long, long long, int>, CUtensorMap> g_maps;
 
 cudaError_t get_tensor_map(const void* ptr, long long rows, long long cols, long long ld, int box_rows, int box_cols,
-                           CUtensorMap* out) {
+                           CUtensorMap* out, int elem_bytes) {
   std::lock_guard<std::mutex> lock(g_map_mu);
   if (g_encode == nullptr) {
     void* fn = nullptr;
@@ -304,16 +371,18 @@ cudaError_t get_tensor_map(const void* ptr, long long rows, long long cols, long
     if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
     g_encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
   }
-  auto key = std::make_tuple(ptr, rows, cols, ld, box_rows * 1024 + box_cols);
+  auto key = std::make_tuple(ptr, rows, cols, ld, (box_rows * 1024 + box_cols) * 8 + elem_bytes);
   auto it = g_maps.find(key);
   if (it != g_maps.end()) { *out = it->second; return cudaSuccess; }
-  if ((reinterpret_cast<uintptr_t>(ptr) & 15u) != 0 || (ld * 2) % 16 != 0 || box_cols * 2 > 128) return cudaErrorInvalidValue;
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15u) != 0 || (ld * elem_bytes) % 16 != 0 || box_cols * elem_bytes > 128 ||
+      (elem_bytes != 2 && elem_bytes != 4))
+    return cudaErrorInvalidValue;
   CUtensorMap m;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * elem_bytes};
   cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+  CUresult r = g_encode(&m, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
@@ -357,8 +426,8 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     const int splits = pick_splits((N + BM - 1) / BM, 2);
     if ((e = get_tensor_map(W, N, K, K, BM, BK, &ma)) != cudaSuccess) return e;
     if ((e = get_tensor_map(A, a_cap, K, K, bn, BK, &mb)) != cudaSuccess) return e;
-    if (bn == 32) return launch_cfg<32, true>(ma, mb, N, M, K, epi, bias, out, ldc, status, st, qd, splits);
-    return launch_cfg<64, true>(ma, mb, N, M, K, epi, bias, out, ldc, status, st, qd, splits);
+    if (bn == 32) return launch_cfg<32, true>(ma, mb, ma, 0, N, M, K, epi, bias, out, ldc, status, st, qd, splits);
+    return launch_cfg<64, true>(ma, mb, ma, 0, N, M, K, epi, bias, out, ldc, status, st, qd, splits);
   }
   int bn = bn_hint;
   const long long mt = (M + BM - 1) / BM;
@@ -372,11 +441,22 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
   const int splits = pick_splits(mt * ((N + bn - 1) / bn), 4);
   if ((e = get_tensor_map(A, a_cap, K, K, BM, BK, &ma)) != cudaSuccess) return e;
   if ((e = get_tensor_map(W, N, K, K, bn, BK, &mb)) != cudaSuccess) return e;
+  // output through TMA where the layout allows 16-byte-aligned rows (see the kernel's epilogue)
+  CUtensorMap mo = ma;
+  int tma_out = 0;
+  if (epi == EPI_RESIDUAL && (ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+    if ((e = get_tensor_map(out, M, N, ldc, BM, 32, &mo, 4)) != cudaSuccess) return e;
+    tma_out = 1;
+  } else if ((epi == EPI_STORE || epi == EPI_GELU) && bn >= 64 && (ldc & 7) == 0 &&
+             (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+    if ((e = get_tensor_map(out, M, N, ldc, BM, 64, &mo, 2)) != cudaSuccess) return e;
+    tma_out = 1;
+  }
   switch (bn) {
-    case 256: return launch_cfg<256, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
-    case 128: return launch_cfg<128, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
-    case 64: return launch_cfg<64, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
-    default: return launch_cfg<32, false>(ma, mb, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
+    case 256: return launch_cfg<256, false>(ma, mb, mo, tma_out, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
+    case 128: return launch_cfg<128, false>(ma, mb, mo, tma_out, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
+    case 64: return launch_cfg<64, false>(ma, mb, mo, tma_out, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
+    default: return launch_cfg<32, false>(ma, mb, mo, tma_out, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
   }
 }
 

@@ -105,11 +105,42 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // make generic-proxy writes to shared memory visible to the async proxy (TMA / tensor core reads)
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// TMA tile store / add-reduce from shared memory (bulk async-group completion)
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tma_wait_group_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+// barrier among a subset of the CTA's warps
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+// ... that also AND-reduces a predicate over the participating threads
+__device__ __forceinline__ bool named_bar_and(int id, int threads, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %3, 0;\n\t"
+      "bar.red.and.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(threads), "r"((uint32_t)pred)
+      : "memory");
+  return r != 0;
+}
+
 }  // namespace tc
 
-// 2-D bf16 tensor [rows, cols] with row stride ld elements; box = box_rows x box_cols, 128-byte swizzle.
+// 2-D bf16 (elem_bytes 2) or fp32 (elem_bytes 4) tensor [rows, cols] with row stride ld elements;
+// box = box_rows x box_cols (at most 128 bytes wide), 128-byte swizzle.
 // Maps are cached per (pointer, shape, box).
 cudaError_t get_tensor_map(const void* ptr, long long rows, long long cols, long long ld, int box_rows, int box_cols,
-                           CUtensorMap* out);
+                           CUtensorMap* out, int elem_bytes = 2);
 
 }  // namespace sdd
