@@ -97,6 +97,7 @@ struct Buffers {
   float2* partial_p;
   float* h;                    // residual stream, fp32
   void *xn, *qkv, *att, *mlp, *xf;  // activations in the model dtype
+  void *xn_lo, *mlp_lo, *xf_lo;  // rounding remainders of xn / mlp / xf (hi/lo pairs of the target's MLP and LM head)
   void* vt;                    // drafter V transposed [batch][d_q][lcap_max] (tensor-core path)
   void* kv;                    // target KV cache [layer][batch][n_ctx][2][d]
 };
@@ -141,6 +142,10 @@ static size_t carve(const Dims& D, const Net& P, const Net& Q, uint8_t* base, Bu
   b.mlp = take(mx(rq * Q.d, rp * P.d) * 4 * D.esize);
   b.xf = take(Bn * (G + 1) * mx(Q.d, P.d) * D.esize);
   b.vt = take(Bn * (size_t)Q.d * D.lcap_max * D.esize);
+  // same capacities as their hi halves, so that one tensor-map extent describes both
+  b.xn_lo = take(mx(rq * Q.d, rp * P.d) * D.esize);
+  b.mlp_lo = take(mx(rq * Q.d, rp * P.d) * 4 * D.esize);
+  b.xf_lo = take(Bn * (G + 1) * mx(Q.d, P.d) * D.esize);
   b.kv = take((size_t)P.n_layer * Bn * P.n_ctx * 2 * P.d * D.esize);
   if (B) *B = b;
   return off;
@@ -167,6 +172,7 @@ struct sdd_ctx {
   int runahead;
   int lcap;                    // padded rows per sequence of the current round's drafter forwards
   size_t act_elems, xf_elems;  // capacity (elements) of the xn / att buffers (mlp: 4x) and of xf
+  bool hilo;                   // SDD_HILO != 0 (default): hi/lo activation pairs in the target's MLP and LM head
   bool force_simt;             // SDD_GEMM=simt: run bf16 GEMMs on the CUDA-core kernel (cross-check)
   int bn_hint;                 // SDD_GEMM_BN: N tile of the tensor-core GEMM (0 = choose)
   bool use_graph;              // SDD_GRAPH != 0: sdd_step replays a captured graph per row-count bucket
@@ -234,13 +240,14 @@ static void fill_dims(const Net& P, const Net& Q, const sdd_params* p, int max_p
 // `a_elems` is the capacity of the A buffer in elements (the tensor map of an activation buffer covers all of it)
 template <typename T>
 static int gemm(sdd_ctx* c, int cat, const void* A, size_t a_elems, const void* W, const float* bias, long long M, int N,
-                int K, int epi, void* out, int ldc, const QkvDst* qd = nullptr) {
+                int K, int epi, void* out, int ldc, const QkvDst* qd = nullptr, const void* A_lo = nullptr,
+                void* out_lo = nullptr) {
   if (M <= 0) return SDD_OK;
   ProfScope prof(c, cat);
   c->launches++;
   if (std::is_same<T, __nv_bfloat16>::value && !c->force_simt) {
     SDD_CUDA(launch_gemm_tc((const __nv_bfloat16*)A, (long long)(a_elems / (size_t)K), (const __nv_bfloat16*)W, bias, (int)M,
-                            N, K, epi, out, ldc, c->bn_hint, &c->B.rs->status, c->st, qd));
+                            N, K, epi, out, ldc, c->bn_hint, &c->B.rs->status, c->st, qd, (const __nv_bfloat16*)A_lo, out_lo));
   } else {
     SDD_CUDA(launch_gemm_simt<T>((const T*)A, K, (const T*)W, bias, (int)M, N, K, epi, out, ldc, c->st));
   }
@@ -262,7 +269,7 @@ static bool use_tc(const sdd_ctx* c, const Net& N) {
 
 // one transformer block on `rows` rows; attention is issued by the caller-supplied functor
 template <typename T, typename QkvFn, typename AttnFn>
-static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, QkvFn qkv_dst, AttnFn attn) {
+static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, bool hilo_mlp, QkvFn qkv_dst, AttnFn attn) {
   const Buffers& B = c->B;
   const int d = N.d;
   for (int l = 0; l < N.n_layer; ++l) {
@@ -274,9 +281,13 @@ static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, QkvFn 
                     3 * d, fused ? &qd : nullptr));
     SDD_TRY(attn(l));
     SDD_TRY(gemm<T>(c, gcat, B.att, c->act_elems, L.w_o, L.b_o, rows, d, d, EPI_RESIDUAL, B.h, d));
-    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln2_g, L.ln2_b, (T*)B.xn, rows, d, c->st));
-    SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_fc1, L.b_fc1, rows, 4 * d, d, EPI_GELU, B.mlp, 4 * d));
-    SDD_TRY(gemm<T>(c, gcat, B.mlp, 4 * c->act_elems, L.w_fc2, L.b_fc2, rows, d, 4 * d, EPI_RESIDUAL, B.h, d));
+    // hilo_mlp: the MLP's two products take their activations as hi/lo bf16 pairs (see sdd_gemm_tc.cu)
+    T* xn_lo = hilo_mlp ? (T*)B.xn_lo : nullptr;
+    void* mlp_lo = hilo_mlp ? B.mlp_lo : nullptr;
+    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln2_g, L.ln2_b, (T*)B.xn, rows, d, c->st, xn_lo));
+    SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_fc1, L.b_fc1, rows, 4 * d, d, EPI_GELU, B.mlp, 4 * d, nullptr, xn_lo,
+                    mlp_lo));
+    SDD_TRY(gemm<T>(c, gcat, B.mlp, 4 * c->act_elems, L.w_fc2, L.b_fc2, rows, d, 4 * d, EPI_RESIDUAL, B.h, d, nullptr, mlp_lo));
   }
   return SDD_OK;
 }
@@ -292,7 +303,7 @@ static int forward_drafter(sdd_ctx* c) {
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_drafter<T>((const T*)Q.wte, (const T*)Q.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
                                         D.batch, D.gamma, lcap, Q.d, B.h, c->st));
   const bool tc = use_tc<T>(c, Q);
-  SDD_TRY((run_blocks<T>(c, Q, rows, CAT_GEMM_Q,
+  SDD_TRY((run_blocks<T>(c, Q, rows, CAT_GEMM_Q, false,
     [&](int, QkvDst* qd) -> bool {
       if (!tc) return false;
       qd->k_dst = nullptr; qd->vt_dst = (__nv_bfloat16*)B.vt; qd->ctx_len = B.ctx_len; qd->rows_per_seq = lcap;
@@ -331,7 +342,7 @@ static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) 
   const bool tc = use_tc<T>(c, P);
   // tensor-core path: per layer the cache is K [B][n_ctx][d] followed by V^T [B][d][n_ctx];
   // CUDA-core path: [B][n_ctx][K|V][d]
-  SDD_TRY((run_blocks<T>(c, P, rows, CAT_GEMM_P,
+  SDD_TRY((run_blocks<T>(c, P, rows, CAT_GEMM_P, tc && c->hilo,
     [&](int l, QkvDst* qd) -> bool {
       if (!tc) return false;
       __nv_bfloat16* kc = (__nv_bfloat16*)B.kv + (size_t)l * layer_elems;
@@ -356,8 +367,10 @@ static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) 
       return SDD_OK;
     })));
   if (lm_head) {
-    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, P.lnf_g, P.lnf_b, (T*)B.xf, rows, P.d, c->st));
-    SDD_TRY(gemm<T>(c, CAT_HEAD_P, B.xf, c->xf_elems, P.wte, nullptr, rows, D.V, P.d, EPI_STORE_F32, B.logits_p, D.V));
+    T* xf_lo = (tc && c->hilo) ? (T*)B.xf_lo : nullptr;
+    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, P.lnf_g, P.lnf_b, (T*)B.xf, rows, P.d, c->st, xf_lo));
+    SDD_TRY(gemm<T>(c, CAT_HEAD_P, B.xf, c->xf_elems, P.wte, nullptr, rows, D.V, P.d, EPI_STORE_F32, B.logits_p, D.V, nullptr,
+                    xf_lo));
   }
   return SDD_OK;
 }
@@ -473,6 +486,8 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
     c->xf_elems = (size_t)params->batch * (params->gamma + 1) * (c->Q.d > c->P.d ? c->Q.d : c->P.d);
     const char* g = getenv("SDD_GEMM");
     c->force_simt = g != nullptr && strcmp(g, "simt") == 0;
+    const char* hl = getenv("SDD_HILO");
+    c->hilo = hl == nullptr || atoi(hl) != 0;
     const char* bn = getenv("SDD_GEMM_BN");
     c->bn_hint = bn ? atoi(bn) : 0;
     const char* gr = getenv("SDD_GRAPH");

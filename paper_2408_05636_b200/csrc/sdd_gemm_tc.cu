@@ -10,6 +10,11 @@
 // verification forward, where only gamma+1 tokens exist and the kernel is a weight-streaming pass; the
 // epilogue then writes the transposed tile so that consecutive lanes write consecutive features.
 //
+// HILO: the activation operand may come as two bf16 tensors, hi = bf16(x) and lo = bf16(x - hi), and the kernel
+// accumulates W x hi + W x lo into the same TMEM tile (16 significant bits of the activations instead of 8).  The
+// target network's MLP and LM-head products use it: their logits are compared against an fp64 oracle, and the
+// rounding of the activations to bf16 is the largest error term of a 48-layer forward.
+//
 // Every wait on an mbarrier is bounded: when the limit passes the thread raises the CTA's abort flag and
 // the device status word, all roles leave their loops, the producer waits (bounded) for the copies it
 // still has in flight, TMEM is freed and the CTA returns.
@@ -31,33 +36,42 @@ constexpr int BK = 64;           // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int THREADS = 192;     // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
 
-template <int BN>
-constexpr int stage_bytes() { return BM * BK * 2 + BN * BK * 2; }
-// shared-memory ring depth per N tile: as deep as one CTA per SM allows (about 190 KB), so that a short K loop
-// has all of its tiles in flight at once
-template <int BN>
-constexpr int ring_stages() { return BN <= 64 ? 8 : (BN == 128 ? 6 : 4); }
-template <int BN>
-constexpr int smem_bytes() { return ring_stages<BN>() * stage_bytes<BN>() + 1024 /*alignment slack*/ + 256 /*barriers*/; }
+// one stage = A tile + B tile (+ the lo tile of the activation operand: the A side unless SWAP)
+template <int BN, bool SWAP, bool HILO>
+constexpr int stage_bytes() { return BM * BK * 2 + BN * BK * 2 + (HILO ? (SWAP ? BN : BM) * BK * 2 : 0); }
+// shared-memory ring depth: as deep as one CTA per SM allows (about 190 KB), so that a short K loop has all of its
+// tiles in flight at once
+template <int BN, bool SWAP, bool HILO>
+constexpr int ring_stages() {
+  constexpr int s = (200 * 1024) / stage_bytes<BN, SWAP, HILO>();
+  return s > 8 ? 8 : s;
+}
+template <int BN, bool SWAP, bool HILO>
+constexpr int smem_bytes() {
+  return ring_stages<BN, SWAP, HILO>() * stage_bytes<BN, SWAP, HILO>() + 1024 /*alignment slack*/ + 256 /*barriers*/;
+}
 
 // grid = (N tiles, M tiles, K splits).  With more than one K split every CTA accumulates its share of the K
 // range and adds it to the fp32 output with atomics (EPI_RESIDUAL only; the bias is added by split 0).
-template <int BN, bool SWAP>
+template <int BN, bool SWAP, bool HILO>
 __global__ void __launch_bounds__(THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_out, int tma_out, int rows_a, int rows_b, int K, int epi,
-               const float* __restrict__ bias, void* __restrict__ out, int ldc, int* status, const QkvDst qd) {
-  constexpr int STAGES = ring_stages<BN>();
+               const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_out, int tma_out,
+               int rows_a, int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out,
+               void* __restrict__ out_lo, int ldc, int* status, const QkvDst qd) {
+  constexpr int STAGES = ring_stages<BN, SWAP, HILO>();
+  constexpr int STAGE_BYTES = stage_bytes<BN, SWAP, HILO>();
+  constexpr int LO_OFF = BM * BK * 2 + BN * BK * 2;     // offset of the lo tile inside a stage
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = base + STAGES * stage_bytes<BN>();
+  const uint32_t bar_base = base + STAGES * STAGE_BYTES;
   // barrier block: full[STAGES], empty[STAGES], tmem_full, then the TMEM base address and the abort flag
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
   uint8_t* generic_base = smem_raw + (base - smem_u32(smem_raw));
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(generic_base + STAGES * stage_bytes<BN>() + 8 * (2 * STAGES + 1));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(generic_base + STAGES * stage_bytes<BN>() + 8 * (2 * STAGES + 1) + 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(generic_base + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 1));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(generic_base + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 1) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.y * BM;      // offset along the A operand's rows (MMA M axis)
@@ -94,10 +108,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int s = kb % STAGES;
         const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
         if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, status)) break;
-        mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes<BN>());
-        const uint32_t sa = base + s * stage_bytes<BN>();
+        mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES);
+        const uint32_t sa = base + s * STAGE_BYTES;
         tma_load_2d(sa, &map_a, full_bar(s), (kb0 + kb) * BK, m0);
         tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), (kb0 + kb) * BK, n0);
+        if (HILO) tma_load_2d(sa + LO_OFF, &map_lo, full_bar(s), (kb0 + kb) * BK, SWAP ? n0 : m0);
         issued = kb + 1;
       }
       if (*abort_flag) {
@@ -119,12 +134,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ok = mbar_wait(full_bar(s), ph, abort_flag, status);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t sa = base + s * stage_bytes<BN>();
+        const uint32_t sa = base + s * STAGE_BYTES;
         const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + BM * BK * 2);
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; ++k)
           umma(tmem_base, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
                (kb > 0 || k > 0) ? 1u : 0u);
+        if (HILO) {
+          const uint64_t dl = make_smem_desc(sa + LO_OFF);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t o = (uint64_t)(k * UMMA_K * 2 / 16);
+            if (SWAP) umma(tmem_base, da + o, dl + o, idesc, 1u);
+            else umma(tmem_base, dl + o, db + o, idesc, 1u);
+          }
+        }
         umma_commit(empty_bar(s));     // frees the stage once these MMAs have read it
       }
       if (ok) umma_commit(tmem_full_bar);
@@ -249,12 +273,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   }
                   *reinterpret_cast<uint4*>(o + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
+                if (out_lo != nullptr) {   // second half of the hi/lo pair: lo = bf16(x - hi)
+                  __nv_bfloat16* ol = reinterpret_cast<__nv_bfloat16*>(out_lo) + (long long)r * ldc + c0;
+                  for (int j = 0; j < 32; ++j) {
+                    float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
+                    if (epi == EPI_GELU) x = gelu_tanh_fast(x);
+                    ol[j] = __float2bfloat16_rn(x - __bfloat162float(__float2bfloat16_rn(x)));
+                  }
+                }
               } else {
                 for (int j = 0; j < 32; ++j) {
                   if (c0 + j < rows_b) {
                     float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
                     if (epi == EPI_GELU) x = gelu_tanh_fast(x);
-                    o[j] = __float2bfloat16_rn(x);
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                    o[j] = hi;
+                    if (out_lo != nullptr)
+                      reinterpret_cast<__nv_bfloat16*>(out_lo)[(long long)r * ldc + c0 + j] = __float2bfloat16_rn(x - __bfloat162float(hi));
                   }
                 }
               }
@@ -306,8 +341,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                   }
                 }
-              } else if (epi == EPI_STORE) reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(x);
-              else if (epi == EPI_GELU) reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(gelu_tanh_fast(x));
+              } else if (epi == EPI_STORE || epi == EPI_GELU) {
+                if (epi == EPI_GELU) x = gelu_tanh_fast(x);
+                const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                reinterpret_cast<__nv_bfloat16*>(out)[o] = hi;
+                if (out_lo != nullptr) reinterpret_cast<__nv_bfloat16*>(out_lo)[o] = __float2bfloat16_rn(x - __bfloat162float(hi));
+              }
               else if (epi == EPI_RESIDUAL) { if (split) atomicAdd(reinterpret_cast<float*>(out) + o, x); else reinterpret_cast<float*>(out)[o] += x; }
               else reinterpret_cast<float*>(out)[o] = x;
             }
@@ -327,19 +366,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 // host side: tensor maps (cached per pointer / shape / box) and launch
 // ---------------------------------------------------------------------------------------------
-template <int BN, bool SWAP>
-static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, int tma_out, int rows_a,
-                              int rows_b, int K, int epi,
-                              const float* bias, void* out, int ldc, int* status, cudaStream_t st, const QkvDst& qd,
-                              int splits) {
+template <int BN, bool SWAP, bool HILO>
+static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& mo,
+                              int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias, void* out, void* out_lo,
+                              int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits) {
   dim3 grid((rows_b + BN - 1) / BN, (rows_a + BM - 1) / BM, splits);
-  launch_k(gemm_tc_kernel<BN, SWAP>, dim3(grid), dim3(THREADS), smem_bytes<BN>(), st, ma, mb, mo, tma_out, rows_a, rows_b, K, epi, bias, out, ldc, status, qd);
+  launch_k(gemm_tc_kernel<BN, SWAP, HILO>, grid, dim3(THREADS), smem_bytes<BN, SWAP, HILO>(), st, ma, mb, ml, mo, tma_out,
+           rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd);
   return cudaGetLastError();
+}
+template <int BN, bool SWAP>
+static cudaError_t launch_hl(bool hilo, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml,
+                             const CUtensorMap& mo, int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias,
+                             void* out, void* out_lo, int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits) {
+  if (hilo)
+    return launch_cfg<BN, SWAP, true>(ma, mb, ml, mo, tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
+  return launch_cfg<BN, SWAP, false>(ma, mb, ml, mo, tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
 }
 
 template <int BN, bool SWAP>
 static cudaError_t prepare_one() {
-  return cudaFuncSetAttribute(gemm_tc_kernel<BN, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<BN>());
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, SWAP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       smem_bytes<BN, SWAP, false>());
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_tc_kernel<BN, SWAP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              smem_bytes<BN, SWAP, true>());
 }
 
 }  // namespace tc
@@ -394,7 +445,8 @@ cudaError_t get_tensor_map(const void* ptr, long long rows, long long cols, long
 
 // A: activations [M rows used, capacity a_cap rows, K], W: weights [N, K]; both dense bf16.
 cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_bfloat16* W, const float* bias, int M, int N,
-                           int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st, const QkvDst* qkv) {
+                           int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st, const QkvDst* qkv,
+                           const __nv_bfloat16* A_lo, void* out_lo) {
   using namespace tc;
   if (M <= 0 || N <= 0) return cudaSuccess;
   static std::once_flag once;
@@ -406,8 +458,10 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     if (qkv == nullptr || (qkv->d & 63) != 0) return cudaErrorInvalidValue;
     qd = *qkv;
   }
-  CUtensorMap ma, mb;
+  CUtensorMap ma, mb, ml;
   cudaError_t e;
+  const bool hilo = A_lo != nullptr;
+  if (out_lo != nullptr && epi != EPI_STORE && epi != EPI_GELU) return cudaErrorInvalidValue;
   const int total_kb = (K + BK - 1) / BK;
   constexpr int SMS = 148;
   // K splits fill idle SMs of a single-wave grid; only the residual epilogue can add partial sums
@@ -426,8 +480,10 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     const int splits = pick_splits((N + BM - 1) / BM, 2);
     if ((e = get_tensor_map(W, N, K, K, BM, BK, &ma)) != cudaSuccess) return e;
     if ((e = get_tensor_map(A, a_cap, K, K, bn, BK, &mb)) != cudaSuccess) return e;
-    if (bn == 32) return launch_cfg<32, true>(ma, mb, ma, 0, N, M, K, epi, bias, out, ldc, status, st, qd, splits);
-    return launch_cfg<64, true>(ma, mb, ma, 0, N, M, K, epi, bias, out, ldc, status, st, qd, splits);
+    ml = mb;
+    if (hilo && (e = get_tensor_map(A_lo, a_cap, K, K, bn, BK, &ml)) != cudaSuccess) return e;
+    if (bn == 32) return launch_hl<32, true>(hilo, ma, mb, ml, ma, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
+    return launch_hl<64, true>(hilo, ma, mb, ml, ma, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
   }
   int bn = bn_hint;
   const long long mt = (M + BM - 1) / BM;
@@ -441,22 +497,24 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
   const int splits = pick_splits(mt * ((N + bn - 1) / bn), 4);
   if ((e = get_tensor_map(A, a_cap, K, K, BM, BK, &ma)) != cudaSuccess) return e;
   if ((e = get_tensor_map(W, N, K, K, bn, BK, &mb)) != cudaSuccess) return e;
+  ml = ma;
+  if (hilo && (e = get_tensor_map(A_lo, a_cap, K, K, BM, BK, &ml)) != cudaSuccess) return e;
   // output through TMA where the layout allows 16-byte-aligned rows (see the kernel's epilogue)
   CUtensorMap mo = ma;
   int tma_out = 0;
   if (epi == EPI_RESIDUAL && (ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
     if ((e = get_tensor_map(out, M, N, ldc, BM, 32, &mo, 4)) != cudaSuccess) return e;
     tma_out = 1;
-  } else if ((epi == EPI_STORE || epi == EPI_GELU) && bn >= 64 && (ldc & 7) == 0 &&
+  } else if ((epi == EPI_STORE || epi == EPI_GELU) && out_lo == nullptr && bn >= 64 && (ldc & 7) == 0 &&
              (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
     if ((e = get_tensor_map(out, M, N, ldc, BM, 64, &mo, 2)) != cudaSuccess) return e;
     tma_out = 1;
   }
   switch (bn) {
-    case 256: return launch_cfg<256, false>(ma, mb, mo, tma_out, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
-    case 128: return launch_cfg<128, false>(ma, mb, mo, tma_out, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
-    case 64: return launch_cfg<64, false>(ma, mb, mo, tma_out, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
-    default: return launch_cfg<32, false>(ma, mb, mo, tma_out, M, N, K, epi, bias, out, ldc, status, st, qd, splits);
+    case 256: return launch_hl<256, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
+    case 128: return launch_hl<128, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
+    case 64: return launch_hl<64, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
+    default: return launch_hl<32, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
   }
 }
 

@@ -61,7 +61,8 @@ constexpr float LN_EPS = 1e-5f;
 
 template <typename T>
 __device__ __forceinline__ void layernorm_row(const float* __restrict__ src, const float* __restrict__ g,
-                                              const float* __restrict__ bta, T* __restrict__ dst, int d) {
+                                              const float* __restrict__ bta, T* __restrict__ dst, T* __restrict__ dst_lo,
+                                              int d) {
   const int lane = threadIdx.x & 31;
   float x[LN_MAX_PER_LANE];
   float sum = 0.f;
@@ -83,18 +84,23 @@ __device__ __forceinline__ void layernorm_row(const float* __restrict__ src, con
 #pragma unroll
   for (int i = 0; i < LN_MAX_PER_LANE; ++i) {
     const int e = i * 32 + lane;
-    if (e < d) dst[e] = from_f32<T>((x[i] - mu) * rstd * g[e] + bta[e]);
+    if (e < d) {
+      const float y = (x[i] - mu) * rstd * g[e] + bta[e];
+      const T hi = from_f32<T>(y);
+      dst[e] = hi;
+      if (dst_lo != nullptr) dst_lo[e] = from_f32<T>(y - to_f32<T>(hi));   // second half of a hi/lo pair
+    }
   }
 }
 
 template <typename T>
 __global__ void __launch_bounds__(128)
 layernorm_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
-                 T* __restrict__ out, long long rows, int d) {
+                 T* __restrict__ out, T* __restrict__ out_lo, long long rows, int d) {
   pdl_wait();
   const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
   if (row >= rows) return;
-  layernorm_row<T>(h + row * d, g, bta, out + row * d, d);
+  layernorm_row<T>(h + row * d, g, bta, out + row * d, out_lo != nullptr ? out_lo + row * d : nullptr, d);
 }
 
 template <typename T>
@@ -105,7 +111,7 @@ layernorm_slots_kernel(const float* __restrict__ h, const float* __restrict__ g,
   const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
   if (r >= batch * gamma) return;
   const int b = r / gamma, j = r - b * gamma;
-  layernorm_row<T>(h + ((long long)b * L_cap + ctx_len[b] + j) * d, g, bta, out + (long long)r * d, d);
+  layernorm_row<T>(h + ((long long)b * L_cap + ctx_len[b] + j) * d, g, bta, out + (long long)r * d, nullptr, d);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -147,10 +153,10 @@ cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, i
 }
 template <typename T>
 cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* out, long long rows, int d,
-                             cudaStream_t st) {
+                             cudaStream_t st, T* out_lo) {
   if (rows <= 0) return cudaSuccess;
   if (d > LN_MAX_PER_LANE * 32) return cudaErrorInvalidValue;
-  launch_k(layernorm_kernel<T>, dim3((unsigned)((rows + 3) / 4)), dim3(128), 0, st, h, g, b, out, rows, d);
+  launch_k(layernorm_kernel<T>, dim3((unsigned)((rows + 3) / 4)), dim3(128), 0, st, h, g, b, out, out_lo, rows, d);
   return cudaGetLastError();
 }
 template <typename T>
@@ -173,7 +179,8 @@ cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int bat
                                                int, int, float*, cudaStream_t);                                         \
   template cudaError_t launch_embed_target<T>(const T*, const T*, const int*, int, const int*, const int*, int, int,    \
                                               int, int, int, float*, cudaStream_t);                                     \
-  template cudaError_t launch_layernorm<T>(const float*, const float*, const float*, T*, long long, int, cudaStream_t); \
+  template cudaError_t launch_layernorm<T>(const float*, const float*, const float*, T*, long long, int, cudaStream_t, \
+                                           T*);                                                                         \
   template cudaError_t launch_layernorm_slots<T>(const float*, const float*, const float*, T*, const int*, int, int,    \
                                                  int, int, cudaStream_t);                                               \
   template cudaError_t launch_kv_append<T>(const T*, T*, const int*, int, int, int, int, int, cudaStream_t);

@@ -61,9 +61,11 @@ template <typename T>
 cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                 const int* slot_ids, int batch, int gamma, int rows_per_seq, int mode, int d, float* h,
                                 cudaStream_t st);
-// LayerNorm of `rows` rows of h (fp32, row stride d) into out (activation type)
+// LayerNorm of `rows` rows of h (fp32, row stride d) into out (activation type); out_lo (optional) receives the
+// rounding remainder y - out so that (out, out_lo) carries y to about 16 significant bits
 template <typename T>
-cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* out, long long rows, int d, cudaStream_t st);
+cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* out, long long rows, int d, cudaStream_t st,
+                             T* out_lo = nullptr);
 // final LayerNorm of the gamma slot rows of every sequence: out[b*gamma + j] = LN(h[b*L_cap + ctx_len[b] + j])
 template <typename T>
 cudaError_t launch_layernorm_slots(const float* h, const float* g, const float* b, T* out, const int* ctx_len, int batch,
@@ -81,9 +83,11 @@ cudaError_t launch_gemm_simt(const T* A, int lda, const T* W, const float* bias,
 
 // bf16 tensor-core GEMM (tcgen05 / TMEM / TMA).  A is a dense [a_cap, K] buffer of which M rows are used;
 // bn_hint selects the N tile (0 = choose); a bounded wait that expires sets *status = DEV_TIMEOUT.
+// A_lo (optional): second half of a hi/lo activation pair, same shape as A; the product uses A + A_lo.
+// out_lo (optional, bf16 epilogues): receives bf16(x - bf16(x)) next to out = bf16(x).
 cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_bfloat16* W, const float* bias, int M, int N,
                            int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st,
-                           const QkvDst* qkv = nullptr);
+                           const QkvDst* qkv = nullptr, const __nv_bfloat16* A_lo = nullptr, void* out_lo = nullptr);
 
 // one-time set-up of the tensor-core kernels (dynamic shared-memory limits); also done lazily on first launch
 cudaError_t tc_prepare_gemm();
