@@ -169,10 +169,14 @@ int32_t sdd_accept_logits_static(const float* logits_p, const float* logits_q, c
  *   n_tile   0 = let the library choose, else 32 / 64 / 128 / 256 (only for M > 64)
  *   use_tensor_cores 1 = tcgen05 kernel, 0 = CUDA-core kernel
  *   status_word device int32 (may be null): set to 1 if a bounded device-side wait expired
- * K must be a multiple of 8; A and W 16-byte aligned. */
+ *   A_lo (may be null) second half of a hi/lo activation pair, same shape as A: the product uses A + A_lo
+ *        (how the target's MLP and LM head carry their activations to about 16 significant bits)
+ *   out_lo (may be null; epilogues 0 and 1) receives bf16(x - bf16(x)) next to out = bf16(x)
+ * K must be a multiple of 8; A, A_lo and W 16-byte aligned. */
 int32_t sdd_debug_gemm_bf16(const void* A, int64_t a_rows_capacity, const void* W, const float* bias, int32_t M,
                             int32_t N, int32_t K, int32_t epilogue, void* out, int32_t ldc, int32_t n_tile,
-                            int32_t use_tensor_cores, int32_t* status_word, void* stream);
+                            int32_t use_tensor_cores, int32_t* status_word, void* stream, const void* A_lo,
+                            void* out_lo);
 
 /* Diagnostic: the library's bf16 tensor-core attention on its own (d_head = 64), as used inside both
  * networks' blocks: out = softmax(Q K^T / 8 [+ mask]) V per head.

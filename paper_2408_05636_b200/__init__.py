@@ -79,7 +79,7 @@ def lib() -> C.CDLL:
         L.sdd_accept_scratch_bytes.restype = u64
         L.sdd_accept_logits.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, u64, u64, vp, vp, vp, vp, vp]
         L.sdd_accept_logits_static.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, u64, u64, vp, vp, vp, vp]
-        L.sdd_debug_gemm_bf16.argtypes = [vp, C.c_int64, vp, vp, i32, i32, i32, i32, vp, i32, i32, i32, vp, vp]
+        L.sdd_debug_gemm_bf16.argtypes = [vp, C.c_int64, vp, vp, i32, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp]
         L.sdd_debug_attention_bf16.argtypes = [vp, C.c_int64, i32, i32, vp, C.c_int64, i32, i32, i32, vp, i32, vp, i32, vp,
                                                i32, i32, i32, i32, i32, vp, vp]
         L.sdd_tap.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(u64)]
@@ -195,15 +195,18 @@ def sdd_accept_logits_static(logits_p, logits_q, draft_ids, n_accept, out_ids, a
 
 
 def sdd_debug_gemm_bf16(A, W, bias, M: int, epilogue: int, out, n_tile: int = 0, use_tensor_cores: bool = True,
-                        status=None, stream=None):
-    """out = epilogue(A[:M] @ W.T + bias) with the library's bf16 GEMM; A [cap, K], W [N, K] bf16 CUDA tensors."""
+                        status=None, stream=None, A_lo=None, out_lo=None):
+    """out = epilogue((A[:M] + A_lo[:M]) @ W.T + bias) with the library's bf16 GEMM; A [cap, K], W [N, K] bf16 CUDA
+    tensors; out_lo (bf16 epilogues) receives the rounding remainder of out."""
     torch = _torch()
     cap, K = A.shape
     N = W.shape[0]
     st = stream if stream is not None else torch.cuda.current_stream(A.device)
     _check(lib().sdd_debug_gemm_bf16(A.data_ptr(), cap, W.data_ptr(), bias.data_ptr() if bias is not None else None, M, N,
                                      K, epilogue, out.data_ptr(), out.stride(0), n_tile, 1 if use_tensor_cores else 0,
-                                     status.data_ptr() if status is not None else None, st.cuda_stream),
+                                     status.data_ptr() if status is not None else None, st.cuda_stream,
+                                     A_lo.data_ptr() if A_lo is not None else None,
+                                     out_lo.data_ptr() if out_lo is not None else None),
            "sdd_debug_gemm_bf16")
 
 

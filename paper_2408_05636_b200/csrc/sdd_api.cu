@@ -676,13 +676,15 @@ int32_t sdd_accept_logits(const float* logits_p, const float* logits_q, const in
 
 int32_t sdd_debug_gemm_bf16(const void* A, int64_t a_rows_capacity, const void* W, const float* bias, int32_t M, int32_t N,
                             int32_t K, int32_t epilogue, void* out, int32_t ldc, int32_t n_tile, int32_t use_tensor_cores,
-                            int32_t* status_word, void* stream) {
+                            int32_t* status_word, void* stream, const void* A_lo, void* out_lo) {
   if (!A || !W || !out || M < 1 || N < 1 || K < 8 || (K % 8) != 0 || epilogue < 0 || epilogue > 3) return SDD_E_ARG;
   if (a_rows_capacity < M || ldc < N) return SDD_E_ARG;
+  if ((A_lo != nullptr || out_lo != nullptr) && !use_tensor_cores) return SDD_E_UNIMPL;
+  if (out_lo != nullptr && epilogue > 1) return SDD_E_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   if (use_tensor_cores)
     SDD_CUDA(launch_gemm_tc((const __nv_bfloat16*)A, a_rows_capacity, (const __nv_bfloat16*)W, bias, M, N, K, epilogue, out,
-                            ldc, n_tile, status_word, st));
+                            ldc, n_tile, status_word, st, nullptr, (const __nv_bfloat16*)A_lo, out_lo));
   else
     SDD_CUDA(launch_gemm_simt<__nv_bfloat16>((const __nv_bfloat16*)A, K, (const __nv_bfloat16*)W, bias, M, N, K, epilogue,
                                              out, ldc, st));

@@ -56,7 +56,22 @@ __device__ __forceinline__ float scalar_uniform(PhiloxKey key, uint32_t purpose,
   return word_to_uniform(philox4x32_10(0u, j, rnd, rng_c3(purpose, k, b), key).x);
 }
 
-__device__ __forceinline__ float gumbel_from_uniform(float u) { return -logf(-logf(u)); }
+// Gumbel variate -log(-log u) for u = odd multiple of 2^-24 in (0, 1), to about 2e-6 absolute.
+// The inner logarithm needs care next to u = 1, where the largest variates (the likely arg-max winners) come
+// from: there 1 - u is exact in fp32 and -log(1 - t) is summed as a series; elsewhere the hardware log2 does.
+__device__ __forceinline__ float gumbel_from_uniform(float u) {
+  const float t = 1.0f - u;
+  float ser = fmaf(t, 1.f / 9.f, 1.f / 8.f);
+  ser = fmaf(t, ser, 1.f / 7.f);
+  ser = fmaf(t, ser, 1.f / 6.f);
+  ser = fmaf(t, ser, 1.f / 5.f);
+  ser = fmaf(t, ser, 1.f / 4.f);
+  ser = fmaf(t, ser, 1.f / 3.f);
+  ser = fmaf(t, ser, 1.f / 2.f);
+  ser = fmaf(t, ser, 1.f);
+  const float y = t < 0.125f ? t * ser : -__logf(u);
+  return -__logf(y);
+}
 
 // ---------------------------------------------------------------------------------------------
 // reductions

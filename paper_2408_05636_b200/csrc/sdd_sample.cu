@@ -325,7 +325,7 @@ unmask_sample_kernel(const float* __restrict__ step_logits,  // [B, gamma, V]
 // = 1 when the rows were stored already divided by the temperature).  log q(x) comes either from
 // `logq_in` (round pipeline) or from the q-row partial statistics (stand-alone call).
 // ---------------------------------------------------------------------------------------------
-constexpr int ACCEPT_THREADS = 512;
+constexpr int ACCEPT_THREADS = 256;
 
 __global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(ACCEPT_THREADS)
 accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_rows, const int* __restrict__ draft_ids,
@@ -422,28 +422,47 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
     }
     const uint32_t c3 = rng_c3(resid ? RNG_RESID : RNG_BONUS, 0u, (uint32_t)b);
     const int nblk = (V + 3) >> 2;
-    for (int blk = rank * ACCEPT_THREADS + threadIdx.x; blk < nblk; blk += VC * ACCEPT_THREADS) {
-      const uint4 w = philox4x32_10((uint32_t)blk, (uint32_t)n, rnd, c3, key);
-      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+    // two blocks of four entries per iteration, with all loads of the iteration issued before any arithmetic
+    constexpr int UNR = 2;
+    for (int blk0 = rank * ACCEPT_THREADS + threadIdx.x; blk0 < nblk; blk0 += UNR * VC * ACCEPT_THREADS) {
+      float xp[UNR][4], xq[UNR][4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int v = blk * 4 + c;
-        if (v < V) {
-          const float g = gumbel_from_uniform(word_to_uniform(ww[c]));
-          const float zp = prow[v] * inv_tau_p - lsep;   // log p_v
-          ArgMax cand;
-          cand.i = v;
-          cand.s = zp + g;
-          if (resid) {
-            fallback = argmax_better(fallback, cand);    // a draw from p itself, if max(0, p - q) == 0 everywhere
-            const float zq = qrow[v] * inv_tau_q_rows - lseq;
-            const float wv = expf(zp) - expf(zq);
-            if (wv > 0.f) {
-              cand.s = logf(wv) + g;
+      for (int u = 0; u < UNR; ++u) {
+        const int blk = blk0 + u * VC * ACCEPT_THREADS;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int v = blk * 4 + c;
+          const bool in = blk < nblk && v < V;
+          xp[u][c] = in ? __ldg(prow + v) : 0.f;
+          xq[u][c] = (in && resid) ? __ldg(qrow + v) : 0.f;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < UNR; ++u) {
+        const int blk = blk0 + u * VC * ACCEPT_THREADS;
+        if (blk >= nblk) break;
+        const uint4 w = philox4x32_10((uint32_t)blk, (uint32_t)n, rnd, c3, key);
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int v = blk * 4 + c;
+          if (v < V) {
+            const float g = gumbel_from_uniform(word_to_uniform(ww[c]));
+            const float zp = xp[u][c] * inv_tau_p - lsep;   // log p_v
+            ArgMax cand;
+            cand.i = v;
+            cand.s = zp + g;
+            if (resid) {
+              fallback = argmax_better(fallback, cand);    // a draw from p itself, if max(0, p - q) == 0 everywhere
+              const float zq = xq[u][c] * inv_tau_q_rows - lseq;
+              const float wv = __expf(zp) - __expf(zq);
+              if (wv > 0.f) {
+                cand.s = __logf(wv) + g;
+                best = argmax_better(best, cand);
+              }
+            } else {
               best = argmax_better(best, cand);
             }
-          } else {
-            best = argmax_better(best, cand);
           }
         }
       }

@@ -72,3 +72,34 @@ def test_simt_and_tc_agree():
     sdd.sdd_debug_gemm_bf16(A, W, None, 200, 3, o2, 0, False)
     torch.cuda.synchronize()
     assert (o1 - o2).abs().max().item() < 1e-3
+
+
+@pytest.mark.parametrize("M,N,K", [(17, 768, 3072), (33, 3072, 768), (300, 512, 256), (1000, 1024, 512)])
+def test_hi_lo_activation_pairs(M, N, K):
+    """A given as hi + lo bf16 halves: the product must match the fp32 matmul of the un-split activations far more
+    closely than a single bf16 rounding allows; the GELU epilogue's (out, out_lo) pair likewise."""
+    import paper_2408_05636_b200 as sdd
+    g = torch.Generator(device="cuda").manual_seed(M + N)
+    x = torch.randn(M + 5, K, device="cuda", generator=g)
+    hi = x.to(torch.bfloat16)
+    lo = (x - hi.float()).to(torch.bfloat16)
+    W = (torch.randn(N, K, device="cuda", generator=g) * 0.05).to(torch.bfloat16)
+    bias = torch.randn(N, device="cuda", generator=g)
+    ref = x[:M] @ W.float().t() + bias
+    out = torch.zeros(M, N, device="cuda")
+    sdd.sdd_debug_gemm_bf16(hi, W, bias, M, 3, out, 0, True, None, None, lo)
+    single = torch.zeros(M, N, device="cuda")
+    sdd.sdd_debug_gemm_bf16(hi, W, bias, M, 3, single)
+    torch.cuda.synchronize()
+    err_pair = (out - ref).abs().max().item()
+    err_single = (single - ref).abs().max().item()
+    assert err_pair < 2e-4 * max(1.0, ref.abs().max().item()) and err_pair < err_single / 20
+    # GELU epilogue writing a hi/lo pair
+    o_hi = torch.zeros(M, N, device="cuda", dtype=torch.bfloat16)
+    o_lo = torch.zeros(M, N, device="cuda", dtype=torch.bfloat16)
+    sdd.sdd_debug_gemm_bf16(hi, W, bias, M, 1, o_hi, 0, True, None, None, lo, o_lo)
+    torch.cuda.synchronize()
+    gref = torch.nn.functional.gelu(ref, approximate="tanh")
+    pair = o_hi.float() + o_lo.float()
+    assert (pair - gref).abs().max().item() < 2e-3 * max(1.0, gref.abs().max().item())     # hardware tanh ~ 2^-11
+    assert (pair - gref).abs().max().item() <= (o_hi.float() - gref).abs().max().item()
