@@ -131,7 +131,11 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(device))
     peaks = load_peaks()
-    wl = synth.WORKLOADS[WORKLOAD]
+    wl = synth.WORKLOADS[args.workload]
+    if args.gamma or args.T:
+        wl = synth.scaled_workload(wl, gamma=args.gamma or wl.gamma, T=args.T or wl.T)
+    if args.workload != WORKLOAD and not args.rounds_only:
+        raise SystemExit("other workloads than the headline one are timed with --rounds-only")
     wp, wq, dp, dq = make_models(wl, device)
     V = wl.target.vocab
 
@@ -140,22 +144,24 @@ def run_ours(args):
     def new_session():
         seed = wl.prompt_seed + 1000 * rank + gen_idx[0]
         gen_idx[0] += 1
-        prompts = synth.prompt_ids(V, 1, wl.prompt_len, seed)
-        s = sdd.Session(dp, dq, prompts, [wl.prompt_len], wl.gamma, wl.T, wl.max_new, 1.0, 1.0,
+        prompts = synth.prompt_ids(V, wl.batch, wl.prompt_len, seed)
+        s = sdd.Session(dp, dq, prompts, [wl.prompt_len] * wl.batch, wl.gamma, wl.T, wl.max_new, 1.0, 1.0,
                         wl.philox_seed + gen_idx[0], device)
         s.sdd_sync_status()
         return s
 
     def emitted(s):
-        return int(s.tap_numpy(sdd.TAP_N_EMITTED)[0])
+        """(total, minimum over the batch) of the tokens generated so far"""
+        e = s.tap_numpy(sdd.TAP_N_EMITTED)
+        return int(e.sum()), int(e.min())
 
     def run_rounds(n, timed):
         """Runs n rounds (across generations if needed).  Returns (device ms, tokens, launches)."""
         nonlocal sess
         ms_total, tok_total, launch_total, left = 0.0, 0, 0, n
         while left > 0:
-            e0 = emitted(sess)
-            if e0 >= wl.max_new:
+            e0, emin = emitted(sess)
+            if emin >= wl.max_new:
                 sess.close()
                 sess = new_session()
                 e0 = 0
@@ -177,7 +183,7 @@ def run_ours(args):
             _, l1 = sess.sdd_counters()
             # rounds enqueued after the generation completed emit nothing but still ran: they are counted
             ms_total += ev0.elapsed_time(ev1)
-            tok_total += emitted(sess) - e0
+            tok_total += emitted(sess)[0] - e0
             launch_total += l1 - l0
             left -= done
         return ms_total, tok_total, launch_total
@@ -210,7 +216,8 @@ def run_ours(args):
             dist.destroy_process_group()
         return
     if args.rounds_only:
-        print(json.dumps({"metric": METRIC, "value": round(value, 2), "unit": UNIT, "steps": args.steps,
+        print(json.dumps({"metric": METRIC, "workload": wl.name, "batch": wl.batch, "gamma": wl.gamma, "T": wl.T,
+                          "value": round(value, 2), "unit": UNIT, "steps": args.steps,
                           "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4), "gpu_launches": int(launches),
                           "note": "rounds only"}))
         return
@@ -225,7 +232,7 @@ def run_ours(args):
     cat_work = {n: 0.0 for n in sdd.PROF_NAMES}
     kinds = {}
     for _ in range(prof_rounds):
-        if emitted(sess) >= wl.max_new:
+        if emitted(sess)[1] >= wl.max_new:
             sess.close()
             sess = new_session()
         c = int(sess.tap_numpy(sdd.TAP_CTX_LEN)[0])
@@ -398,6 +405,10 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=WORKLOAD, choices=sorted(synth.WORKLOADS),
+                    help="with --rounds-only: time another configuration (default: the headline one)")
+    ap.add_argument("--gamma", type=int, default=0)
+    ap.add_argument("--T", type=int, default=0)
     ap.add_argument("--rounds-only", action="store_true",
                     help="run only the warm-up and timed rounds and print a short line (for profiler captures)")
     args = ap.parse_args()

@@ -172,6 +172,7 @@ struct sdd_ctx {
   int runahead;
   int lcap;                    // padded rows per sequence of the current round's drafter forwards
   size_t act_elems, xf_elems;  // capacity (elements) of the xn / att buffers (mlp: 4x) and of xf
+  bool cache_skip;             // SDD_CACHE_SKIP != 0 (default): skip drafter evaluations whose input did not change
   bool hilo;                   // SDD_HILO != 0 (default): hi/lo activation pairs in the target's MLP and LM head
   bool force_simt;             // SDD_GEMM=simt: run bf16 GEMMs on the CUDA-core kernel (cross-check)
   int bn_hint;                 // SDD_GEMM_BN: N tile of the tensor-core GEMM (0 = choose)
@@ -241,15 +242,15 @@ static void fill_dims(const Net& P, const Net& Q, const sdd_params* p, int max_p
 template <typename T>
 static int gemm(sdd_ctx* c, int cat, const void* A, size_t a_elems, const void* W, const float* bias, long long M, int N,
                 int K, int epi, void* out, int ldc, const QkvDst* qd = nullptr, const void* A_lo = nullptr,
-                void* out_lo = nullptr) {
+                void* out_lo = nullptr, const int* skip = nullptr) {
   if (M <= 0) return SDD_OK;
   ProfScope prof(c, cat);
   c->launches++;
   if (std::is_same<T, __nv_bfloat16>::value && !c->force_simt) {
     SDD_CUDA(launch_gemm_tc((const __nv_bfloat16*)A, (long long)(a_elems / (size_t)K), (const __nv_bfloat16*)W, bias, (int)M,
-                            N, K, epi, out, ldc, c->bn_hint, &c->B.rs->status, c->st, qd, (const __nv_bfloat16*)A_lo, out_lo));
+                            N, K, epi, out, ldc, c->bn_hint, &c->B.rs->status, c->st, qd, (const __nv_bfloat16*)A_lo, out_lo, skip));
   } else {
-    SDD_CUDA(launch_gemm_simt<T>((const T*)A, K, (const T*)W, bias, (int)M, N, K, epi, out, ldc, c->st));
+    SDD_CUDA(launch_gemm_simt<T>((const T*)A, K, (const T*)W, bias, (int)M, N, K, epi, out, ldc, c->st, skip));
   }
   return SDD_OK;
 }
@@ -269,25 +270,27 @@ static bool use_tc(const sdd_ctx* c, const Net& N) {
 
 // one transformer block on `rows` rows; attention is issued by the caller-supplied functor
 template <typename T, typename QkvFn, typename AttnFn>
-static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, bool hilo_mlp, QkvFn qkv_dst, AttnFn attn) {
+static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, bool hilo_mlp, const int* skip, QkvFn qkv_dst,
+                      AttnFn attn) {
   const Buffers& B = c->B;
   const int d = N.d;
   for (int l = 0; l < N.n_layer; ++l) {
     const Layer& L = N.layers[l];
-    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln1_g, L.ln1_b, (T*)B.xn, rows, d, c->st));
+    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln1_g, L.ln1_b, (T*)B.xn, rows, d, c->st, nullptr, skip));
     QkvDst qd = {};
     const bool fused = qkv_dst(l, &qd);
     SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_qkv, L.b_qkv, rows, 3 * d, d, fused ? EPI_QKV : EPI_STORE, B.qkv,
-                    3 * d, fused ? &qd : nullptr));
+                    3 * d, fused ? &qd : nullptr, nullptr, nullptr, skip));
     SDD_TRY(attn(l));
-    SDD_TRY(gemm<T>(c, gcat, B.att, c->act_elems, L.w_o, L.b_o, rows, d, d, EPI_RESIDUAL, B.h, d));
+    SDD_TRY(gemm<T>(c, gcat, B.att, c->act_elems, L.w_o, L.b_o, rows, d, d, EPI_RESIDUAL, B.h, d, nullptr, nullptr, nullptr, skip));
     // hilo_mlp: the MLP's two products take their activations as hi/lo bf16 pairs (see sdd_gemm_tc.cu)
     T* xn_lo = hilo_mlp ? (T*)B.xn_lo : nullptr;
     void* mlp_lo = hilo_mlp ? B.mlp_lo : nullptr;
-    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln2_g, L.ln2_b, (T*)B.xn, rows, d, c->st, xn_lo));
+    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln2_g, L.ln2_b, (T*)B.xn, rows, d, c->st, xn_lo, skip));
     SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_fc1, L.b_fc1, rows, 4 * d, d, EPI_GELU, B.mlp, 4 * d, nullptr, xn_lo,
-                    mlp_lo));
-    SDD_TRY(gemm<T>(c, gcat, B.mlp, 4 * c->act_elems, L.w_fc2, L.b_fc2, rows, d, 4 * d, EPI_RESIDUAL, B.h, d, nullptr, mlp_lo));
+                    mlp_lo, skip));
+    SDD_TRY(gemm<T>(c, gcat, B.mlp, 4 * c->act_elems, L.w_fc2, L.b_fc2, rows, d, 4 * d, EPI_RESIDUAL, B.h, d, nullptr, mlp_lo, nullptr,
+                    skip));
   }
   return SDD_OK;
 }
@@ -300,10 +303,12 @@ static int forward_drafter(sdd_ctx* c) {
   const Dims& D = c->D;
   const int lcap = c->lcap;
   const long long rows = (long long)D.batch * lcap;
+  // every kernel of the evaluation returns at once when the previous step revealed nothing (RoundState.skip_forward)
+  const int* skip = &B.rs->skip_forward;
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_drafter<T>((const T*)Q.wte, (const T*)Q.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
-                                        D.batch, D.gamma, lcap, Q.d, B.h, c->st));
+                                        D.batch, D.gamma, lcap, Q.d, B.h, c->st, skip));
   const bool tc = use_tc<T>(c, Q);
-  SDD_TRY((run_blocks<T>(c, Q, rows, CAT_GEMM_Q, false,
+  SDD_TRY((run_blocks<T>(c, Q, rows, CAT_GEMM_Q, false, skip,
     [&](int, QkvDst* qd) -> bool {
       if (!tc) return false;
       qd->k_dst = nullptr; qd->vt_dst = (__nv_bfloat16*)B.vt; qd->ctx_len = B.ctx_len; qd->rows_per_seq = lcap;
@@ -316,15 +321,17 @@ static int forward_drafter(sdd_ctx* c) {
         SDD_LAUNCH(c, CAT_ATTN_Q, launch_attn_tc(qkv, (long long)(c->act_elems / Q.d), 3 * Q.d, 0, qkv,
                                                  (long long)(c->act_elems / Q.d), 3 * Q.d, Q.d, lcap,
                                                  (const __nv_bfloat16*)B.vt, D.lcap_max, (__nv_bfloat16*)B.att, Q.d, B.ctx_len,
-                                                 D.batch, Q.n_head, Q.d, D.gamma, 0, lcap, &B.rs->status, c->st));
+                                                 D.batch, Q.n_head, Q.d, D.gamma, 0, lcap, &B.rs->status, c->st, skip));
       } else {
         SDD_LAUNCH(c, CAT_ATTN_Q, launch_attn_bidir<T>((const T*)B.qkv, (T*)B.att, B.ctx_len, D.batch, D.gamma, lcap, Q.n_head,
-                                                       Q.d_head, c->st));
+                                                       Q.d_head, c->st, skip));
       }
       return SDD_OK;
     })));
-  SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm_slots<T>(B.h, Q.lnf_g, Q.lnf_b, (T*)B.xf, B.ctx_len, D.batch, D.gamma, lcap, Q.d, c->st));
-  SDD_TRY(gemm<T>(c, CAT_HEAD_Q, B.xf, c->xf_elems, Q.wte, nullptr, (long long)D.batch * D.gamma, D.V, Q.d, EPI_STORE_F32, B.step_logits, D.V));
+  SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm_slots<T>(B.h, Q.lnf_g, Q.lnf_b, (T*)B.xf, B.ctx_len, D.batch, D.gamma, lcap, Q.d, c->st,
+                                                         skip));
+  SDD_TRY(gemm<T>(c, CAT_HEAD_Q, B.xf, c->xf_elems, Q.wte, nullptr, (long long)D.batch * D.gamma, D.V, Q.d, EPI_STORE_F32, B.step_logits, D.V,
+                  nullptr, nullptr, nullptr, skip));
   return SDD_OK;
 }
 
@@ -342,7 +349,7 @@ static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) 
   const bool tc = use_tc<T>(c, P);
   // tensor-core path: per layer the cache is K [B][n_ctx][d] followed by V^T [B][d][n_ctx];
   // CUDA-core path: [B][n_ctx][K|V][d]
-  SDD_TRY((run_blocks<T>(c, P, rows, CAT_GEMM_P, tc && c->hilo,
+  SDD_TRY((run_blocks<T>(c, P, rows, CAT_GEMM_P, tc && c->hilo, nullptr,
     [&](int l, QkvDst* qd) -> bool {
       if (!tc) return false;
       __nv_bfloat16* kc = (__nv_bfloat16*)B.kv + (size_t)l * layer_elems;
@@ -410,7 +417,7 @@ static int draft_step_t(sdd_ctx* c) {
   const int k = D.T - c->steps_done;
   SDD_TRY(forward_drafter<T>(c));
   SDD_LAUNCH(c, CAT_SAMPLE, launch_unmask_sample(B.step_logits, B.slot_ids, B.q_logits, B.logq, B.reveal_step, D.batch, D.gamma, D.V, k,
-                                     c->inv_tau_q, c->key, B.rs, c->st));
+                                     c->inv_tau_q, c->key, B.rs, c->cache_skip ? 1 : 0, c->st));
   c->steps_done++;
   return SDD_OK;
 }
@@ -486,6 +493,8 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
     c->xf_elems = (size_t)params->batch * (params->gamma + 1) * (c->Q.d > c->P.d ? c->Q.d : c->P.d);
     const char* g = getenv("SDD_GEMM");
     c->force_simt = g != nullptr && strcmp(g, "simt") == 0;
+    const char* cs = getenv("SDD_CACHE_SKIP");
+    c->cache_skip = cs == nullptr || atoi(cs) != 0;
     const char* hl = getenv("SDD_HILO");
     c->hilo = hl == nullptr || atoi(hl) != 0;
     const char* bn = getenv("SDD_GEMM_BN");
@@ -545,7 +554,7 @@ static int round_prologue(sdd_ctx* c) {
   return SDD_OK;
 }
 static int enqueue_draft_begin(sdd_ctx* c) {
-  SDD_LAUNCH(c, CAT_GLUE, launch_reset_slots(c->B.slot_ids, c->B.reveal_step, c->D.batch * c->D.gamma, c->D.V, c->st));
+  SDD_LAUNCH(c, CAT_GLUE, launch_reset_slots(c->B.slot_ids, c->B.reveal_step, c->D.batch * c->D.gamma, c->D.V, c->B.rs, c->st));
   c->steps_done = 0;
   return SDD_OK;
 }

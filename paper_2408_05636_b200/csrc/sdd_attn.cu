@@ -54,8 +54,9 @@ __device__ __forceinline__ void attn_one_query(const T* __restrict__ q, const T*
 template <typename T, int DH>
 __global__ void __launch_bounds__(128)
 attn_bidir_kernel(const T* __restrict__ qkv, T* __restrict__ out, const int* __restrict__ ctx_len, int gamma, int L_cap,
-                  int n_head) {
+                  int n_head, const int* __restrict__ skip) {
   pdl_wait();
+  if (skip != nullptr && *skip) return;
   const int i = blockIdx.x * 4 + (threadIdx.x >> 5), h = blockIdx.y, b = blockIdx.z;
   if (i >= L_cap) return;
   const int d = n_head * DH;
@@ -95,10 +96,10 @@ attn_cached_kernel(const T* __restrict__ qkv, const T* __restrict__ cache, T* __
 
 template <typename T>
 cudaError_t launch_attn_bidir(const T* qkv, T* out, const int* ctx_len, int batch, int gamma, int L_cap, int n_head,
-                              int d_head, cudaStream_t st) {
+                              int d_head, cudaStream_t st, const int* skip) {
   dim3 grid((L_cap + 3) / 4, n_head, batch);
-  if (d_head == 64) launch_k(attn_bidir_kernel<T, 64>, dim3(grid), dim3(128), 0, st, qkv, out, ctx_len, gamma, L_cap, n_head);
-  else if (d_head == 32) launch_k(attn_bidir_kernel<T, 32>, dim3(grid), dim3(128), 0, st, qkv, out, ctx_len, gamma, L_cap, n_head);
+  if (d_head == 64) launch_k(attn_bidir_kernel<T, 64>, dim3(grid), dim3(128), 0, st, qkv, out, ctx_len, gamma, L_cap, n_head, skip);
+  else if (d_head == 32) launch_k(attn_bidir_kernel<T, 32>, dim3(grid), dim3(128), 0, st, qkv, out, ctx_len, gamma, L_cap, n_head, skip);
   else return cudaErrorInvalidValue;
   return cudaGetLastError();
 }
@@ -117,7 +118,8 @@ cudaError_t launch_attn_cached(const T* qkv, const T* cache, T* out, const int* 
 }
 
 #define SDD_INSTANTIATE_ATTN(T)                                                                                  \
-  template cudaError_t launch_attn_bidir<T>(const T*, T*, const int*, int, int, int, int, int, cudaStream_t);   \
+  template cudaError_t launch_attn_bidir<T>(const T*, T*, const int*, int, int, int, int, int, cudaStream_t,   \
+                                            const int*);                                                       \
   template cudaError_t launch_attn_cached<T>(const T*, const T*, T*, const int*, int, int, int, int, int, int, \
                                              cudaStream_t);
 SDD_INSTANTIATE_ATTN(float)

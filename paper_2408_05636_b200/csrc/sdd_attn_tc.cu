@@ -31,6 +31,12 @@ constexpr int AT_BAR_OFF = AT_Q_BYTES + AT_P_BYTES + AT_KV_STAGES * AT_STAGE_BYT
 constexpr int AT_SMEM = AT_BAR_OFF + 1024 + 256;
 constexpr uint32_t AT_TMEM_COLS = 256;              // S: columns 0..127, PV: columns 128..191
 
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 struct AttnParams {
   __nv_bfloat16* out;
   int ld_out;
@@ -42,6 +48,7 @@ struct AttnParams {
   int q_col0, k_col0;   // column of head 0 in the Q / K tensors
   int d;                // model width = rows of one sequence in the V^T tensor
   int* status;
+  const int* skip;      // may be null; *skip != 0: return at once (skipped drafter evaluation)
 };
 
 __global__ void __launch_bounds__(AT_THREADS)
@@ -49,6 +56,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                const __grid_constant__ CUtensorMap map_vt, const AttnParams prm) {
   const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   pdl_wait();   // ctx_len and Q / K / V^T come from earlier kernels
+  if (prm.skip != nullptr && *prm.skip) return;
   const int c = prm.ctx_len[b];
   const int q0 = qt * 128;
   int n_valid_q;
@@ -167,18 +175,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (!ok) break;
       fence_after_sync();
       const int key0 = t * 128;
+      // rows that see the whole tile (every tile but the last one, or the diagonal one under the causal mask)
+      // skip the per-entry visibility test
+      const bool full = key0 + 128 <= key_limit;
       float mx = -INFINITY;
 #pragma unroll 1
       for (int cc = 0; cc < 4; ++cc) {
         uint32_t v[32];
         tmem_ld32(t_lane + (uint32_t)(cc * 32), v);
+        if (full) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (key0 + cc * 32 + j < key_limit) mx = fmaxf(mx, __uint_as_float(v[j]));
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (key0 + cc * 32 + j < key_limit) mx = fmaxf(mx, __uint_as_float(v[j]));
+        }
       }
       const float m_new = fmaxf(m, mx * scale);
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
-      const float corr = m == -INFINITY ? 0.f : exp2f(m - m_use);
+      const float corr = m == -INFINITY ? 0.f : ex2(m - m_use);
       float sum = 0.f;
 #pragma unroll 1
       for (int cc = 0; cc < 4; ++cc) {
@@ -191,8 +207,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int j0 = g * 8 + 2 * e;
-            const float p0 = (key0 + cc * 32 + j0 < key_limit) ? exp2f(fmaf(__uint_as_float(v[j0]), scale, -m_use)) : 0.f;
-            const float p1 = (key0 + cc * 32 + j0 + 1 < key_limit) ? exp2f(fmaf(__uint_as_float(v[j0 + 1]), scale, -m_use)) : 0.f;
+            float p0 = ex2(fmaf(__uint_as_float(v[j0]), scale, -m_use));
+            float p1 = ex2(fmaf(__uint_as_float(v[j0 + 1]), scale, -m_use));
+            if (!full) {
+              if (!(key0 + cc * 32 + j0 < key_limit)) p0 = 0.f;
+              if (!(key0 + cc * 32 + j0 + 1 < key_limit)) p1 = 0.f;
+            }
             sum += p0 + p1;
             __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
             pk[e] = *reinterpret_cast<uint32_t*>(&h2);
@@ -248,7 +268,7 @@ cudaError_t tc_prepare_attn() {
 cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q_ld, int q_col0, const __nv_bfloat16* k,
                            long long k_rows_total, int k_ld, int k_col0, int k_rows_per_seq, const __nv_bfloat16* vt,
                            int vt_ld, __nv_bfloat16* out, int ld_out, const int* ctx_len, int batch, int n_head, int d,
-                           int gamma, int mode, int q_rows_per_seq, int* status, cudaStream_t st) {
+                           int gamma, int mode, int q_rows_per_seq, int* status, cudaStream_t st, const int* skip) {
   using namespace tc;
   if (q_rows_per_seq <= 0) return cudaSuccess;
   if (d != n_head * AT_DH || (ld_out & 7) != 0) return cudaErrorInvalidValue;
@@ -264,7 +284,7 @@ cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q
   AttnParams p;
   p.out = out; p.ld_out = ld_out; p.ctx_len = ctx_len; p.mode = mode; p.gamma = gamma;
   p.q_rows_per_seq = q_rows_per_seq; p.k_rows_per_seq = k_rows_per_seq; p.q_col0 = q_col0; p.k_col0 = k_col0;
-  p.d = d; p.status = status;
+  p.d = d; p.status = status; p.skip = skip;
   dim3 grid((q_rows_per_seq + 127) / 128, n_head, batch);
   launch_k(attn_tc_kernel, dim3(grid), dim3(AT_THREADS), AT_SMEM, st, mq, mk, mv, p);
   return cudaGetLastError();

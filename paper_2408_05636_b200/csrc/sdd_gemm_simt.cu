@@ -10,8 +10,9 @@ constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16, SG_THREADS = 256;
 template <typename T>
 __global__ void __launch_bounds__(SG_THREADS)
 gemm_simt_kernel(const T* __restrict__ A, int lda, const T* __restrict__ W, const float* __restrict__ bias, int M, int N,
-                 int K, int epi, void* __restrict__ out, int ldc) {
+                 int K, int epi, void* __restrict__ out, int ldc, const int* __restrict__ skip) {
   pdl_wait();
+  if (skip != nullptr && *skip) return;
   __shared__ float As[SG_BK][SG_BM + 4];
   __shared__ float Ws[SG_BK][SG_BN + 4];
   const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
@@ -59,16 +60,16 @@ gemm_simt_kernel(const T* __restrict__ A, int lda, const T* __restrict__ W, cons
 
 template <typename T>
 cudaError_t launch_gemm_simt(const T* A, int lda, const T* W, const float* bias, int M, int N, int K, int epi, void* out,
-                             int ldc, cudaStream_t st) {
+                             int ldc, cudaStream_t st, const int* skip) {
   if (M <= 0 || N <= 0) return cudaSuccess;
   dim3 grid((N + SG_BN - 1) / SG_BN, (M + SG_BM - 1) / SG_BM);
-  launch_k(gemm_simt_kernel<T>, dim3(grid), dim3(SG_THREADS), 0, st, A, lda, W, bias, M, N, K, epi, out, ldc);
+  launch_k(gemm_simt_kernel<T>, dim3(grid), dim3(SG_THREADS), 0, st, A, lda, W, bias, M, N, K, epi, out, ldc, skip);
   return cudaGetLastError();
 }
 
 template cudaError_t launch_gemm_simt<float>(const float*, int, const float*, const float*, int, int, int, int, void*, int,
-                                             cudaStream_t);
+                                             cudaStream_t, const int*);
 template cudaError_t launch_gemm_simt<__nv_bfloat16>(const __nv_bfloat16*, int, const __nv_bfloat16*, const float*, int,
-                                                     int, int, int, void*, int, cudaStream_t);
+                                                     int, int, int, void*, int, cudaStream_t, const int*);
 
 }  // namespace sdd

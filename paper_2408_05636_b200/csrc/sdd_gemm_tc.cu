@@ -58,7 +58,11 @@ __global__ void __launch_bounds__(THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_out, int tma_out,
                int rows_a, int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out,
-               void* __restrict__ out_lo, int ldc, int* status, const QkvDst qd) {
+               void* __restrict__ out_lo, int ldc, int* status, const QkvDst qd, const int* __restrict__ skip) {
+  if (skip != nullptr) {   // launches of a drafter evaluation: nothing to do if the evaluation is skipped
+    pdl_wait();
+    if (*skip) return;
+  }
   constexpr int STAGES = ring_stages<BN, SWAP, HILO>();
   constexpr int STAGE_BYTES = stage_bytes<BN, SWAP, HILO>();
   constexpr int LO_OFF = BM * BK * 2 + BN * BK * 2;     // offset of the lo tile inside a stage
@@ -369,19 +373,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 template <int BN, bool SWAP, bool HILO>
 static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& mo,
                               int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias, void* out, void* out_lo,
-                              int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits) {
+                              int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits, const int* skip) {
   dim3 grid((rows_b + BN - 1) / BN, (rows_a + BM - 1) / BM, splits);
   launch_k(gemm_tc_kernel<BN, SWAP, HILO>, grid, dim3(THREADS), smem_bytes<BN, SWAP, HILO>(), st, ma, mb, ml, mo, tma_out,
-           rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd);
+           rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip);
   return cudaGetLastError();
 }
 template <int BN, bool SWAP>
 static cudaError_t launch_hl(bool hilo, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml,
                              const CUtensorMap& mo, int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias,
-                             void* out, void* out_lo, int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits) {
+                             void* out, void* out_lo, int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits,
+                             const int* skip) {
   if (hilo)
-    return launch_cfg<BN, SWAP, true>(ma, mb, ml, mo, tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
-  return launch_cfg<BN, SWAP, false>(ma, mb, ml, mo, tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
+    return launch_cfg<BN, SWAP, true>(ma, mb, ml, mo, tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
+  return launch_cfg<BN, SWAP, false>(ma, mb, ml, mo, tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
 }
 
 template <int BN, bool SWAP>
@@ -446,7 +451,7 @@ cudaError_t get_tensor_map(const void* ptr, long long rows, long long cols, long
 // A: activations [M rows used, capacity a_cap rows, K], W: weights [N, K]; both dense bf16.
 cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_bfloat16* W, const float* bias, int M, int N,
                            int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st, const QkvDst* qkv,
-                           const __nv_bfloat16* A_lo, void* out_lo) {
+                           const __nv_bfloat16* A_lo, void* out_lo, const int* skip) {
   using namespace tc;
   if (M <= 0 || N <= 0) return cudaSuccess;
   static std::once_flag once;
@@ -482,8 +487,8 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     if ((e = get_tensor_map(A, a_cap, K, K, bn, BK, &mb)) != cudaSuccess) return e;
     ml = mb;
     if (hilo && (e = get_tensor_map(A_lo, a_cap, K, K, bn, BK, &ml)) != cudaSuccess) return e;
-    if (bn == 32) return launch_hl<32, true>(hilo, ma, mb, ml, ma, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
-    return launch_hl<64, true>(hilo, ma, mb, ml, ma, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
+    if (bn == 32) return launch_hl<32, true>(hilo, ma, mb, ml, ma, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
+    return launch_hl<64, true>(hilo, ma, mb, ml, ma, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
   }
   int bn = bn_hint;
   const long long mt = (M + BM - 1) / BM;
@@ -511,10 +516,10 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     tma_out = 1;
   }
   switch (bn) {
-    case 256: return launch_hl<256, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
-    case 128: return launch_hl<128, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
-    case 64: return launch_hl<64, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
-    default: return launch_hl<32, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits);
+    case 256: return launch_hl<256, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
+    case 128: return launch_hl<128, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
+    case 64: return launch_hl<64, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
+    default: return launch_hl<32, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
   }
 }
 

@@ -11,8 +11,9 @@ namespace sdd {
 template <typename T>
 __global__ void embed_drafter_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
                                      int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
-                                     int gamma, int L_cap, int d, float* __restrict__ h) {
+                                     int gamma, int L_cap, int d, float* __restrict__ h, const int* __restrict__ skip) {
   pdl_wait();
+  if (skip != nullptr && *skip) return;
   const int i = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
   float* __restrict__ dst = h + ((long long)b * L_cap + i) * d;
@@ -96,8 +97,9 @@ __device__ __forceinline__ void layernorm_row(const float* __restrict__ src, con
 template <typename T>
 __global__ void __launch_bounds__(128)
 layernorm_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
-                 T* __restrict__ out, T* __restrict__ out_lo, long long rows, int d) {
+                 T* __restrict__ out, T* __restrict__ out_lo, long long rows, int d, const int* __restrict__ skip) {
   pdl_wait();
+  if (skip != nullptr && *skip) return;
   const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
   if (row >= rows) return;
   layernorm_row<T>(h + row * d, g, bta, out + row * d, out_lo != nullptr ? out_lo + row * d : nullptr, d);
@@ -106,8 +108,10 @@ layernorm_kernel(const float* __restrict__ h, const float* __restrict__ g, const
 template <typename T>
 __global__ void __launch_bounds__(128)
 layernorm_slots_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
-                       T* __restrict__ out, const int* __restrict__ ctx_len, int batch, int gamma, int L_cap, int d) {
+                       T* __restrict__ out, const int* __restrict__ ctx_len, int batch, int gamma, int L_cap, int d,
+                       const int* __restrict__ skip) {
   pdl_wait();
+  if (skip != nullptr && *skip) return;
   const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
   if (r >= batch * gamma) return;
   const int b = r / gamma, j = r - b * gamma;
@@ -137,9 +141,10 @@ __global__ void kv_append_kernel(const T* __restrict__ qkv, T* __restrict__ cach
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 cudaError_t launch_embed_drafter(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
-                                 const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st) {
+                                 const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st,
+                                 const int* skip) {
   launch_k(embed_drafter_kernel<T>, dim3(dim3(L_cap, batch)), dim3(128), 0, st, wte, wpe, tokens, tok_stride, ctx_len, slot_ids, gamma,
-                                                              L_cap, d, h);
+                                                              L_cap, d, h, skip);
   return cudaGetLastError();
 }
 template <typename T>
@@ -153,17 +158,17 @@ cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, i
 }
 template <typename T>
 cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* out, long long rows, int d,
-                             cudaStream_t st, T* out_lo) {
+                             cudaStream_t st, T* out_lo, const int* skip) {
   if (rows <= 0) return cudaSuccess;
   if (d > LN_MAX_PER_LANE * 32) return cudaErrorInvalidValue;
-  launch_k(layernorm_kernel<T>, dim3((unsigned)((rows + 3) / 4)), dim3(128), 0, st, h, g, b, out, out_lo, rows, d);
+  launch_k(layernorm_kernel<T>, dim3((unsigned)((rows + 3) / 4)), dim3(128), 0, st, h, g, b, out, out_lo, rows, d, skip);
   return cudaGetLastError();
 }
 template <typename T>
 cudaError_t launch_layernorm_slots(const float* h, const float* g, const float* b, T* out, const int* ctx_len, int batch,
-                                   int gamma, int L_cap, int d, cudaStream_t st) {
+                                   int gamma, int L_cap, int d, cudaStream_t st, const int* skip) {
   if (d > LN_MAX_PER_LANE * 32) return cudaErrorInvalidValue;
-  launch_k(layernorm_slots_kernel<T>, dim3((batch * gamma + 3) / 4), dim3(128), 0, st, h, g, b, out, ctx_len, batch, gamma, L_cap, d);
+  launch_k(layernorm_slots_kernel<T>, dim3((batch * gamma + 3) / 4), dim3(128), 0, st, h, g, b, out, ctx_len, batch, gamma, L_cap, d, skip);
   return cudaGetLastError();
 }
 template <typename T>
@@ -176,13 +181,13 @@ cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int bat
 
 #define SDD_INSTANTIATE_GLUE(T)                                                                                          \
   template cudaError_t launch_embed_drafter<T>(const T*, const T*, const int*, int, const int*, const int*, int, int,   \
-                                               int, int, float*, cudaStream_t);                                         \
+                                               int, int, float*, cudaStream_t, const int*);                             \
   template cudaError_t launch_embed_target<T>(const T*, const T*, const int*, int, const int*, const int*, int, int,    \
                                               int, int, int, float*, cudaStream_t);                                     \
   template cudaError_t launch_layernorm<T>(const float*, const float*, const float*, T*, long long, int, cudaStream_t, \
-                                           T*);                                                                         \
+                                           T*, const int*);                                                                         \
   template cudaError_t launch_layernorm_slots<T>(const float*, const float*, const float*, T*, const int*, int, int,    \
-                                                 int, int, cudaStream_t);                                               \
+                                                 int, int, cudaStream_t, const int*);                                   \
   template cudaError_t launch_kv_append<T>(const T*, T*, const int*, int, int, int, int, int, cudaStream_t);
 SDD_INSTANTIATE_GLUE(float)
 SDD_INSTANTIATE_GLUE(__nv_bfloat16)

@@ -9,7 +9,11 @@ namespace sdd {
 struct RoundState {
   int status;          // DEV_OK or the first device-side error
   uint32_t round;      // rounds committed so far == Philox round index of the round in flight
-  uint32_t pad[2];
+  uint32_t revealed;   // slots revealed by the denoising step in flight (all sequences)
+  uint32_t ticket;     // CTAs of that step's sampling kernel that have finished
+  int skip_forward;    // 1: the last step revealed nothing, so the next drafter evaluation would reproduce the
+                       //    logits it already has ("cache" strategy): its kernels return at once
+  int pad[3];
 };
 
 // How a target forward maps its rows to sequence positions.
@@ -37,13 +41,15 @@ struct QkvDst {
   int rows_per_seq, mode, d, k_seq_rows, vt_ld;
 };
 
+// Every kernel of a drafter evaluation takes `skip` (may be null): when *skip != 0 the kernel returns at once.
+
 // ---- vocabulary kernels (sdd_sample.cu) -----------------------------------------------------
 int stats_chunks_for(int V);
 cudaError_t launch_row_stats(const float* a, long long rows_a, const float* b, long long rows_b, int V, float inv_tau_a,
                              float inv_tau_b, float2* partial, cudaStream_t st);
 cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float* q_logits, float* logq, int* reveal_step,
                                  int batch, int gamma, int V, int k, float inv_tau_q, PhiloxKey key,
-                                 const RoundState* rs, cudaStream_t st);
+                                 RoundState* rs, int cache_skip, cudaStream_t st);
 cudaError_t launch_accept(const float* logits_p, const float* q_rows, const int* draft_ids, const float* logq_in,
                           const float2* partial_p, const float2* partial_q, int rows, int gamma, int V, float inv_tau_p,
                           float inv_tau_q_rows, PhiloxKey key, uint32_t rnd, const RoundState* rs, float* accept_prob,
@@ -51,12 +57,13 @@ cudaError_t launch_accept(const float* logits_p, const float* q_rows, const int*
 cudaError_t launch_commit(int* tokens, int tok_stride, int* ctx_len, int* n_emitted, const int* slot_ids,
                           const int* n_accept, const int* extra_token, int batch, int gamma, int max_new, RoundState* rs,
                           int* out_ids, int* n_out, volatile int* host_mirror, cudaStream_t st);
-cudaError_t launch_reset_slots(int* slot_ids, int* reveal_step, int n, int mask_id, cudaStream_t st);
+cudaError_t launch_reset_slots(int* slot_ids, int* reveal_step, int n, int mask_id, RoundState* rs, cudaStream_t st);
 
 // ---- glue (sdd_glue.cu) ---------------------------------------------------------------------
 template <typename T>
 cudaError_t launch_embed_drafter(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
-                                 const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st);
+                                 const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st,
+                                 const int* skip = nullptr);
 template <typename T>
 cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                 const int* slot_ids, int batch, int gamma, int rows_per_seq, int mode, int d, float* h,
@@ -65,11 +72,11 @@ cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, i
 // rounding remainder y - out so that (out, out_lo) carries y to about 16 significant bits
 template <typename T>
 cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* out, long long rows, int d, cudaStream_t st,
-                             T* out_lo = nullptr);
+                             T* out_lo = nullptr, const int* skip = nullptr);
 // final LayerNorm of the gamma slot rows of every sequence: out[b*gamma + j] = LN(h[b*L_cap + ctx_len[b] + j])
 template <typename T>
 cudaError_t launch_layernorm_slots(const float* h, const float* g, const float* b, T* out, const int* ctx_len, int batch,
-                                   int gamma, int L_cap, int d, cudaStream_t st);
+                                   int gamma, int L_cap, int d, cudaStream_t st, const int* skip = nullptr);
 // copy the K and V thirds of qkv rows into the cache: cache[b][pos][0|1][d]
 template <typename T>
 cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int batch, int rows_per_seq, int mode, int n_ctx,
@@ -79,7 +86,7 @@ cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int bat
 // C[M, N] = A[M, K] * W[N, K]^T; A row stride lda, W row stride K, out row stride ldc.
 template <typename T>
 cudaError_t launch_gemm_simt(const T* A, int lda, const T* W, const float* bias, int M, int N, int K, int epi, void* out,
-                             int ldc, cudaStream_t st);
+                             int ldc, cudaStream_t st, const int* skip = nullptr);
 
 // bf16 tensor-core GEMM (tcgen05 / TMEM / TMA).  A is a dense [a_cap, K] buffer of which M rows are used;
 // bn_hint selects the N tile (0 = choose); a bounded wait that expires sets *status = DEV_TIMEOUT.
@@ -87,7 +94,8 @@ cudaError_t launch_gemm_simt(const T* A, int lda, const T* W, const float* bias,
 // out_lo (optional, bf16 epilogues): receives bf16(x - bf16(x)) next to out = bf16(x).
 cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_bfloat16* W, const float* bias, int M, int N,
                            int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st,
-                           const QkvDst* qkv = nullptr, const __nv_bfloat16* A_lo = nullptr, void* out_lo = nullptr);
+                           const QkvDst* qkv = nullptr, const __nv_bfloat16* A_lo = nullptr, void* out_lo = nullptr,
+                           const int* skip = nullptr);
 
 // one-time set-up of the tensor-core kernels (dynamic shared-memory limits); also done lazily on first launch
 cudaError_t tc_prepare_gemm();
@@ -99,13 +107,14 @@ cudaError_t tc_prepare_attn();
 cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q_ld, int q_col0, const __nv_bfloat16* k,
                            long long k_rows_total, int k_ld, int k_col0, int k_rows_per_seq, const __nv_bfloat16* vt,
                            int vt_ld, __nv_bfloat16* out, int ld_out, const int* ctx_len, int batch, int n_head, int d,
-                           int gamma, int mode, int q_rows_per_seq, int* status, cudaStream_t st);
+                           int gamma, int mode, int q_rows_per_seq, int* status, cudaStream_t st,
+                           const int* skip = nullptr);
 
 // ---- attention (sdd_attn.cu) ----------------------------------------------------------------
 // drafter: every row of a sequence attends to rows 0 .. ctx_len[b] + gamma - 1 of the same sequence
 template <typename T>
 cudaError_t launch_attn_bidir(const T* qkv, T* out, const int* ctx_len, int batch, int gamma, int L_cap, int n_head,
-                              int d_head, cudaStream_t st);
+                              int d_head, cudaStream_t st, const int* skip = nullptr);
 // target: row j of sequence b (position p, see TargetMode) attends to cache positions 0 .. p
 template <typename T>
 cudaError_t launch_attn_cached(const T* qkv, const T* cache, T* out, const int* ctx_len, int batch, int rows_per_seq,

@@ -247,25 +247,24 @@ __device__ __forceinline__ MaxSum block_maxsum(MaxSum ms, float* s_m, float* s_s
 // ---------------------------------------------------------------------------------------------
 constexpr int SAMPLE_THREADS = 512;
 
-__global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(SAMPLE_THREADS)
-unmask_sample_kernel(const float* __restrict__ step_logits,  // [B, gamma, V]
+// returns true in every CTA of a cluster whose slot was revealed by this step
+__device__ __forceinline__ bool unmask_sample_row(const float* __restrict__ step_logits,  // [B, gamma, V]
                      int* __restrict__ slot_ids,             // [B, gamma]  (V = masked)
                      float* __restrict__ q_logits,           // [B, gamma, V]
                      float* __restrict__ logq,               // [B, gamma]
                      int* __restrict__ reveal_step,          // [B, gamma]
                      int gamma, int V, int k, float inv_tau_q, PhiloxKey key, const RoundState* __restrict__ rs) {
-  pdl_wait();
   cg::cluster_group cl = cg::this_cluster();
   const int rank = (int)cl.block_rank();
   const int j = blockIdx.x / VC, b = blockIdx.y;
   const uint32_t rnd = rs->round;
   const long long row = (long long)b * gamma + j;
   // every CTA of the cluster takes the same decision from the same inputs, before anyone writes the slot
-  if (slot_ids[row] != V) return;  // already revealed: carried over unchanged
+  if (slot_ids[row] != V) return false;  // already revealed: carried over unchanged
   // reveal with probability 1/k: u = m * 2^-24 with m odd, so u < 1/k  <=>  m * k < 2^24 (exact, k <= 255)
   const uint32_t wu = philox4x32_10(0u, (uint32_t)j, rnd, rng_c3(RNG_UNMASK, (uint32_t)k, (uint32_t)b), key).x;
   const uint32_t m_odd = ((wu >> 9) << 1) | 1u;
-  if (!(m_odd * (uint32_t)k < (1u << 24))) return;
+  if (!(m_odd * (uint32_t)k < (1u << 24))) return false;
 
   const float* __restrict__ src = step_logits + row * V;
   float* __restrict__ dst = q_logits + row * V;
@@ -316,6 +315,30 @@ unmask_sample_kernel(const float* __restrict__ step_logits,  // [B, gamma, V]
     reveal_step[row] = k;
   }
   cl.sync();   // partials stay alive until rank 0 has read them
+  return true;
+}
+
+
+// The last CTA of the grid to finish publishes whether this step revealed anything at all: if not, the next drafter
+// evaluation would see the same input and reproduce the logits it already has, so its kernels are told to return
+// at once (the paper's "ddpm cache" strategy: a step without change costs no network evaluation).
+__global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(SAMPLE_THREADS)
+unmask_sample_kernel(const float* __restrict__ step_logits, int* __restrict__ slot_ids, float* __restrict__ q_logits,
+                     float* __restrict__ logq, int* __restrict__ reveal_step, int gamma, int V, int k, float inv_tau_q,
+                     PhiloxKey key, RoundState* __restrict__ rs, int cache_skip) {
+  pdl_wait();
+  const bool revealed = unmask_sample_row(step_logits, slot_ids, q_logits, logq, reveal_step, gamma, V, k, inv_tau_q, key, rs);
+  if (threadIdx.x == 0) {
+    if (revealed && (blockIdx.x % VC) == 0) atomicAdd(&rs->revealed, 1u);
+    __threadfence();
+    const uint32_t t = atomicAdd(&rs->ticket, 1u);
+    if (t == gridDim.x * gridDim.y - 1) {
+      __threadfence();
+      const uint32_t n = atomicExch(&rs->revealed, 0u);
+      rs->skip_forward = (cache_skip && n == 0u) ? 1 : 0;
+      rs->ticket = 0u;
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -546,9 +569,11 @@ __global__ void commit_kernel(int* __restrict__ tokens, int tok_stride, int* __r
   }
 }
 
-__global__ void reset_slots_kernel(int* __restrict__ slot_ids, int* __restrict__ reveal_step, int n, int mask_id) {
+__global__ void reset_slots_kernel(int* __restrict__ slot_ids, int* __restrict__ reveal_step, int n, int mask_id,
+                                   RoundState* __restrict__ rs) {
   pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i == 0) { rs->skip_forward = 0; rs->revealed = 0u; rs->ticket = 0u; }   // a round's first evaluation always runs
   if (i < n) {
     slot_ids[i] = mask_id;
     reveal_step[i] = 0;
@@ -576,10 +601,10 @@ cudaError_t launch_row_stats(const float* a, long long rows_a, const float* b, l
 
 cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float* q_logits, float* logq, int* reveal_step,
                                  int batch, int gamma, int V, int k, float inv_tau_q, PhiloxKey key,
-                                 const RoundState* rs, cudaStream_t st) {
+                                 RoundState* rs, int cache_skip, cudaStream_t st) {
   dim3 grid(VC * gamma, batch);
   launch_k(unmask_sample_kernel, dim3(grid), dim3(SAMPLE_THREADS), 0, st, step_logits, slot_ids, q_logits, logq, reveal_step, gamma, V, k,
-                                                       inv_tau_q, key, rs);
+                                                       inv_tau_q, key, rs, cache_skip);
   return cudaGetLastError();
 }
 
@@ -602,8 +627,8 @@ cudaError_t launch_commit(int* tokens, int tok_stride, int* ctx_len, int* n_emit
   return cudaGetLastError();
 }
 
-cudaError_t launch_reset_slots(int* slot_ids, int* reveal_step, int n, int mask_id, cudaStream_t st) {
-  launch_k(reset_slots_kernel, dim3((n + 255) / 256), dim3(256), 0, st, slot_ids, reveal_step, n, mask_id);
+cudaError_t launch_reset_slots(int* slot_ids, int* reveal_step, int n, int mask_id, RoundState* rs, cudaStream_t st) {
+  launch_k(reset_slots_kernel, dim3((n + 255) / 256), dim3(256), 0, st, slot_ids, reveal_step, n, mask_id, rs);
   return cudaGetLastError();
 }
 

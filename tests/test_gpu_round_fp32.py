@@ -107,3 +107,22 @@ def test_call_order_and_argument_errors():
     with pytest.raises(sdd.SddError) as e:         # swapped models
         sdd.Session(dq, dp, prompts, [wl.prompt_len], 8, 4, 10)
     assert e.value.status == sdd.SDD_E_ARG
+
+
+def test_cache_skip_changes_nothing(monkeypatch):
+    """A denoising step that reveals nothing leaves the drafter's input unchanged, so the next evaluation is skipped
+    and its logits are reused ("ddpm cache").  Tokens must be identical with the skip switched off."""
+    import paper_2408_05636_b200 as sdd
+    wl = synth.WORKLOADS["tiny_fp32"]
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 2, wl.prompt_len, wl.prompt_seed)
+    outs = []
+    for flag in ("1", "0"):
+        monkeypatch.setenv("SDD_CACHE_SKIP", flag)
+        # T much larger than gamma: most steps reveal nothing
+        s = sdd.Session(dp, dq, prompts, [wl.prompt_len, 20], 4, 12, 24, 1.0, 1.0, wl.philox_seed)
+        toks, clen = s.generate()
+        outs.append((toks.copy(), clen.copy()))
+        s.close()
+    assert np.array_equal(outs[0][1], outs[1][1]) and np.array_equal(outs[0][0], outs[1][0])
+    assert outs[0][1].min() > wl.prompt_len - 13
