@@ -2,7 +2,7 @@
 //
 // One CTA owns 128 query rows of one head of one sequence and walks over the keys in tiles of 128:
 //   S  = Q K^T          tcgen05.mma, 128 x 128 fp32 accumulator in TMEM (Q, K tiles via TMA, K-major)
-//   P  = exp2(S - max)  four soft-max warps, one thread per query row (tcgen05.ld gives a thread its row);
+//   P  = exp2(S - max)  eight soft-max warps, two threads per query row (tcgen05.ld gives a thread its row);
 //                       P is written as bf16 into shared memory in the 128-byte-swizzled K-major layout
 //   PV = P V            tcgen05.mma with V^T tiles ([d_head, keys], keys contiguous) as the second operand,
 //                       64-column fp32 accumulator in TMEM, folded into the per-thread output row with the
@@ -19,7 +19,7 @@
 namespace sdd {
 namespace tc {
 
-constexpr int AT_THREADS = 192;
+constexpr int AT_THREADS = 320;              // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: soft-max
 constexpr int AT_DH = 64;
 constexpr int AT_Q_BYTES = 128 * 64 * 2;            // 16 KB
 constexpr int AT_P_BYTES = 2 * 128 * 64 * 2;        // two k-blocks of 64 keys: 32 KB
@@ -28,7 +28,7 @@ constexpr int AT_VT_BYTES = 2 * 64 * 64 * 2;        // two boxes [64 d_head rows
 constexpr int AT_STAGE_BYTES = AT_K_BYTES + AT_VT_BYTES;
 constexpr int AT_KV_STAGES = 2;
 constexpr int AT_BAR_OFF = AT_Q_BYTES + AT_P_BYTES + AT_KV_STAGES * AT_STAGE_BYTES;   // 112 KB
-constexpr int AT_SMEM = AT_BAR_OFF + 1024 + 256;
+constexpr int AT_SMEM = AT_BAR_OFF + 1024 + 128 + 3 * 1024;   // barriers, then the soft-max exchange arrays
 constexpr uint32_t AT_TMEM_COLS = 256;              // S: columns 0..127, PV: columns 128..191
 
 __device__ __forceinline__ float ex2(float x) {
@@ -51,7 +51,7 @@ struct AttnParams {
   const int* skip;      // may be null; *skip != 0: return at once (skipped drafter evaluation)
 };
 
-__global__ void __launch_bounds__(AT_THREADS)
+__global__ void __launch_bounds__(AT_THREADS, 2)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_vt, const AttnParams prm) {
   const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -88,7 +88,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    mbar_init(q_full, 1); mbar_init(s_full, 1); mbar_init(p_ready, 128); mbar_init(pv_full, 1);
+    mbar_init(q_full, 1); mbar_init(s_full, 1); mbar_init(p_ready, 256); mbar_init(pv_full, 1);
     for (int s = 0; s < AT_KV_STAGES; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -152,6 +152,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
   } else {
+    // soft-max warps 2..9: two threads per query row.  Warp w reads TMEM lane quarter w & 3; warps 2..5 take key
+    // columns 0..63 of the tile (and output columns 0..31), warps 6..9 key columns 64..127 (output columns 32..63).
+    const int hf = (warp - 2) >> 2;
     const int r = (warp & 3) * 32 + lane;
     const int i = q0 + r;
     const bool valid = i < n_valid_q;
@@ -163,26 +166,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (!valid) key_limit = 0;
     const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     const float scale = 0.125f * 1.4426950408889634f;  // 1/sqrt(64) * log2(e)
+    float* s_max = reinterpret_cast<float*>(gbase + AT_BAR_OFF + 128);          // [2 tile parities][2 halves][128 rows]
+    float* s_l = s_max + 2 * 2 * 128;                                            // [2 halves][128 rows]
     float m = -INFINITY, l = 0.f;
-    float o[AT_DH];
+    float o[AT_DH / 2];
 #pragma unroll
-    for (int j = 0; j < AT_DH; ++j) o[j] = 0.f;
-    uint8_t* p_row = gbase + AT_Q_BYTES + r * 128;
+    for (int j = 0; j < AT_DH / 2; ++j) o[j] = 0.f;
+    uint8_t* p_row = gbase + AT_Q_BYTES + hf * (128 * 64 * 2) + r * 128;         // this thread's 64 keys = one k-block row
     const int sw = r & 7;
     bool ok = true;
     for (int t = 0; t < num_kt; ++t) {
       ok = __all_sync(0xffffffffu, mbar_wait(s_full, (uint32_t)t & 1u, abort_flag, prm.status));
+      ok = named_bar_and(1, 256, ok);                  // also orders the reuse of s_max[t & 1] (last read at tile t - 2)
       if (!ok) break;
       fence_after_sync();
-      const int key0 = t * 128;
-      // rows that see the whole tile (every tile but the last one, or the diagonal one under the causal mask)
-      // skip the per-entry visibility test
-      const bool full = key0 + 128 <= key_limit;
+      const int key0 = t * 128 + hf * 64;
+      // rows that see all of their 64 keys skip the per-entry visibility test
+      const bool full = key0 + 64 <= key_limit;
+      // the 64 scores are read twice from TMEM (once for the maximum, once for the exponentials) instead of being
+      // kept in 64 registers: two CTAs per SM need the kernel to stay near 100 registers
+      uint32_t v[32];
       float mx = -INFINITY;
 #pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(t_lane + (uint32_t)(cc * 32), v);
+      for (int cc = 0; cc < 2; ++cc) {
+        tmem_ld32(t_lane + (uint32_t)(hf * 64 + cc * 32), v);
         if (full) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
@@ -192,15 +199,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             if (key0 + cc * 32 + j < key_limit) mx = fmaxf(mx, __uint_as_float(v[j]));
         }
       }
+      float* sm = s_max + (t & 1) * 256;
+      sm[hf * 128 + r] = mx;
+      named_bar_sync(2, 256);
+      mx = fmaxf(mx, sm[(hf ^ 1) * 128 + r]);
       const float m_new = fmaxf(m, mx * scale);
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
       const float corr = m == -INFINITY ? 0.f : ex2(m - m_use);
       float sum = 0.f;
 #pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(t_lane + (uint32_t)(cc * 32), v);
-        uint8_t* blk = p_row + (cc >> 1) * (128 * 64 * 2);
+      for (int cc = 0; cc < 2; ++cc) {
+        tmem_ld32(t_lane + (uint32_t)(hf * 64 + cc * 32), v);
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           uint32_t pk[4];
@@ -217,37 +226,38 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
             pk[e] = *reinterpret_cast<uint32_t*>(&h2);
           }
-          const int chunk = (cc & 1) * 4 + g;           // 16-byte chunk of this row inside the 64-key block
-          *reinterpret_cast<uint4*>(blk + ((chunk ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          *reinterpret_cast<uint4*>(p_row + (((cc * 4 + g) ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
       }
-      l = l * corr + sum;
+      l = l * corr + sum;     // this thread's half of the row sum; the halves share m, so they add up at the end
       m = m_new;
       fence_async_smem();
       mbar_arrive(p_ready);
       ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)t & 1u, abort_flag, prm.status));
       if (!ok) break;
       fence_after_sync();
+      tmem_ld32(t_lane + 128u + (uint32_t)(hf * 32), v);
 #pragma unroll
-      for (int cc = 0; cc < 2; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(t_lane + 128u + (uint32_t)(cc * 32), v);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) o[cc * 32 + j] = fmaf(o[cc * 32 + j], corr, __uint_as_float(v[j]));
-      }
+      for (int j = 0; j < 32; ++j) o[j] = fmaf(o[j], corr, __uint_as_float(v[j]));
     }
-    if (ok && valid) {
-      const float inv = 1.f / l;
-      __nv_bfloat16* dst = prm.out + ((long long)b * prm.q_rows_per_seq + i) * prm.ld_out + h * AT_DH;
+    ok = named_bar_and(1, 256, ok);
+    if (ok) {
+      s_l[hf * 128 + r] = l;
+      named_bar_sync(2, 256);
+      l += s_l[(hf ^ 1) * 128 + r];
+      if (valid) {
+        const float inv = 1.f / l;
+        __nv_bfloat16* dst = prm.out + ((long long)b * prm.q_rows_per_seq + i) * prm.ld_out + h * AT_DH + hf * 32;
 #pragma unroll
-      for (int g = 0; g < 8; ++g) {
-        uint32_t pk[4];
+        for (int g = 0; g < 4; ++g) {
+          uint32_t pk[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          __nv_bfloat162 h2 = __floats2bfloat162_rn(o[g * 8 + 2 * e] * inv, o[g * 8 + 2 * e + 1] * inv);
-          pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+          for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(o[g * 8 + 2 * e] * inv, o[g * 8 + 2 * e + 1] * inv);
+            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+          }
+          *reinterpret_cast<uint4*>(dst + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
-        *reinterpret_cast<uint4*>(dst + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
     }
   }
