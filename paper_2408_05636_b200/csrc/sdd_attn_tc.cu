@@ -10,6 +10,9 @@
 // The same kernel serves the drafter (no mask: every row sees every row of its sequence) and the target
 // (row at position p sees cache positions 0..p).  V is consumed transposed, which the QKV GEMM's epilogue
 // produces for free; that keeps both MMAs on K-major operands.
+// Shared memory: the K tile of a stage is dead once S = Q K^T has completed and stays unused until P V has
+// completed (only then is the stage handed back to the producer), so the first half of P (keys 0..63) is written
+// over it; with that the CTA needs 96 KB and two CTAs share an SM, one's soft-max overlapping the other's MMAs.
 // Waits are bounded exactly as in the GEMM kernel.
 #include <mutex>
 
@@ -22,12 +25,12 @@ namespace tc {
 constexpr int AT_THREADS = 320;              // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: soft-max
 constexpr int AT_DH = 64;
 constexpr int AT_Q_BYTES = 128 * 64 * 2;            // 16 KB
-constexpr int AT_P_BYTES = 2 * 128 * 64 * 2;        // two k-blocks of 64 keys: 32 KB
+constexpr int AT_P_BYTES = 128 * 64 * 2;            // P k-block 1 (keys 64..127); k-block 0 reuses the K tile, see below
 constexpr int AT_K_BYTES = 128 * 64 * 2;            // 16 KB
 constexpr int AT_VT_BYTES = 2 * 64 * 64 * 2;        // two boxes [64 d_head rows x 64 keys]: 16 KB
 constexpr int AT_STAGE_BYTES = AT_K_BYTES + AT_VT_BYTES;
 constexpr int AT_KV_STAGES = 2;
-constexpr int AT_BAR_OFF = AT_Q_BYTES + AT_P_BYTES + AT_KV_STAGES * AT_STAGE_BYTES;   // 112 KB
+constexpr int AT_BAR_OFF = AT_Q_BYTES + AT_P_BYTES + AT_KV_STAGES * AT_STAGE_BYTES;   // 96 KB: two CTAs per SM
 constexpr int AT_SMEM = AT_BAR_OFF + 1024 + 128 + 3 * 1024;   // barriers, then the soft-max exchange arrays
 constexpr uint32_t AT_TMEM_COLS = 256;              // S: columns 0..127, PV: columns 128..191
 
@@ -142,7 +145,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         fence_after_sync();
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb) {
-          const uint64_t dp = make_smem_desc(sP + kb * (128 * 64 * 2));
+          const uint64_t dp = make_smem_desc(kb == 0 ? sK(s) : sP);
           const uint64_t dv = make_smem_desc(sVT(s) + kb * (64 * 64 * 2));
 #pragma unroll
           for (int k = 0; k < 4; ++k) umma(tmem_base + 128u, dp + 2u * k, dv + 2u * k, idesc_pv, (kb | k) ? 1u : 0u);
@@ -172,7 +175,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     float o[AT_DH / 2];
 #pragma unroll
     for (int j = 0; j < AT_DH / 2; ++j) o[j] = 0.f;
-    uint8_t* p_row = gbase + AT_Q_BYTES + hf * (128 * 64 * 2) + r * 128;         // this thread's 64 keys = one k-block row
     const int sw = r & 7;
     bool ok = true;
     for (int t = 0; t < num_kt; ++t) {
@@ -181,6 +183,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (!ok) break;
       fence_after_sync();
       const int key0 = t * 128 + hf * 64;
+      // this thread's 64 probabilities are one row of a P k-block: block 0 lies over the stage's (consumed) K tile
+      uint8_t* p_row = gbase + (hf == 0 ? AT_Q_BYTES + AT_P_BYTES + (t & 1) * AT_STAGE_BYTES : AT_Q_BYTES) + r * 128;
       // rows that see all of their 64 keys skip the per-entry visibility test
       const bool full = key0 + 64 <= key_limit;
       // the 64 scores are read twice from TMEM (once for the maximum, once for the exponentials) instead of being
