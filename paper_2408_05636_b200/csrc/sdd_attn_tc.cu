@@ -59,6 +59,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                const __grid_constant__ CUtensorMap map_vt, const AttnParams prm) {
   const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   pdl_wait();   // ctx_len and Q / K / V^T come from earlier kernels
+  pdl_launch_dependents();
   if (prm.skip != nullptr && *prm.skip) return;
   const int c = prm.ctx_len[b];
   const int q0 = qt * 128;

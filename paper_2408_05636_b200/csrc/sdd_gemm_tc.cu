@@ -59,10 +59,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_out, int tma_out,
                int rows_a, int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out,
                void* __restrict__ out_lo, int ldc, int* status, const QkvDst qd, const int* __restrict__ skip) {
-  if (skip != nullptr) {   // launches of a drafter evaluation: nothing to do if the evaluation is skipped
-    pdl_wait();
-    if (*skip) return;
-  }
+
   constexpr int STAGES = ring_stages<BN, SWAP, HILO>();
   constexpr int STAGE_BYTES = stage_bytes<BN, SWAP, HILO>();
   constexpr int LO_OFF = BM * BK * 2 + BN * BK * 2;     // offset of the lo tile inside a stage
@@ -104,8 +101,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // everything above touched only shared / tensor memory; global inputs may still be in production
   pdl_wait();
   pdl_launch_dependents();
+  // launches of a drafter evaluation do nothing when the evaluation is skipped (they still free their TMEM below)
+  const bool active = skip == nullptr || *skip == 0;
 
-  if (warp == 0) {
+  if (!active) {
+  } else if (warp == 0) {
     if (lane == 0) {
       int issued = 0;
       for (int kb = 0; kb < num_kb; ++kb) {

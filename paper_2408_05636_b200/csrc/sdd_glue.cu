@@ -13,6 +13,7 @@ __global__ void embed_drafter_kernel(const T* __restrict__ wte, const T* __restr
                                      int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
                                      int gamma, int L_cap, int d, float* __restrict__ h, const int* __restrict__ skip) {
   pdl_wait();
+  pdl_launch_dependents();
   if (skip != nullptr && *skip) return;
   const int i = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
@@ -34,6 +35,7 @@ __global__ void embed_target_kernel(const T* __restrict__ wte, const T* __restri
                                     int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
                                     int gamma, int rows_per_seq, int mode, int d, float* __restrict__ h) {
   pdl_wait();
+  pdl_launch_dependents();
   const int j = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
   float* __restrict__ dst = h + ((long long)b * rows_per_seq + j) * d;
@@ -99,6 +101,7 @@ __global__ void __launch_bounds__(128)
 layernorm_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
                  T* __restrict__ out, T* __restrict__ out_lo, long long rows, int d, const int* __restrict__ skip) {
   pdl_wait();
+  pdl_launch_dependents();
   if (skip != nullptr && *skip) return;
   const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -111,6 +114,7 @@ layernorm_slots_kernel(const float* __restrict__ h, const float* __restrict__ g,
                        T* __restrict__ out, const int* __restrict__ ctx_len, int batch, int gamma, int L_cap, int d,
                        const int* __restrict__ skip) {
   pdl_wait();
+  pdl_launch_dependents();
   if (skip != nullptr && *skip) return;
   const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
   if (r >= batch * gamma) return;
@@ -125,6 +129,7 @@ template <typename T>
 __global__ void kv_append_kernel(const T* __restrict__ qkv, T* __restrict__ cache, const int* __restrict__ ctx_len,
                                  int rows_per_seq, int mode, int n_ctx, int d) {
   pdl_wait();
+  pdl_launch_dependents();
   const int j = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
   int pos;
