@@ -105,6 +105,21 @@ def round_work(wl, c: int):
     return w
 
 
+def aggregate_over_ranks(ms, toks, dist, device):
+    """Whole-job figures of independent replicas: the slowest rank's device time, the sum of the tokens."""
+    import torch
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    k = torch.tensor([float(toks)], device=device, dtype=torch.float64)
+    dist.all_reduce(k, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(k.item())
+
+
+def replica_prompt_seed(base_seed: int, rank: int, generation: int) -> int:
+    """Every replica (rank) and every generation of a replica gets its own prompt."""
+    return base_seed + 1000 * rank + generation
+
+
 def make_models(wl, device):
     import paper_2408_05636_b200 as sdd
     wp = synth.model_weights(wl.target, wl.weight_seed, wl.dtype)
@@ -142,7 +157,7 @@ def run_ours(args):
     gen_idx = [0]
 
     def new_session():
-        seed = wl.prompt_seed + 1000 * rank + gen_idx[0]
+        seed = replica_prompt_seed(wl.prompt_seed, rank, gen_idx[0])
         gen_idx[0] += 1
         prompts = synth.prompt_ids(V, wl.batch, wl.prompt_len, seed)
         s = sdd.Session(dp, dq, prompts, [wl.prompt_len] * wl.batch, wl.gamma, wl.T, wl.max_new, 1.0, 1.0,
@@ -198,12 +213,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
-        t = torch.tensor([ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        k = torch.tensor([toks], device=device, dtype=torch.float64)
-        dist.all_reduce(k, op=dist.ReduceOp.SUM)
-        toks = int(k.item())
+        ms, toks = aggregate_over_ranks(ms, toks, dist, device)
     # keep the GPU busy a little longer so that the clock sampler sees load (same work, untimed)
     t_end = time.time() + (0.0 if args.rounds_only else 1.0)
     while time.time() < t_end:
