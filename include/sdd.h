@@ -221,7 +221,8 @@ int32_t sdd_counters(sdd_ctx* ctx, uint64_t* rounds, uint64_t* kernel_launches);
 /* Optional per-launch timing, for measurement only (it adds two CUDA events around every kernel
  * launch, so it is not meant to be left on).  sdd_profile_begin starts collecting; sdd_profile_end
  * synchronises the stream and returns, per kernel category, the summed device time in milliseconds
- * and the number of launches (arrays of n_categories >= SDD_PROF_COUNT entries). */
+ * and the number of launches (arrays of n_categories >= SDD_PROF_COUNT entries).  The event pairs are
+ * recorded inside the round's graph; the cost of an empty pair, measured in the same graph, is subtracted. */
 enum {
   SDD_PROF_GEMM_DRAFTER = 0, SDD_PROF_GEMM_TARGET = 1, SDD_PROF_HEAD_DRAFTER = 2, SDD_PROF_HEAD_TARGET = 3,
   SDD_PROF_ATTN_DRAFTER = 4, SDD_PROF_ATTN_TARGET = 5, SDD_PROF_LAYERNORM = 6, SDD_PROF_GLUE = 7,

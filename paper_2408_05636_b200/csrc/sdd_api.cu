@@ -200,14 +200,21 @@ struct ProfScope {
         c->prof_ev.push_back(e);
       }
     }
-    cudaEventRecord(c->prof_ev[c->prof_used], c->st);
+    record(c->prof_ev[c->prof_used]);
     c->prof_cat.push_back(cat);
     on = true;
   }
   ~ProfScope() {
     if (!on) return;
-    cudaEventRecord(c->prof_ev[c->prof_used + 1], c->st);
+    record(c->prof_ev[c->prof_used + 1]);
     c->prof_used += 2;
+  }
+  // inside a stream capture a plain record only orders work; the external flag makes it a graph node that stamps
+  // the event when the graph runs
+  void record(cudaEvent_t e) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    cudaStreamIsCapturing(c->st, &cs);
+    cudaEventRecordWithFlags(e, c->st, cs == cudaStreamCaptureStatusActive ? cudaEventRecordExternal : cudaEventRecordDefault);
   }
 };
 
@@ -554,6 +561,8 @@ static int round_prologue(sdd_ctx* c) {
   return SDD_OK;
 }
 static int enqueue_draft_begin(sdd_ctx* c) {
+  // per-launch timing: a few empty event pairs per round measure what a pair costs by itself (subtracted later)
+  for (int i = 0; i < 4 && c->profiling; ++i) { ProfScope calib(c, CAT_COUNT); }
   SDD_LAUNCH(c, CAT_GLUE, launch_reset_slots(c->B.slot_ids, c->B.reveal_step, c->D.batch * c->D.gamma, c->D.V, c->B.rs, c->st));
   c->steps_done = 0;
   return SDD_OK;
@@ -765,11 +774,21 @@ int32_t sdd_profile_end(sdd_ctx* c, double* ms_per_category, uint64_t* launches_
   c->profiling = false;
   SDD_CUDA(cudaStreamSynchronize(c->st));
   for (int i = 0; i < n_categories; ++i) { ms_per_category[i] = 0.0; launches_per_category[i] = 0; }
+  double empty_ms = 0.0;
+  uint64_t empty_n = 0;
   for (size_t i = 0; i + 1 < c->prof_used + 1 && i / 2 < c->prof_cat.size(); i += 2) {
     float ms = 0.f;
     SDD_CUDA(cudaEventElapsedTime(&ms, c->prof_ev[i], c->prof_ev[i + 1]));
-    ms_per_category[c->prof_cat[i / 2]] += ms;
-    launches_per_category[c->prof_cat[i / 2]] += 1;
+    const int cat = c->prof_cat[i / 2];
+    if (cat == CAT_COUNT) { empty_ms += ms; empty_n += 1; continue; }
+    ms_per_category[cat] += ms;
+    launches_per_category[cat] += 1;
+  }
+  // subtract the cost of an empty event pair from every measured launch
+  const double per_pair = empty_n ? empty_ms / (double)empty_n : 0.0;
+  for (int i = 0; i < CAT_COUNT; ++i) {
+    ms_per_category[i] -= per_pair * (double)launches_per_category[i];
+    if (ms_per_category[i] < 0.0) ms_per_category[i] = 0.0;
   }
   c->prof_used = 0;
   c->prof_cat.clear();

@@ -39,28 +39,29 @@ constexpr int THREADS = 192;     // warp 0: TMA producer, warp 1: MMA issuer + T
 // one stage = A tile + B tile (+ the lo tile of the activation operand: the A side unless SWAP)
 template <int BN, bool SWAP, bool HILO>
 constexpr int stage_bytes() { return BM * BK * 2 + BN * BK * 2 + (HILO ? (SWAP ? BN : BM) * BK * 2 : 0); }
-// shared-memory ring depth: as deep as one CTA per SM allows (about 190 KB), so that a short K loop has all of its
-// tiles in flight at once
-template <int BN, bool SWAP, bool HILO>
+// shared-memory ring depth.  DEEP (grids of at most one wave): as deep as one CTA per SM allows (about 200 KB), so
+// that a short K loop has all of its tiles in flight at once.  Otherwise (multi-wave grids): half of that, so that two
+// CTAs share an SM and one's epilogue and prologue overlap the other's main loop.
+template <int BN, bool SWAP, bool HILO, bool DEEP>
 constexpr int ring_stages() {
-  constexpr int s = (200 * 1024) / stage_bytes<BN, SWAP, HILO>();
-  return s > 8 ? 8 : s;
+  constexpr int s = ((DEEP ? 200 : 100) * 1024) / stage_bytes<BN, SWAP, HILO>();
+  return s > 8 ? 8 : (s < 2 ? 2 : s);
 }
-template <int BN, bool SWAP, bool HILO>
+template <int BN, bool SWAP, bool HILO, bool DEEP>
 constexpr int smem_bytes() {
-  return ring_stages<BN, SWAP, HILO>() * stage_bytes<BN, SWAP, HILO>() + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  return ring_stages<BN, SWAP, HILO, DEEP>() * stage_bytes<BN, SWAP, HILO>() + 1024 /*alignment slack*/ + 256 /*barriers*/;
 }
 
 // grid = (N tiles, M tiles, K splits).  With more than one K split every CTA accumulates its share of the K
 // range and adds it to the fp32 output with atomics (EPI_RESIDUAL only; the bias is added by split 0).
-template <int BN, bool SWAP, bool HILO>
+template <int BN, bool SWAP, bool HILO, bool DEEP>
 __global__ void __launch_bounds__(THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_out, int tma_out,
                int rows_a, int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out,
                void* __restrict__ out_lo, int ldc, int* status, const QkvDst qd, const int* __restrict__ skip) {
 
-  constexpr int STAGES = ring_stages<BN, SWAP, HILO>();
+  constexpr int STAGES = ring_stages<BN, SWAP, HILO, DEEP>();
   constexpr int STAGE_BYTES = stage_bytes<BN, SWAP, HILO>();
   constexpr int LO_OFF = BM * BK * 2 + BN * BK * 2;     // offset of the lo tile inside a stage
   extern __shared__ uint8_t smem_raw[];
@@ -370,14 +371,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 // host side: tensor maps (cached per pointer / shape / box) and launch
 // ---------------------------------------------------------------------------------------------
+template <int BN, bool SWAP, bool HILO, bool DEEP>
+static cudaError_t launch_cfg2(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& mo,
+                              int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias, void* out, void* out_lo,
+                              int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits, const int* skip) {
+  dim3 grid((rows_b + BN - 1) / BN, (rows_a + BM - 1) / BM, splits);
+  launch_k(gemm_tc_kernel<BN, SWAP, HILO, DEEP>, grid, dim3(THREADS), smem_bytes<BN, SWAP, HILO, DEEP>(), st, ma, mb, ml, mo, tma_out,
+           rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip);
+  return cudaGetLastError();
+}
 template <int BN, bool SWAP, bool HILO>
 static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& mo,
                               int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias, void* out, void* out_lo,
                               int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits, const int* skip) {
-  dim3 grid((rows_b + BN - 1) / BN, (rows_a + BM - 1) / BM, splits);
-  launch_k(gemm_tc_kernel<BN, SWAP, HILO>, grid, dim3(THREADS), smem_bytes<BN, SWAP, HILO>(), st, ma, mb, ml, mo, tma_out,
-           rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip);
-  return cudaGetLastError();
+  // more than two waves of CTAs: shallow rings, two CTAs per SM (needs 2 x BN TMEM columns <= 512: always true)
+  const long long ctas = (long long)((rows_b + BN - 1) / BN) * ((rows_a + BM - 1) / BM) * splits;
+  if (ctas > 2 * 148)
+    return launch_cfg2<BN, SWAP, HILO, false>(ma, mb, ml, mo, tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status,
+                                              st, qd, splits, skip);
+  return launch_cfg2<BN, SWAP, HILO, true>(ma, mb, ml, mo, tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, st,
+                                           qd, splits, skip);
 }
 template <int BN, bool SWAP>
 static cudaError_t launch_hl(bool hilo, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml,
@@ -391,11 +404,14 @@ static cudaError_t launch_hl(bool hilo, const CUtensorMap& ma, const CUtensorMap
 
 template <int BN, bool SWAP>
 static cudaError_t prepare_one() {
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, SWAP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       smem_bytes<BN, SWAP, false>());
+  cudaError_t e;
+#define SDD_PREP(HILO, DEEP)                                                                                      \
+  e = cudaFuncSetAttribute(gemm_tc_kernel<BN, SWAP, HILO, DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                           smem_bytes<BN, SWAP, HILO, DEEP>());                                                \
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(gemm_tc_kernel<BN, SWAP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              smem_bytes<BN, SWAP, true>());
+  SDD_PREP(false, true) SDD_PREP(false, false) SDD_PREP(true, true) SDD_PREP(true, false)
+#undef SDD_PREP
+  return cudaSuccess;
 }
 
 }  // namespace tc
