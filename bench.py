@@ -29,6 +29,10 @@ import synth  # noqa: E402
 WORKLOAD = "small_bf16"
 METRIC = "SpecDiff generated tokens/s at bs=1"
 UNIT = "tokens/s"
+CONFIG = {"workload": "bf16 12L d768 target + 12L d768 masked-diffusion drafter, V=50257, prompt 256, "
+                      "gamma=16, T=8, batch 1, 256 new tokens",
+          "l2": "no flush: consecutive rounds of one generation; each round streams ~0.5 GB of weights (> 126 MB L2)",
+          "multi_gpu": "independent replicas, no collective on the data path"}
 
 
 def load_peaks():
@@ -321,10 +325,7 @@ def run_ours(args):
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "bf16 12L d768 target + 12L d768 masked-diffusion drafter, V=50257, prompt 256, "
-                               "gamma=16, T=8, batch 1, 256 new tokens",
-                   "l2": "no flush: consecutive rounds of one generation; each round streams ~0.5 GB of weights (> 126 MB L2)",
-                   "multi_gpu": "independent replicas, no collective on the data path"},
+        "config": CONFIG,
         "tokens_per_step": round(toks / args.steps / world, 3),
         "clocks": clock_info, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "roofline_accept_kernel": accept_roof, "roofline_gemm_kernel": gemm_roof,
@@ -401,8 +402,7 @@ def run_reference(args):
             "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": done, "steps_requested": args.steps,
             "warmup": args.warmup, "ms_per_step": round(dt * 1e3 / done, 2), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "bf16-rounded weights, 12L d768 target + 12L d768 masked-diffusion drafter, V=50257, "
-                                   "prompt 256, gamma=16, T=8, batch 1"},
+            "config": CONFIG,
             "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}

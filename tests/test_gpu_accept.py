@@ -76,3 +76,23 @@ def test_argument_errors():
         sdd.sdd_accept_logits(lp, lq, ids, 1.0, 0.0, 0, 0)      # mixed greedy / stochastic
     assert e.value.status == sdd.SDD_E_ARG
     assert sdd.sdd_accept_scratch_bytes(0, 1, 1) == 0
+
+
+def test_extreme_shapes():
+    """Largest supported draft length (gamma = 256 fills the decision stage's thread block), a single row with a
+    single draft, and a vocabulary of two."""
+    for rows, gamma, V in ((2, 256, 40), (1, 1, 2), (3, 200, 129)):
+        case = synth.accept_case(rows, gamma, V, 0.4, seed=rows + gamma)
+        log, n = _run_case(case, 1.0, 1.0, seed=5, rnd=1)
+        assert len(log) <= 1
+    import paper_2408_05636_b200 as sdd
+    case = synth.accept_case(1, 2, 16, 0.5, seed=1)
+    lp, lq = torch.from_numpy(case.logits_p).cuda(), torch.from_numpy(case.logits_q).cuda()
+    ids = torch.from_numpy(case.draft_ids).cuda()
+    L = sdd.lib()
+    out = torch.zeros(8, dtype=torch.int32, device="cuda")
+    prob = torch.zeros(8, device="cuda")
+    scratch = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    # gamma beyond the supported maximum is refused before anything is launched
+    assert L.sdd_accept_logits(lp.data_ptr(), lq.data_ptr(), ids.data_ptr(), 1, 257, 16, 1.0, 1.0, 0, 0, out.data_ptr(),
+                               out.data_ptr(), prob.data_ptr(), scratch.data_ptr(), None) == sdd.SDD_E_ARG
