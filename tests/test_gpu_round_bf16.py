@@ -50,3 +50,16 @@ def test_xl_bf16_one_round_reduced_T():
     print("near-ties:", log, "max logit err q/p:", stats["max_q_err"], stats["max_p_err"])
     assert len(log) <= 2
     s.close()
+
+
+def test_small_bf16_greedy_round():
+    """Temperature 0 (the setting of every result the paper reports): draft = arg-max, accept iff it equals the
+    target's arg-max, extra token = target arg-max; checked stage by stage on the library's own logits."""
+    import paper_2408_05636_b200 as sdd
+    wl = synth.scaled_workload(synth.WORKLOADS["small_bf16"], T=2)
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 1, 64, wl.prompt_seed)
+    s = sdd.Session(dp, dq, prompts, [64], wl.gamma, 2, 40, 0.0, 0.0, wl.philox_seed)
+    log, stats = roundcheck.check_rounds(s, mp, mq, wl, 2, 0.0, 0.0, TOL)
+    assert not log
+    s.close()
