@@ -245,6 +245,7 @@ def run_ours(args):
     cat_n = {n: 0 for n in sdd.PROF_NAMES}
     cat_work = {n: 0.0 for n in sdd.PROF_NAMES}
     kinds = {}
+    acc_stats = {"accepted": 0, "tested": 0, "ratio_sum": 0.0}
     for _ in range(prof_rounds):
         if emitted(sess)[1] >= wl.max_new:
             sess.close()
@@ -253,6 +254,11 @@ def run_ours(args):
         sess.sdd_profile_begin()
         sess.sdd_step()
         res = sess.sdd_profile_end()
+        n_acc = int(sess.tap_numpy(sdd.TAP_N_ACCEPT)[0])
+        tested = n_acc + 1 if n_acc < wl.gamma else wl.gamma
+        acc_stats["accepted"] += n_acc
+        acc_stats["tested"] += tested
+        acc_stats["ratio_sum"] += float(sess.tap_numpy(sdd.TAP_ACCEPT_PROB)[:tested].sum())
         work = round_work(wl, c)
         for n, (m, k) in res.items():
             cat_ms[n] += m
@@ -278,6 +284,39 @@ def run_ours(args):
                 "traffic": None, "peak_source": f"of {peaks['source']}",
                 "timing": f"CUDA-event pairs around every launch in a separate pass of {prof_rounds} rounds"}
     sess.close()
+
+    # ---- the paper's closed forms next to the measurement (Eq. 2, Eq. 3) and the autoregressive context line ----
+    alpha_hat = acc_stats["accepted"] / max(1, acc_stats["tested"])
+    mean_min = acc_stats["ratio_sum"] / max(1, acc_stats["tested"])   # E_x~q min(1, p/q) = sum_x min(p, q)
+    ln_q = wl.T * (2 * wl.drafter.n_layer + 1)
+    ln_p = 2 * wl.target.n_layer + 1
+    drafter_ms = (cat_ms["gemm_drafter"] + cat_ms["head_drafter"] + cat_ms["attn_drafter"] + cat_ms["sample"] +
+                  cat_ms["glue"] + cat_ms["layernorm"] * ln_q / (ln_q + ln_p))
+    frac_q = drafter_ms / total_ms
+    ms_round = ms / args.steps
+    c1 = frac_q * ms_round / wl.T
+    c2 = (1.0 - frac_q) * ms_round
+    e_tok = (1 - alpha_hat ** (wl.gamma + 1)) / (1 - alpha_hat) if alpha_hat < 1 else wl.gamma + 1
+    s_ar = new_session()
+    for _ in range(4):
+        s_ar.sdd_ar_step()
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ar_steps = 128
+    s_ar.stream.synchronize()
+    a0.record(s_ar.stream)
+    for _ in range(ar_steps):
+        s_ar.sdd_ar_step()
+    a1.record(s_ar.stream)
+    s_ar.sdd_sync_status()
+    ar_ms = a0.elapsed_time(a1) / ar_steps
+    s_ar.close()
+    model = {"alpha_hat": round(alpha_hat, 4), "mean_sum_min_pq": round(mean_min, 4),
+             "tokens_per_round_eq2": round(e_tok, 3), "tokens_per_round_measured": round(toks / args.steps / world, 3),
+             "c1_ms_per_drafter_evaluation": round(c1, 4), "c2_ms_target_and_accept": round(c2, 4),
+             "tokens_per_s_eq3": round(e_tok / ((wl.T * c1 + c2) * 1e-3), 1),
+             "autoregressive_target_tokens_per_s": round(1e3 / ar_ms, 1),
+             "note": "Eq. 2 / Eq. 3 of the paper with the measured acceptance rate and stage times; the autoregressive line "
+                     "is plain decoding of the same synthetic target (sdd_ar_step), context only"}
 
     # ---- stand-alone kernels (paper_2408_05636_b200.microbench) --------------------------------
     from paper_2408_05636_b200 import microbench
@@ -329,7 +368,7 @@ def run_ours(args):
         "tokens_per_step": round(toks / args.steps / world, 3),
         "clocks": clock_info, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "roofline_accept_kernel": accept_roof, "roofline_gemm_kernel": gemm_roof,
-        "kernels": kernels, "cpu_baseline": cpu,
+        "kernels": kernels, "paper_model": model, "cpu_baseline": cpu,
     }
     print(json.dumps(line))
     if dist is not None:

@@ -116,6 +116,14 @@ int32_t sdd_verify_accept(sdd_ctx* ctx, int32_t* out_ids, int32_t* n_out);
 /* One whole round = sdd_draft + sdd_verify_accept. */
 int32_t sdd_step(sdd_ctx* ctx, int32_t* out_ids, int32_t* n_out);
 
+/* Plain autoregressive decoding of the target, one token per call: the "standard generation" that the paper's
+ * speed-ups are quoted against (Table 1, row "Autoregressive"), expressed as a round with an empty draft (gamma = 0:
+ * nothing to test, the emitted token is the draw from p).  May be mixed freely with sdd_step between rounds; the
+ * Philox round index advances by one per call and the draw uses the bonus stream at slot 0.
+ * out_ids: device int32 [batch] (one token per sequence, -1 if the sequence is complete), n_out: device int32 [batch];
+ * either may be null. */
+int32_t sdd_ar_step(sdd_ctx* ctx, int32_t* out_ids, int32_t* n_out);
+
 /* Non-blocking progress read (host): rounds whose commit has been seen so far, and the smallest
  * number of generated tokens over the batch at that point.  Either pointer may be null. */
 int32_t sdd_progress(sdd_ctx* ctx, uint64_t* rounds_done, int32_t* min_emitted);

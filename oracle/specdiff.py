@@ -254,6 +254,22 @@ def autoregressive_greedy(model_p: Model, prompt, n_new: int) -> np.ndarray:
     return np.array(ids, dtype=np.int64)
 
 
+def autoregressive_sample(model_p: Model, prompt, n_new: int, tau_p: float, seed: int, b: int = 0,
+                          first_round: int = 0) -> np.ndarray:
+    """Standard generation (Section "Preliminaries": x_{i+1} ~ p(. | x_{1:i}), one token per evaluation of M_p),
+    written as rounds of Algorithm 1 with an empty draft: nothing is tested and the returned token is the draw
+    from p, so it shares the round counter and the random stream of the speculative rounds."""
+    ids = [int(x) for x in prompt]
+    V = model_p.shape.vocab
+    for r in range(n_new):
+        lam = model_p.logits(np.array(ids), [len(ids) - 1])
+        res = accept_resample(lam, np.zeros((0, V)), np.zeros(0), np.zeros(0, np.int64), tau_p, tau_p, seed,
+                              first_round + r, b)
+        assert res.n == 0
+        ids.append(res.t)
+    return np.array(ids, dtype=np.int64)
+
+
 # ----------------------------------------------------------------------------------
 # closed forms the paper states (Appendix "Drafter Convergence Analysis")
 # ----------------------------------------------------------------------------------

@@ -30,7 +30,7 @@ PROF_NAMES = ["gemm_drafter", "gemm_target", "head_drafter", "head_target", "att
 
 EXPORTS = [
     "sdd_workspace_bytes", "sdd_create", "sdd_draft_begin", "sdd_draft_step", "sdd_draft",
-    "sdd_verify_accept", "sdd_step", "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
+    "sdd_verify_accept", "sdd_step", "sdd_ar_step", "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
     "sdd_accept_logits_static", "sdd_debug_gemm_bf16", "sdd_debug_attention_bf16",
     "sdd_tap", "sdd_counters", "sdd_profile_begin", "sdd_profile_end", "sdd_sync_status", "sdd_destroy", "sdd_strerror", "sdd_last_cuda_error",
 ]
@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
             getattr(L, n).argtypes = [vp]
         L.sdd_verify_accept.argtypes = [vp, vp, vp]
         L.sdd_step.argtypes = [vp, vp, vp]
+        L.sdd_ar_step.argtypes = [vp, vp, vp]
         L.sdd_progress.argtypes = [vp, C.POINTER(u64), C.POINTER(i32)]
         L.sdd_accept_scratch_bytes.argtypes = [i32, i32, i32]
         L.sdd_accept_scratch_bytes.restype = u64
@@ -264,6 +265,12 @@ class Session:
 
     def sdd_step(self):
         _check(lib().sdd_step(self.h, self.out_ids.data_ptr(), self.n_out.data_ptr()), "sdd_step")
+
+    def sdd_ar_step(self):
+        """One plain autoregressive token per sequence (emitted ids in self.ar_ids [batch])."""
+        if not hasattr(self, "ar_ids"):
+            self.ar_ids = self.torch.empty(self.batch, dtype=self.torch.int32, device=self.device)
+        _check(lib().sdd_ar_step(self.h, self.ar_ids.data_ptr(), self.n_out.data_ptr()), "sdd_ar_step")
 
     def sdd_sync_status(self): _check(lib().sdd_sync_status(self.h), "sdd_sync_status")
 

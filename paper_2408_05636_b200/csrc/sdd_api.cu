@@ -430,17 +430,19 @@ static int draft_step_t(sdd_ctx* c) {
 }
 
 template <typename T>
-static int verify_accept_t(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
+static int verify_accept_t(sdd_ctx* c, int gamma, int32_t* out_ids, int32_t* n_out) {
+  // gamma = the round's draft length; gamma = 0 is plain autoregressive decoding of the target: one token is fed,
+  // nothing is tested, and the extra token is the draw from p (Algorithm 1 with an empty draft)
   const Buffers& B = c->B;
   const Dims& D = c->D;
-  SDD_TRY(forward_target<T>(c, TARGET_VERIFY, D.gamma + 1, true));
-  SDD_LAUNCH(c, CAT_STATS, launch_row_stats(B.logits_p, (long long)D.batch * (D.gamma + 1), nullptr, 0, D.V, c->inv_tau_p, 0.f,
+  SDD_TRY(forward_target<T>(c, TARGET_VERIFY, gamma + 1, true));
+  SDD_LAUNCH(c, CAT_STATS, launch_row_stats(B.logits_p, (long long)D.batch * (gamma + 1), nullptr, 0, D.V, c->inv_tau_p, 0.f,
                                  B.partial_p, c->st));
-  SDD_LAUNCH(c, CAT_ACCEPT, launch_accept(B.logits_p, B.q_logits, B.slot_ids, B.logq, B.partial_p, nullptr, D.batch, D.gamma, D.V,
+  SDD_LAUNCH(c, CAT_ACCEPT, launch_accept(B.logits_p, B.q_logits, B.slot_ids, B.logq, B.partial_p, nullptr, D.batch, gamma, D.V,
                               c->inv_tau_p, c->inv_tau_p == 0.f ? 0.f : 1.f, c->key, 0u, B.rs, B.accept_prob, B.n_accept,
                               B.extra_token, nullptr, c->st));
   SDD_LAUNCH(c, CAT_COMMIT, launch_commit(B.tokens, D.tok_stride, B.ctx_len, B.n_emitted, B.slot_ids, B.n_accept, B.extra_token,
-                              D.batch, D.gamma, D.max_new, B.rs, out_ids, n_out, c->mirror_dev, c->st));
+                              D.batch, gamma, D.max_new, B.rs, out_ids, n_out, c->mirror_dev, c->st));
   return SDD_OK;
 }
 
@@ -570,14 +572,15 @@ static int enqueue_draft_begin(sdd_ctx* c) {
 static int enqueue_draft_step(sdd_ctx* c) {
   return c->P.dtype == SDD_BF16 ? draft_step_t<__nv_bfloat16>(c) : draft_step_t<float>(c);
 }
-static int enqueue_verify_accept(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
-  return c->P.dtype == SDD_BF16 ? verify_accept_t<__nv_bfloat16>(c, out_ids, n_out) : verify_accept_t<float>(c, out_ids, n_out);
+static int enqueue_verify_accept(sdd_ctx* c, int gamma, int32_t* out_ids, int32_t* n_out) {
+  return c->P.dtype == SDD_BF16 ? verify_accept_t<__nv_bfloat16>(c, gamma, out_ids, n_out)
+                                : verify_accept_t<float>(c, gamma, out_ids, n_out);
 }
-static int round_epilogue(sdd_ctx* c) {
+static int round_epilogue(sdd_ctx* c, int max_emitted) {
   SDD_CUDA(cudaEventRecord(c->ev[c->rounds % c->ev.size()], c->st));
   c->rounds++;
   c->steps_done = -1;
-  for (auto& ub : c->c_ub) ub += c->D.gamma + 1;
+  for (auto& ub : c->c_ub) ub += max_emitted;
   return SDD_OK;
 }
 
@@ -602,8 +605,8 @@ int32_t sdd_draft(sdd_ctx* c) {
 int32_t sdd_verify_accept(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
   if (c == nullptr) return SDD_E_ARG;
   if (c->steps_done != c->D.T) return SDD_E_STATE;
-  SDD_TRY(enqueue_verify_accept(c, out_ids, n_out));
-  return round_epilogue(c);
+  SDD_TRY(enqueue_verify_accept(c, c->D.gamma, out_ids, n_out));
+  return round_epilogue(c, c->D.gamma + 1);
 }
 
 // One whole round.  Every launch parameter of a round is fixed for a given padded row count (all lengths,
@@ -627,7 +630,7 @@ int32_t sdd_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
     SDD_CUDA(cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal));
     int s = enqueue_draft_begin(c);
     for (int i = 0; i < c->D.T && s == SDD_OK; ++i) s = enqueue_draft_step(c);
-    if (s == SDD_OK) s = enqueue_verify_accept(c, out_ids, n_out);
+    if (s == SDD_OK) s = enqueue_verify_accept(c, c->D.gamma, out_ids, n_out);
     cudaGraph_t g = nullptr;
     cudaError_t e = cudaStreamEndCapture(c->st, &g);
     c->steps_done = -1;
@@ -645,7 +648,41 @@ int32_t sdd_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
   }
   SDD_CUDA(cudaGraphLaunch(it->second.exec, c->st));
   c->launches += it->second.launches;
-  return round_epilogue(c);
+  return round_epilogue(c, c->D.gamma + 1);
+}
+
+// Plain autoregressive decoding of the target (the baseline of Table 1): a round with an empty draft.
+int32_t sdd_ar_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
+  if (c == nullptr) return SDD_E_ARG;
+  if (c->steps_done != -1) return SDD_E_STATE;
+  if (c->rounds >= (uint64_t)c->runahead)
+    SDD_CUDA(cudaEventSynchronize(c->ev[(c->rounds - c->runahead) % c->ev.size()]));
+  if (!c->use_graph || c->profiling) {
+    SDD_TRY(enqueue_verify_accept(c, 0, out_ids, n_out));
+    return round_epilogue(c, 1);
+  }
+  const auto key = std::make_tuple(0, (void*)out_ids, (void*)n_out);   // row count 0 never names a SpecDiff round
+  auto it = c->graphs.find(key);
+  if (it == c->graphs.end()) {
+    const uint64_t l0 = c->launches;
+    SDD_CUDA(cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal));
+    const int s = enqueue_verify_accept(c, 0, out_ids, n_out);
+    cudaGraph_t g = nullptr;
+    cudaError_t e = cudaStreamEndCapture(c->st, &g);
+    if (s != SDD_OK) { if (g) cudaGraphDestroy(g); return s; }
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamEndCapture");
+    sdd_ctx::GraphEntry ge;
+    ge.exec = nullptr;
+    ge.launches = c->launches - l0;
+    c->launches = l0;
+    e = cudaGraphInstantiate(&ge.exec, g, 0);
+    cudaGraphDestroy(g);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGraphInstantiate");
+    it = c->graphs.emplace(key, ge).first;
+  }
+  SDD_CUDA(cudaGraphLaunch(it->second.exec, c->st));
+  c->launches += it->second.launches;
+  return round_epilogue(c, 1);
 }
 
 int32_t sdd_progress(sdd_ctx* c, uint64_t* rounds_done, int32_t* min_emitted) {

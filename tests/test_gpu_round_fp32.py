@@ -126,3 +126,35 @@ def test_cache_skip_changes_nothing(monkeypatch):
         s.close()
     assert np.array_equal(outs[0][1], outs[1][1]) and np.array_equal(outs[0][0], outs[1][0])
     assert outs[0][1].min() > wl.prompt_len - 13
+
+
+def test_autoregressive_steps_match_oracle_and_mix_with_rounds():
+    """sdd_ar_step = a round with an empty draft: tokens must equal the oracle's, also when interleaved with
+    speculative rounds (shared round counter and KV cache)."""
+    import paper_2408_05636_b200 as sdd
+    wl = synth.WORKLOADS["tiny_fp32"]
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 2, wl.prompt_len, wl.prompt_seed)
+    plen = [wl.prompt_len, 9]
+    s = sdd.Session(dp, dq, prompts, plen, wl.gamma, wl.T, 60, 1.0, 1.0, wl.philox_seed)
+    for _ in range(5):
+        s.sdd_ar_step()
+    s.sdd_sync_status()
+    toks = s.tap_numpy(sdd.TAP_TOKENS).reshape(2, -1)
+    clen = s.tap_numpy(sdd.TAP_CTX_LEN)
+    for b in range(2):
+        ref = sd.autoregressive_sample(mp, prompts[b, : plen[b]], 5, 1.0, wl.philox_seed, b=b)
+        assert clen[b] == plen[b] + 5 and np.array_equal(toks[b, : clen[b]], ref)
+    assert list(s.ar_ids.cpu().numpy()) == [int(toks[b, clen[b] - 1]) for b in range(2)]
+    # speculative rounds continue from there (rounds 5, 6), then one more plain token (round 7)
+    log, stats = roundcheck.check_rounds(s, mp, mq, wl, 2, 1.0, 1.0, TOL, first_round=5)
+    assert len(log) <= 1
+    before = s.tap_numpy(sdd.TAP_CTX_LEN).copy()
+    toks_before = s.tap_numpy(sdd.TAP_TOKENS).reshape(2, -1).copy()
+    s.sdd_ar_step()
+    s.sdd_sync_status()
+    toks = s.tap_numpy(sdd.TAP_TOKENS).reshape(2, -1)
+    for b in range(2):
+        ref = sd.autoregressive_sample(mp, toks_before[b, : before[b]], 1, 1.0, wl.philox_seed, b=b, first_round=7)
+        assert toks[b, before[b]] == ref[-1]
+    s.close()

@@ -143,3 +143,21 @@ def test_generate_bookkeeping_stochastic():
     # same seed -> same output; another seed -> (almost surely) another
     ids2, _ = sd.generate(mp, mq, [1, 2], 3, 2, 7, 1.0, 1.0, 5)
     assert np.array_equal(ids, ids2)
+
+
+def test_autoregressive_sampling_is_a_round_with_an_empty_draft():
+    mp, mq = _tiny_pair(V=5, seed=41, std=0.25)
+    ctx = np.array([1, 4, 2])
+    p1 = _softmax(mp.logits(ctx, [2])[0])
+    N = 2500
+    counts = np.zeros(5)
+    for rnd in range(N):
+        counts[sd.autoregressive_sample(mp, ctx, 1, 1.0, 9, first_round=rnd)[-1]] += 1
+    assert stats.chisquare(counts, p1 * N).pvalue > 1e-3          # the draw follows the target distribution
+    # greedy limit: identical to arg-max decoding
+    assert np.array_equal(sd.autoregressive_sample(mp, ctx, 6, 0.0, 9), sd.autoregressive_greedy(mp, ctx, 6))
+    # the draw is the bonus stream at slot 0 of the round
+    from oracle import philox as px
+    lam = mp.logits(ctx, [2])[0]
+    g = px.vocab_gumbels(9, px.BONUS, 7, 0, 0, 0, 5)
+    assert sd.autoregressive_sample(mp, ctx, 1, 1.0, 9, first_round=7)[-1] == int(np.argmax(lam + g))
