@@ -20,6 +20,8 @@
 // still has in flight, TMEM is freed and the CTA returns.
 #include <cudaTypedefs.h>
 
+#include <cstdlib>
+
 #include <map>
 #include <mutex>
 #include <tuple>
@@ -50,6 +52,211 @@ constexpr int ring_stages() {
 template <int BN, bool SWAP, bool HILO, bool DEEP>
 constexpr int smem_bytes() {
   return ring_stages<BN, SWAP, HILO, DEEP>() * stage_bytes<BN, SWAP, HILO>() + 1024 /*alignment slack*/ + 256 /*barriers*/;
+}
+
+// ---------------------------------------------------------------------------------------------
+// epilogues (shared by the one-tile and the persistent kernel); called by the four epilogue warps, q = TMEM lane
+// quarter of the calling warp, tmem_acc = first column of the tile's accumulator
+// ---------------------------------------------------------------------------------------------
+template <int BN>
+__device__ __forceinline__ void epilogue_tma(uint32_t tmem_acc, int m0, int n0, int q, int lane, int epi,
+                                             const float* __restrict__ bias, int rows_b, const CUtensorMap* map_out,
+                                             uint8_t* stage_generic, uint32_t stage_u32, int& n_store) {
+  // Output through shared memory and TMA: every thread writes its row's 128-byte piece of the tile into a
+  // staging buffer (128-byte swizzle, so that the 32 rows of a warp spread over all banks), one thread issues a
+  // tile store (bf16 outputs) or an add-reduce (fp32 residual stream; also correct under K splits).  The operand
+  // ring is free by now: tmem_full completes only after every MMA has read its stage.
+  const int rl = q * 32 + lane;               // row inside the tile
+  const int sw = rl & 7;
+  const bool is_issuer = threadIdx.x == 64;
+  const bool f32 = epi == EPI_RESIDUAL;
+  constexpr int CHUNKS = BN / 32;
+  #pragma unroll 1
+  for (int cc = 0; cc < CHUNKS; ++cc) {
+    uint32_t v[32];
+    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
+    const int c0 = n0 + cc * 32;
+    // fp32: one 32-column chunk fills a 128-byte row; bf16: two chunks do
+    const int buf = f32 ? (cc & 1) : ((cc >> 1) & 1);
+    const bool first_of_buf = f32 || (cc & 1) == 0;
+    const bool last_of_buf = f32 || (cc & 1) == 1 || cc == CHUNKS - 1;
+    if (first_of_buf) {
+      if (is_issuer && n_store >= 2) tma_wait_group_read<1>();   // the store that last used this buffer has read it
+      named_bar_sync(2, 128);
+    }
+    uint8_t* row = stage_generic + buf * (128 * 128) + rl * 128;
+    if (f32) {
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
+        float4 x;
+        x.x = __uint_as_float(v[g * 4 + 0]) + ((bias && c0 + g * 4 + 0 < rows_b) ? bias[c0 + g * 4 + 0] : 0.f);
+        x.y = __uint_as_float(v[g * 4 + 1]) + ((bias && c0 + g * 4 + 1 < rows_b) ? bias[c0 + g * 4 + 1] : 0.f);
+        x.z = __uint_as_float(v[g * 4 + 2]) + ((bias && c0 + g * 4 + 2 < rows_b) ? bias[c0 + g * 4 + 2] : 0.f);
+        x.w = __uint_as_float(v[g * 4 + 3]) + ((bias && c0 + g * 4 + 3 < rows_b) ? bias[c0 + g * 4 + 3] : 0.f);
+        *reinterpret_cast<float4*>(row + ((g ^ sw) << 4)) = x;
+      }
+    } else {
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int j0 = g * 8 + 2 * e;
+          float x0 = __uint_as_float(v[j0]) + ((bias && c0 + j0 < rows_b) ? bias[c0 + j0] : 0.f);
+          float x1 = __uint_as_float(v[j0 + 1]) + ((bias && c0 + j0 + 1 < rows_b) ? bias[c0 + j0 + 1] : 0.f);
+          if (epi == EPI_GELU) { x0 = gelu_tanh_fast(x0); x1 = gelu_tanh_fast(x1); }
+          __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+          pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+        }
+        const int chunk = (cc & 1) * 4 + g;
+        *reinterpret_cast<uint4*>(row + ((chunk ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      }
+    }
+    if (last_of_buf) {
+      fence_async_smem();
+      named_bar_sync(2, 128);
+      if (is_issuer) {
+        const uint32_t src = stage_u32 + buf * (128 * 128);
+        if (f32) tma_reduce_add_2d(map_out, src, c0, m0);
+        else tma_store_2d(map_out, src, n0 + (cc & ~1) * 32, m0);
+        tma_commit_group();
+      }
+      ++n_store;
+    }
+  }
+}
+
+template <int BN, bool SWAP>
+__device__ __forceinline__ void epilogue_manual(uint32_t tmem_acc, int m0, int n0, int q, int lane, int rows_a, int rows_b,
+                                                int epi, const float* __restrict__ bias, void* __restrict__ out,
+                                                void* __restrict__ out_lo, int ldc, bool split, const QkvDst& qd) {
+  const int r = m0 + q * 32 + lane;          // index along the A operand's rows
+  const bool r_ok = r < rows_a;
+#pragma unroll 1
+  for (int cc = 0; cc < BN / 32; ++cc) {
+    uint32_t v[32];
+    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
+    const int c0 = n0 + cc * 32;             // index along the B operand's rows
+    if (!SWAP) {
+      // out[r][c]: r = token row, c = feature
+      if (r_ok && epi == EPI_QKV && c0 >= 2 * qd.d) {
+        // V chunk of token row r: transposed store, consecutive lanes = consecutive positions
+        const int sb = r / qd.rows_per_seq, si = r - sb * qd.rows_per_seq;
+        const int cl = qd.ctx_len[sb];
+        const int pos = qd.mode == 1 ? cl - 1 + si : si;
+        if ((qd.mode != 2 || si < cl - 1) && pos < qd.vt_ld) {
+          __nv_bfloat16* vt = qd.vt_dst + ((long long)sb * qd.d + (c0 - 2 * qd.d)) * qd.vt_ld + pos;
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c0 + j < rows_b) vt[(long long)j * qd.vt_ld] = __float2bfloat16_rn(__uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f));
+        }
+      } else if (r_ok && epi == EPI_QKV && c0 >= qd.d && qd.k_dst != nullptr) {
+        const int sb = r / qd.rows_per_seq, si = r - sb * qd.rows_per_seq;
+        const int cl = qd.ctx_len[sb];
+        const int pos = qd.mode == 1 ? cl - 1 + si : si;
+        if ((qd.mode != 2 || si < cl - 1) && pos < qd.k_seq_rows) {
+          __nv_bfloat16* kd = qd.k_dst + ((long long)sb * qd.k_seq_rows + pos) * qd.d + (c0 - qd.d);
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c0 + j < rows_b) kd[j] = __float2bfloat16_rn(__uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f));
+        }
+      } else if (r_ok) {
+        if (epi == EPI_STORE || epi == EPI_GELU || epi == EPI_QKV) {
+          __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + (long long)r * ldc + c0;
+          if (c0 + 32 <= rows_b && (ldc & 7) == 0) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint32_t pk[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                float x0 = __uint_as_float(v[g * 8 + 2 * e]) + (bias ? bias[c0 + g * 8 + 2 * e] : 0.f);
+                float x1 = __uint_as_float(v[g * 8 + 2 * e + 1]) + (bias ? bias[c0 + g * 8 + 2 * e + 1] : 0.f);
+                if (epi == EPI_GELU) { x0 = gelu_tanh_fast(x0); x1 = gelu_tanh_fast(x1); }
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+                pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(o + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+            if (out_lo != nullptr) {   // second half of the hi/lo pair: lo = bf16(x - hi)
+              __nv_bfloat16* ol = reinterpret_cast<__nv_bfloat16*>(out_lo) + (long long)r * ldc + c0;
+              for (int j = 0; j < 32; ++j) {
+                float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
+                if (epi == EPI_GELU) x = gelu_tanh_fast(x);
+                ol[j] = __float2bfloat16_rn(x - __bfloat162float(__float2bfloat16_rn(x)));
+              }
+            }
+          } else {
+            for (int j = 0; j < 32; ++j) {
+              if (c0 + j < rows_b) {
+                float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
+                if (epi == EPI_GELU) x = gelu_tanh_fast(x);
+                const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                o[j] = hi;
+                if (out_lo != nullptr)
+                  reinterpret_cast<__nv_bfloat16*>(out_lo)[(long long)r * ldc + c0 + j] = __float2bfloat16_rn(x - __bfloat162float(hi));
+              }
+            }
+          }
+        } else {
+          float* o = reinterpret_cast<float*>(out) + (long long)r * ldc + c0;
+          if (epi == EPI_RESIDUAL && !split && c0 + 32 <= rows_b && (ldc & 3) == 0) {
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+              float4 h4 = *reinterpret_cast<float4*>(o + g * 4);
+              h4.x += __uint_as_float(v[g * 4 + 0]) + (bias ? bias[c0 + g * 4 + 0] : 0.f);
+              h4.y += __uint_as_float(v[g * 4 + 1]) + (bias ? bias[c0 + g * 4 + 1] : 0.f);
+              h4.z += __uint_as_float(v[g * 4 + 2]) + (bias ? bias[c0 + g * 4 + 2] : 0.f);
+              h4.w += __uint_as_float(v[g * 4 + 3]) + (bias ? bias[c0 + g * 4 + 3] : 0.f);
+              *reinterpret_cast<float4*>(o + g * 4) = h4;
+            }
+          } else {
+            for (int j = 0; j < 32; ++j) {
+              if (c0 + j < rows_b) {
+                const float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
+                if (epi == EPI_RESIDUAL) { if (split) atomicAdd(o + j, x); else o[j] += x; }
+                else o[j] = x;
+              }
+            }
+          }
+        }
+      }
+    } else {
+      // out[c][r]: c = token, r = feature; consecutive lanes write consecutive features
+      const float bv = (bias != nullptr && r_ok) ? bias[r] : 0.f;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const int c = c0 + j;
+        if (r_ok && c < rows_b) {
+          float x = __uint_as_float(v[j]) + bv;
+          const long long o = (long long)c * ldc + r;
+          if (epi == EPI_QKV) {
+            if (r < qd.d || (r < 2 * qd.d && qd.k_dst == nullptr)) {
+              reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(x);
+            } else {
+              const int sb = c / qd.rows_per_seq, si = c - sb * qd.rows_per_seq;
+              const int cl = qd.ctx_len[sb];
+              const int pos = qd.mode == 1 ? cl - 1 + si : si;
+              if (qd.mode != 2 || si < cl - 1) {
+                if (r < 2 * qd.d) {
+                  if (pos < qd.k_seq_rows)
+                    qd.k_dst[((long long)sb * qd.k_seq_rows + pos) * qd.d + (r - qd.d)] = __float2bfloat16_rn(x);
+                } else if (pos < qd.vt_ld) {
+                  qd.vt_dst[((long long)sb * qd.d + (r - 2 * qd.d)) * qd.vt_ld + pos] = __float2bfloat16_rn(x);
+                }
+              }
+            }
+          } else if (epi == EPI_STORE || epi == EPI_GELU) {
+            if (epi == EPI_GELU) x = gelu_tanh_fast(x);
+            const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+            reinterpret_cast<__nv_bfloat16*>(out)[o] = hi;
+            if (out_lo != nullptr) reinterpret_cast<__nv_bfloat16*>(out_lo)[o] = __float2bfloat16_rn(x - __bfloat162float(hi));
+          }
+          else if (epi == EPI_RESIDUAL) { if (split) atomicAdd(reinterpret_cast<float*>(out) + o, x); else reinterpret_cast<float*>(out)[o] += x; }
+          else reinterpret_cast<float*>(out)[o] = x;
+        }
+      }
+    }
+  }
 }
 
 // grid = (N tiles, M tiles, K splits).  With more than one K split every CTA accumulates its share of the K
@@ -166,198 +373,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const bool ready = named_bar_and(1, 128, mbar_wait(tmem_full_bar, 0u, abort_flag, status));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ready && !SWAP && tma_out) {
-      // Output through shared memory and TMA: every thread writes its row's 128-byte piece of the tile into a
-      // staging buffer (128-byte swizzle, so that the 32 rows of a warp spread over all banks), one thread issues a
-      // tile store (bf16 outputs) or an add-reduce (fp32 residual stream; also correct under K splits).  The operand
-      // ring is free by now: tmem_full completes only after every MMA has read its stage.
-      const int rl = q * 32 + lane;               // row inside the tile
-      const int sw = rl & 7;
-      const bool is_issuer = threadIdx.x == 64;
-      const bool f32 = epi == EPI_RESIDUAL;
-      constexpr int CHUNKS = BN / 32;
       int n_store = 0;
-#pragma unroll 1
-      for (int cc = 0; cc < CHUNKS; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
-        const int c0 = n0 + cc * 32;
-        // fp32: one 32-column chunk fills a 128-byte row; bf16: two chunks do
-        const int buf = f32 ? (cc & 1) : ((cc >> 1) & 1);
-        const bool first_of_buf = f32 || (cc & 1) == 0;
-        const bool last_of_buf = f32 || (cc & 1) == 1 || cc == CHUNKS - 1;
-        if (first_of_buf) {
-          if (is_issuer && n_store >= 2) tma_wait_group_read<1>();   // the store that last used this buffer has read it
-          named_bar_sync(2, 128);
-        }
-        uint8_t* row = generic_base + buf * (128 * 128) + rl * 128;
-        if (f32) {
-#pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            float4 x;
-            x.x = __uint_as_float(v[g * 4 + 0]) + ((bias && c0 + g * 4 + 0 < rows_b) ? bias[c0 + g * 4 + 0] : 0.f);
-            x.y = __uint_as_float(v[g * 4 + 1]) + ((bias && c0 + g * 4 + 1 < rows_b) ? bias[c0 + g * 4 + 1] : 0.f);
-            x.z = __uint_as_float(v[g * 4 + 2]) + ((bias && c0 + g * 4 + 2 < rows_b) ? bias[c0 + g * 4 + 2] : 0.f);
-            x.w = __uint_as_float(v[g * 4 + 3]) + ((bias && c0 + g * 4 + 3 < rows_b) ? bias[c0 + g * 4 + 3] : 0.f);
-            *reinterpret_cast<float4*>(row + ((g ^ sw) << 4)) = x;
-          }
-        } else {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint32_t pk[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int j0 = g * 8 + 2 * e;
-              float x0 = __uint_as_float(v[j0]) + ((bias && c0 + j0 < rows_b) ? bias[c0 + j0] : 0.f);
-              float x1 = __uint_as_float(v[j0 + 1]) + ((bias && c0 + j0 + 1 < rows_b) ? bias[c0 + j0 + 1] : 0.f);
-              if (epi == EPI_GELU) { x0 = gelu_tanh_fast(x0); x1 = gelu_tanh_fast(x1); }
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
-              pk[e] = *reinterpret_cast<uint32_t*>(&h2);
-            }
-            const int chunk = (cc & 1) * 4 + g;
-            *reinterpret_cast<uint4*>(row + ((chunk ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-          }
-        }
-        if (last_of_buf) {
-          fence_async_smem();
-          named_bar_sync(2, 128);
-          if (is_issuer) {
-            const uint32_t src = base + buf * (128 * 128);
-            if (f32) tma_reduce_add_2d(&map_out, src, c0, m0);
-            else tma_store_2d(&map_out, src, n0 + (cc & ~1) * 32, m0);
-            tma_commit_group();
-          }
-          ++n_store;
-        }
-      }
-      if (is_issuer) tma_wait_group_read<0>();      // shared memory stays valid until the copies have read it
+      epilogue_tma<BN>(tmem_base, m0, n0, q, lane, epi, bias, rows_b, &map_out, generic_base, base, n_store);
+      if (threadIdx.x == 64) tma_wait_group_read<0>();      // shared memory stays valid until the copies have read it
     } else if (ready) {
-      const int r = m0 + q * 32 + lane;          // index along the A operand's rows
-      const bool r_ok = r < rows_a;
-#pragma unroll 1
-      for (int cc = 0; cc < BN / 32; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
-        const int c0 = n0 + cc * 32;             // index along the B operand's rows
-        if (!SWAP) {
-          // out[r][c]: r = token row, c = feature
-          if (r_ok && epi == EPI_QKV && c0 >= 2 * qd.d) {
-            // V chunk of token row r: transposed store, consecutive lanes = consecutive positions
-            const int sb = r / qd.rows_per_seq, si = r - sb * qd.rows_per_seq;
-            const int cl = qd.ctx_len[sb];
-            const int pos = qd.mode == 1 ? cl - 1 + si : si;
-            if ((qd.mode != 2 || si < cl - 1) && pos < qd.vt_ld) {
-              __nv_bfloat16* vt = qd.vt_dst + ((long long)sb * qd.d + (c0 - 2 * qd.d)) * qd.vt_ld + pos;
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (c0 + j < rows_b) vt[(long long)j * qd.vt_ld] = __float2bfloat16_rn(__uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f));
-            }
-          } else if (r_ok && epi == EPI_QKV && c0 >= qd.d && qd.k_dst != nullptr) {
-            const int sb = r / qd.rows_per_seq, si = r - sb * qd.rows_per_seq;
-            const int cl = qd.ctx_len[sb];
-            const int pos = qd.mode == 1 ? cl - 1 + si : si;
-            if ((qd.mode != 2 || si < cl - 1) && pos < qd.k_seq_rows) {
-              __nv_bfloat16* kd = qd.k_dst + ((long long)sb * qd.k_seq_rows + pos) * qd.d + (c0 - qd.d);
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (c0 + j < rows_b) kd[j] = __float2bfloat16_rn(__uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f));
-            }
-          } else if (r_ok) {
-            if (epi == EPI_STORE || epi == EPI_GELU || epi == EPI_QKV) {
-              __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + (long long)r * ldc + c0;
-              if (c0 + 32 <= rows_b && (ldc & 7) == 0) {
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                  uint32_t pk[4];
-#pragma unroll
-                  for (int e = 0; e < 4; ++e) {
-                    float x0 = __uint_as_float(v[g * 8 + 2 * e]) + (bias ? bias[c0 + g * 8 + 2 * e] : 0.f);
-                    float x1 = __uint_as_float(v[g * 8 + 2 * e + 1]) + (bias ? bias[c0 + g * 8 + 2 * e + 1] : 0.f);
-                    if (epi == EPI_GELU) { x0 = gelu_tanh_fast(x0); x1 = gelu_tanh_fast(x1); }
-                    __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
-                    pk[e] = *reinterpret_cast<uint32_t*>(&h2);
-                  }
-                  *reinterpret_cast<uint4*>(o + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                }
-                if (out_lo != nullptr) {   // second half of the hi/lo pair: lo = bf16(x - hi)
-                  __nv_bfloat16* ol = reinterpret_cast<__nv_bfloat16*>(out_lo) + (long long)r * ldc + c0;
-                  for (int j = 0; j < 32; ++j) {
-                    float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
-                    if (epi == EPI_GELU) x = gelu_tanh_fast(x);
-                    ol[j] = __float2bfloat16_rn(x - __bfloat162float(__float2bfloat16_rn(x)));
-                  }
-                }
-              } else {
-                for (int j = 0; j < 32; ++j) {
-                  if (c0 + j < rows_b) {
-                    float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
-                    if (epi == EPI_GELU) x = gelu_tanh_fast(x);
-                    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-                    o[j] = hi;
-                    if (out_lo != nullptr)
-                      reinterpret_cast<__nv_bfloat16*>(out_lo)[(long long)r * ldc + c0 + j] = __float2bfloat16_rn(x - __bfloat162float(hi));
-                  }
-                }
-              }
-            } else {
-              float* o = reinterpret_cast<float*>(out) + (long long)r * ldc + c0;
-              if (epi == EPI_RESIDUAL && !split && c0 + 32 <= rows_b && (ldc & 3) == 0) {
-#pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                  float4 h4 = *reinterpret_cast<float4*>(o + g * 4);
-                  h4.x += __uint_as_float(v[g * 4 + 0]) + (bias ? bias[c0 + g * 4 + 0] : 0.f);
-                  h4.y += __uint_as_float(v[g * 4 + 1]) + (bias ? bias[c0 + g * 4 + 1] : 0.f);
-                  h4.z += __uint_as_float(v[g * 4 + 2]) + (bias ? bias[c0 + g * 4 + 2] : 0.f);
-                  h4.w += __uint_as_float(v[g * 4 + 3]) + (bias ? bias[c0 + g * 4 + 3] : 0.f);
-                  *reinterpret_cast<float4*>(o + g * 4) = h4;
-                }
-              } else {
-                for (int j = 0; j < 32; ++j) {
-                  if (c0 + j < rows_b) {
-                    const float x = __uint_as_float(v[j]) + (bias ? bias[c0 + j] : 0.f);
-                    if (epi == EPI_RESIDUAL) { if (split) atomicAdd(o + j, x); else o[j] += x; }
-                    else o[j] = x;
-                  }
-                }
-              }
-            }
-          }
-        } else {
-          // out[c][r]: c = token, r = feature; consecutive lanes write consecutive features
-          const float bv = (bias != nullptr && r_ok) ? bias[r] : 0.f;
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int c = c0 + j;
-            if (r_ok && c < rows_b) {
-              float x = __uint_as_float(v[j]) + bv;
-              const long long o = (long long)c * ldc + r;
-              if (epi == EPI_QKV) {
-                if (r < qd.d || (r < 2 * qd.d && qd.k_dst == nullptr)) {
-                  reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(x);
-                } else {
-                  const int sb = c / qd.rows_per_seq, si = c - sb * qd.rows_per_seq;
-                  const int cl = qd.ctx_len[sb];
-                  const int pos = qd.mode == 1 ? cl - 1 + si : si;
-                  if (qd.mode != 2 || si < cl - 1) {
-                    if (r < 2 * qd.d) {
-                      if (pos < qd.k_seq_rows)
-                        qd.k_dst[((long long)sb * qd.k_seq_rows + pos) * qd.d + (r - qd.d)] = __float2bfloat16_rn(x);
-                    } else if (pos < qd.vt_ld) {
-                      qd.vt_dst[((long long)sb * qd.d + (r - 2 * qd.d)) * qd.vt_ld + pos] = __float2bfloat16_rn(x);
-                    }
-                  }
-                }
-              } else if (epi == EPI_STORE || epi == EPI_GELU) {
-                if (epi == EPI_GELU) x = gelu_tanh_fast(x);
-                const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-                reinterpret_cast<__nv_bfloat16*>(out)[o] = hi;
-                if (out_lo != nullptr) reinterpret_cast<__nv_bfloat16*>(out_lo)[o] = __float2bfloat16_rn(x - __bfloat162float(hi));
-              }
-              else if (epi == EPI_RESIDUAL) { if (split) atomicAdd(reinterpret_cast<float*>(out) + o, x); else reinterpret_cast<float*>(out)[o] += x; }
-              else reinterpret_cast<float*>(out)[o] = x;
-            }
-          }
-        }
-      }
+      epilogue_manual<BN, SWAP>(tmem_base, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, split, qd);
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -365,6 +385,155 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Persistent variant for grids of many tiles (NORMAL orientation): one CTA per SM walks over tiles
+// (tile = blockIdx.x, + gridDim.x, ...; the N index runs fastest when W fits well into L2, so that the CTAs running
+// at one time share few A tiles and every A tile comes from DRAM once; else the M index runs fastest).  Two
+// accumulators live in TMEM, so the MMA warp fills one while the epilogue warps drain the other; the operand ring
+// runs on across tile boundaries.  Extra barriers: tmem_full[2] (MMA -> epilogue), tmem_empty[2] (epilogue -> MMA).
+// ---------------------------------------------------------------------------------------------
+template <int BN, bool HILO>
+constexpr int persist_stages() {
+  constexpr int s = (227 * 1024 - 2 * 128 * 128 - 1024 - 1024 - 512) / stage_bytes<BN, false, HILO>();
+  return s > 8 ? 8 : s;
+}
+template <int BN, bool HILO>
+constexpr int persist_smem_bytes() {
+  return persist_stages<BN, HILO>() * stage_bytes<BN, false, HILO>() + 2 * 128 * 128 + 1024 + 512;
+}
+
+template <int BN, bool HILO>
+__global__ void __launch_bounds__(THREADS)
+gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                       const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_out, int tma_out,
+                       int rows_a, int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out,
+                       void* __restrict__ out_lo, int ldc, int* status, const QkvDst qd, const int* __restrict__ skip,
+                       int tiles_m, int tiles_n, int n_fastest) {
+  constexpr int STAGES = persist_stages<BN, HILO>();
+  constexpr int STAGE_BYTES = stage_bytes<BN, false, HILO>();
+  constexpr int LO_OFF = BM * BK * 2 + BN * BK * 2;
+  constexpr int STAGING_OFF = STAGES * STAGE_BYTES;
+  constexpr int BAR_OFF = STAGING_OFF + 2 * 128 * 128;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* generic_base = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bar_base = base + BAR_OFF;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(generic_base + BAR_OFF + 8 * (2 * STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(generic_base + BAR_OFF + 8 * (2 * STAGES + 4) + 8);
+  constexpr uint32_t TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = (K + BK - 1) / BK;
+  const int n_tiles = tiles_m * tiles_n;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 128); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+  pdl_launch_dependents();
+  const bool active = skip == nullptr || *skip == 0;
+
+  if (!active) {
+  } else if (warp == 0) {
+    if (lane == 0) {
+      long long it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int m0 = (n_fastest ? tile / tiles_n : tile % tiles_m) * BM;
+        const int n0 = (n_fastest ? tile % tiles_n : tile / tiles_m) * BN;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = (int)(it % STAGES);
+          const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, status)) { ok = false; break; }
+          mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES);
+          const uint32_t sa = base + s * STAGE_BYTES;
+          tma_load_2d(sa, &map_a, full_bar(s), kb * BK, m0);
+          tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), kb * BK, n0);
+          if (HILO) tma_load_2d(sa + LO_OFF, &map_lo, full_bar(s), kb * BK, m0);
+        }
+      }
+      if (*abort_flag) {
+        // do not leave while copies into this CTA's shared memory may still be in flight
+        for (long long j = it > STAGES ? it - STAGES : 0; j < it; ++j) {
+          const long long t0 = clock64();
+          while (!mbar_try(full_bar((int)(j % STAGES)), (uint32_t)(j / STAGES) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc<BN>();
+      long long it = 0;
+      int i = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++i) {
+        const int buf = i & 1;
+        ok = mbar_wait(tempty_bar(buf), ((uint32_t)(i >> 1) & 1u) ^ 1u, abort_flag, status);   // accumulator drained
+        if (!ok) break;
+        fence_after_sync();
+        const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = (int)(it % STAGES);
+          ok = mbar_wait(full_bar(s), (uint32_t)(it / STAGES) & 1u, abort_flag, status);
+          if (!ok) break;
+          fence_after_sync();
+          const uint32_t sa = base + s * STAGE_BYTES;
+          const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + BM * BK * 2);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma(acc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          if (HILO) {
+            const uint64_t dl = make_smem_desc(sa + LO_OFF);
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k)
+              umma(acc, dl + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc, 1u);
+          }
+          umma_commit(empty_bar(s));
+        }
+        if (ok) umma_commit(tfull_bar(buf));
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    int n_store = 0, i = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++i) {
+      const int buf = i & 1;
+      const int m0 = (n_fastest ? tile / tiles_n : tile % tiles_m) * BM;
+      const int n0 = (n_fastest ? tile % tiles_n : tile / tiles_m) * BN;
+      const bool ready = named_bar_and(1, 128, mbar_wait(tfull_bar(buf), (uint32_t)(i >> 1) & 1u, abort_flag, status));
+      if (!ready) break;
+      fence_after_sync();
+      const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
+      if (tma_out)
+        epilogue_tma<BN>(acc, m0, n0, q, lane, epi, bias, rows_b, &map_out, generic_base + STAGING_OFF, base + STAGING_OFF, n_store);
+      else
+        epilogue_manual<BN, false>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, false, qd);
+      // this thread's reads of the accumulator are complete (tcgen05.wait::ld inside tmem_ld32): hand it back
+      fence_before_sync();
+      mbar_arrive(tempty_bar(buf));
+    }
+    if (threadIdx.x == 64) tma_wait_group_read<0>();      // staging memory stays valid until the copies have read it
+  }
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    fence_after_sync();
+    tmem_dealloc(tmem_base, TMEM_COLS);
   }
 }
 
@@ -392,6 +561,19 @@ static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, cons
   return launch_cfg2<BN, SWAP, HILO, true>(ma, mb, ml, mo, tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, st,
                                            qd, splits, skip);
 }
+template <int BN, bool HILO>
+static cudaError_t launch_persist(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& mo,
+                                  int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias, void* out,
+                                  void* out_lo, int ldc, int* status, cudaStream_t st, const QkvDst& qd, const int* skip) {
+  const int tiles_m = (rows_a + BM - 1) / BM, tiles_n = (rows_b + BN - 1) / BN;
+  const long long tiles = (long long)tiles_m * tiles_n;
+  const unsigned grid = (unsigned)(tiles < 148 ? tiles : 148);
+  launch_k(gemm_tc_persist_kernel<BN, HILO>, dim3(grid), dim3(THREADS), persist_smem_bytes<BN, HILO>(), st, ma, mb, ml, mo,
+           tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n,
+           (long long)rows_b * K * 2 <= (48ll << 20) ? 1 : 0);
+  return cudaGetLastError();
+}
+
 template <int BN, bool SWAP>
 static cudaError_t launch_hl(bool hilo, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml,
                              const CUtensorMap& mo, int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias,
@@ -425,7 +607,11 @@ cudaError_t tc_prepare_gemm() {
   if ((e = prepare_one<128, false>()) != cudaSuccess) return e;
   if ((e = prepare_one<256, false>()) != cudaSuccess) return e;
   if ((e = prepare_one<32, true>()) != cudaSuccess) return e;
-  return prepare_one<64, true>();
+  if ((e = prepare_one<64, true>()) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_persist_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                persist_smem_bytes<256, false>())) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_tc_persist_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              persist_smem_bytes<256, true>());
 }
 
 static PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
@@ -530,6 +716,13 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
              (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
     if ((e = get_tensor_map(out, M, N, ldc, BM, 64, &mo, 2)) != cudaSuccess) return e;
     tma_out = 1;
+  }
+  // many 256-wide tiles and no K split: the persistent kernel (SDD_GEMM_PERSIST=0 switches it off)
+  static const bool persist_on = [] { const char* e = getenv("SDD_GEMM_PERSIST"); return e == nullptr || atoi(e) != 0; }();
+  if (persist_on && bn == 256 && splits == 1 && mt * ((N + 255) / 256) > 2 * SMS) {
+    if (hilo)
+      return launch_persist<256, true>(ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, skip);
+    return launch_persist<256, false>(ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, skip);
   }
   switch (bn) {
     case 256: return launch_hl<256, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);

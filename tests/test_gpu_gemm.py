@@ -24,6 +24,8 @@ CASES = [
     # M, N, K, n_tile
     (128, 128, 64, 128), (128, 256, 128, 256), (300, 200, 192, 64), (257, 96, 768, 32), (384, 2304, 768, 0),
     (400, 768, 3072, 0), (130, 50257, 128, 128),
+    # many tiles: the persistent kernel with two TMEM accumulators (ragged M and N)
+    (8200, 2000, 192, 0), (5000, 4096, 1024, 0),
     # swapped orientation: M <= 64 rows
     (1, 128, 64, 0), (17, 768, 3072, 0), (17, 2304, 768, 0), (33, 1600, 1600, 0), (64, 777, 256, 0), (17, 50257, 768, 0),
 ]
