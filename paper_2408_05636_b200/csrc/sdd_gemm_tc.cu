@@ -51,21 +51,29 @@ constexpr int ring_stages() {
 }
 template <int BN, bool SWAP, bool HILO, bool DEEP>
 constexpr int smem_bytes() {
-  return ring_stages<BN, SWAP, HILO, DEEP>() * stage_bytes<BN, SWAP, HILO>() + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  return ring_stages<BN, SWAP, HILO, DEEP>() * stage_bytes<BN, SWAP, HILO>() + 1024 /*alignment slack*/ + 256 /*barriers*/ +
+         1024 /*bias*/;
 }
 
 // ---------------------------------------------------------------------------------------------
 // epilogues (shared by the one-tile and the persistent kernel); called by the four epilogue warps, q = TMEM lane
 // quarter of the calling warp, tmem_acc = first column of the tile's accumulator
 // ---------------------------------------------------------------------------------------------
+// the four epilogue warps copy the tile's bias values to shared memory (zero past column N or without a bias)
+template <int BN>
+__device__ __forceinline__ void stage_bias(float* bias_s, const float* __restrict__ bias, int n0, int rows_b) {
+  for (int c = (int)threadIdx.x - 64; c < BN; c += 128) bias_s[c] = (bias != nullptr && n0 + c < rows_b) ? bias[n0 + c] : 0.f;
+  named_bar_sync(2, 128);
+}
+
 template <int BN>
 __device__ __forceinline__ void epilogue_tma(uint32_t tmem_acc, int m0, int n0, int q, int lane, int epi,
-                                             const float* __restrict__ bias, int rows_b, const CUtensorMap* map_out,
+                                             const float* bias_s, const CUtensorMap* map_out,
                                              uint8_t* stage_generic, uint32_t stage_u32, int& n_store) {
   // Output through shared memory and TMA: every thread writes its row's 128-byte piece of the tile into a
   // staging buffer (128-byte swizzle, so that the 32 rows of a warp spread over all banks), one thread issues a
-  // tile store (bf16 outputs) or an add-reduce (fp32 residual stream; also correct under K splits).  The operand
-  // ring is free by now: tmem_full completes only after every MMA has read its stage.
+  // tile store (bf16 outputs) or an add-reduce (fp32 residual stream; also correct under K splits).
+  // bias_s: the tile's BN bias values in shared memory (zeros where there is no bias or no column).
   const int rl = q * 32 + lane;               // row inside the tile
   const int sw = rl & 7;
   const bool is_issuer = threadIdx.x == 64;
@@ -89,10 +97,10 @@ __device__ __forceinline__ void epilogue_tma(uint32_t tmem_acc, int m0, int n0, 
 #pragma unroll
       for (int g = 0; g < 8; ++g) {
         float4 x;
-        x.x = __uint_as_float(v[g * 4 + 0]) + ((bias && c0 + g * 4 + 0 < rows_b) ? bias[c0 + g * 4 + 0] : 0.f);
-        x.y = __uint_as_float(v[g * 4 + 1]) + ((bias && c0 + g * 4 + 1 < rows_b) ? bias[c0 + g * 4 + 1] : 0.f);
-        x.z = __uint_as_float(v[g * 4 + 2]) + ((bias && c0 + g * 4 + 2 < rows_b) ? bias[c0 + g * 4 + 2] : 0.f);
-        x.w = __uint_as_float(v[g * 4 + 3]) + ((bias && c0 + g * 4 + 3 < rows_b) ? bias[c0 + g * 4 + 3] : 0.f);
+        x.x = __uint_as_float(v[g * 4 + 0]) + bias_s[cc * 32 + g * 4 + 0];
+        x.y = __uint_as_float(v[g * 4 + 1]) + bias_s[cc * 32 + g * 4 + 1];
+        x.z = __uint_as_float(v[g * 4 + 2]) + bias_s[cc * 32 + g * 4 + 2];
+        x.w = __uint_as_float(v[g * 4 + 3]) + bias_s[cc * 32 + g * 4 + 3];
         *reinterpret_cast<float4*>(row + ((g ^ sw) << 4)) = x;
       }
     } else {
@@ -102,8 +110,8 @@ __device__ __forceinline__ void epilogue_tma(uint32_t tmem_acc, int m0, int n0, 
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int j0 = g * 8 + 2 * e;
-          float x0 = __uint_as_float(v[j0]) + ((bias && c0 + j0 < rows_b) ? bias[c0 + j0] : 0.f);
-          float x1 = __uint_as_float(v[j0 + 1]) + ((bias && c0 + j0 + 1 < rows_b) ? bias[c0 + j0 + 1] : 0.f);
+          float x0 = __uint_as_float(v[j0]) + bias_s[cc * 32 + j0];
+          float x1 = __uint_as_float(v[j0 + 1]) + bias_s[cc * 32 + j0 + 1];
           if (epi == EPI_GELU) { x0 = gelu_tanh_fast(x0); x1 = gelu_tanh_fast(x1); }
           __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
           pk[e] = *reinterpret_cast<uint32_t*>(&h2);
@@ -370,11 +378,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int q = warp & 3;
     // every lane waits; the outcome is made warp-uniform because tcgen05.ld is a warp-wide instruction
     // (and uniform over the four epilogue warps, which meet at named barriers in the TMA-store path)
+    float* bias_s = reinterpret_cast<float*>(generic_base + STAGES * STAGE_BYTES + 256);
+    if (!SWAP && tma_out) stage_bias<BN>(bias_s, bias, n0, rows_b);     // while the main loop runs
     const bool ready = named_bar_and(1, 128, mbar_wait(tmem_full_bar, 0u, abort_flag, status));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ready && !SWAP && tma_out) {
       int n_store = 0;
-      epilogue_tma<BN>(tmem_base, m0, n0, q, lane, epi, bias, rows_b, &map_out, generic_base, base, n_store);
+      epilogue_tma<BN>(tmem_base, m0, n0, q, lane, epi, bias_s, &map_out, generic_base, base, n_store);
       if (threadIdx.x == 64) tma_wait_group_read<0>();      // shared memory stays valid until the copies have read it
     } else if (ready) {
       epilogue_manual<BN, SWAP>(tmem_base, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, split, qd);
@@ -397,12 +407,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 template <int BN, bool HILO>
 constexpr int persist_stages() {
-  constexpr int s = (227 * 1024 - 2 * 128 * 128 - 1024 - 1024 - 512) / stage_bytes<BN, false, HILO>();
+  constexpr int s = (227 * 1024 - 2 * 128 * 128 - 1024 - 1024 - 512 - 2048) / stage_bytes<BN, false, HILO>();
   return s > 8 ? 8 : s;
 }
 template <int BN, bool HILO>
 constexpr int persist_smem_bytes() {
-  return persist_stages<BN, HILO>() * stage_bytes<BN, false, HILO>() + 2 * 128 * 128 + 1024 + 512;
+  return persist_stages<BN, HILO>() * stage_bytes<BN, false, HILO>() + 2 * 128 * 128 + 1024 + 512 + 2048;
 }
 
 template <int BN, bool HILO>
@@ -515,12 +525,14 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       const int buf = i & 1;
       const int m0 = (n_fastest ? tile / tiles_n : tile % tiles_m) * BM;
       const int n0 = (n_fastest ? tile % tiles_n : tile / tiles_m) * BN;
+      float* bias_s = reinterpret_cast<float*>(generic_base + BAR_OFF + 512) + buf * BN;
+      if (tma_out) stage_bias<BN>(bias_s, bias, n0, rows_b);            // while the tile's main loop runs
       const bool ready = named_bar_and(1, 128, mbar_wait(tfull_bar(buf), (uint32_t)(i >> 1) & 1u, abort_flag, status));
       if (!ready) break;
       fence_after_sync();
       const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
       if (tma_out)
-        epilogue_tma<BN>(acc, m0, n0, q, lane, epi, bias, rows_b, &map_out, generic_base + STAGING_OFF, base + STAGING_OFF, n_store);
+        epilogue_tma<BN>(acc, m0, n0, q, lane, epi, bias_s, &map_out, generic_base + STAGING_OFF, base + STAGING_OFF, n_store);
       else
         epilogue_manual<BN, false>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, false, qd);
       // this thread's reads of the accumulator are complete (tcgen05.wait::ld inside tmem_ld32): hand it back
