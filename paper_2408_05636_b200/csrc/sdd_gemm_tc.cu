@@ -379,12 +379,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // every lane waits; the outcome is made warp-uniform because tcgen05.ld is a warp-wide instruction
     // (and uniform over the four epilogue warps, which meet at named barriers in the TMA-store path)
     float* bias_s = reinterpret_cast<float*>(generic_base + STAGES * STAGE_BYTES + 256);
-    if (!SWAP && tma_out) stage_bias<BN>(bias_s, bias, n0, rows_b);     // while the main loop runs
+    // tma_out == 2 (fused QKV): only tiles that lie wholly in the columns kept in place (Q, and K without a cache)
+    // are plain row-major stores; the others scatter into the K cache / V^T and take the manual path
+    const bool use_tma = !SWAP && (tma_out == 1 || (tma_out == 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d)));
+    if (use_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);     // while the main loop runs
     const bool ready = named_bar_and(1, 128, mbar_wait(tmem_full_bar, 0u, abort_flag, status));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ready && !SWAP && tma_out) {
+    if (ready && use_tma) {
       int n_store = 0;
-      epilogue_tma<BN>(tmem_base, m0, n0, q, lane, epi, bias_s, &map_out, generic_base, base, n_store);
+      epilogue_tma<BN>(tmem_base, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &map_out, generic_base, base,
+                       n_store);
       if (threadIdx.x == 64) tma_wait_group_read<0>();      // shared memory stays valid until the copies have read it
     } else if (ready) {
       epilogue_manual<BN, SWAP>(tmem_base, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, split, qd);
@@ -526,13 +530,15 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       const int m0 = (n_fastest ? tile / tiles_n : tile % tiles_m) * BM;
       const int n0 = (n_fastest ? tile % tiles_n : tile / tiles_m) * BN;
       float* bias_s = reinterpret_cast<float*>(generic_base + BAR_OFF + 512) + buf * BN;
-      if (tma_out) stage_bias<BN>(bias_s, bias, n0, rows_b);            // while the tile's main loop runs
+      const bool use_tma = tma_out == 1 || (tma_out == 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d));
+      if (use_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);            // while the tile's main loop runs
       const bool ready = named_bar_and(1, 128, mbar_wait(tfull_bar(buf), (uint32_t)(i >> 1) & 1u, abort_flag, status));
       if (!ready) break;
       fence_after_sync();
       const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
-      if (tma_out)
-        epilogue_tma<BN>(acc, m0, n0, q, lane, epi, bias_s, &map_out, generic_base + STAGING_OFF, base + STAGING_OFF, n_store);
+      if (use_tma)
+        epilogue_tma<BN>(acc, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &map_out,
+                         generic_base + STAGING_OFF, base + STAGING_OFF, n_store);
       else
         epilogue_manual<BN, false>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, false, qd);
       // this thread's reads of the accumulator are complete (tcgen05.wait::ld inside tmem_ld32): hand it back
@@ -724,10 +730,10 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
   if (epi == EPI_RESIDUAL && (ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
     if ((e = get_tensor_map(out, M, N, ldc, BM, 32, &mo, 4)) != cudaSuccess) return e;
     tma_out = 1;
-  } else if ((epi == EPI_STORE || epi == EPI_GELU) && out_lo == nullptr && bn >= 64 && (ldc & 7) == 0 &&
+  } else if ((epi == EPI_STORE || epi == EPI_GELU || epi == EPI_QKV) && out_lo == nullptr && bn >= 64 && (ldc & 7) == 0 &&
              (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
     if ((e = get_tensor_map(out, M, N, ldc, BM, 64, &mo, 2)) != cudaSuccess) return e;
-    tma_out = 1;
+    tma_out = epi == EPI_QKV ? 2 : 1;   // fused QKV: per tile, see the kernel
   }
   // many 256-wide tiles and no K split: the persistent kernel (SDD_GEMM_PERSIST=0 switches it off)
   static const bool persist_on = [] { const char* e = getenv("SDD_GEMM_PERSIST"); return e == nullptr || atoi(e) != 0; }();
