@@ -25,6 +25,10 @@ Readings of the paper taken here (the paper is silent or garbled on each):
   * temperature tau divides the logits; tau = 0 is greedy decoding (the setting of every
     result the paper reports).
   * the last round's emission is truncated to `max_new`.
+  * "Sequence initialization" names standard speculative decoding for "the initial few tokens" (the evaluation
+    says the first 100) and nothing more.  Taken here: whole speculative-decoding rounds with an autoregressive
+    drafter run while fewer than `n_init` tokens have been generated; the round that crosses `n_init` is kept
+    whole; the rounds share one round counter (and so one random stream layout) with the diffusion rounds.
 MDLM-faithfulness of the unmasking rule: parity unpinned (MDLM's sampler is not available).
 """
 from __future__ import annotations
@@ -120,6 +124,36 @@ def draft(model_q: Model, ctx_ids: np.ndarray, gamma: int, T: int, tau_q: float,
             step_logits.append(lg)
         unmask_sample_step(st, lg, k, tau_q, seed, rnd, b)
     assert np.all(st.slots != st.vocab)  # step k = 1 reveals with probability 1
+    return st, step_logits
+
+
+def sps_draft(model_a: Model, ctx_ids: np.ndarray, gamma: int, tau_q: float, seed: int, rnd: int, b: int,
+              keep_step_logits: bool = False):
+    """Drafting of standard speculative decoding (Section "Preliminaries and Settings", paragraph "Speculative
+    decoding"): an autoregressive drafter M_q produces x_{i+1..i+gamma} one token per evaluation,
+    x_{i+j} ~ q_{i+j}(. | x_{1:i+j-1}), and every q row is stored for the acceptance test.  The draw of slot j uses
+    the same keyed Gumbel stream as the diffusion drafter's draw of slot j."""
+    V = model_a.shape.vocab
+    st = DraftState.fresh(gamma, V)
+    ids = [int(x) for x in ctx_ids]
+    step_logits = []
+    for j in range(gamma):
+        row = model_a.logits(np.array(ids), [len(ids) - 1])[0]
+        if keep_step_logits:
+            step_logits.append(row)
+        if tau_q > 0.0:
+            z = row / tau_q
+            x, gap = argmax_with_gap(z + px.vocab_gumbels(seed, px.DRAFT, rnd, 0, j, b, V))
+            st.qrows[j] = z
+            st.logq[j] = z[x] - logsumexp(z)
+        else:
+            x, gap = argmax_with_gap(row)
+            st.qrows[j] = row
+            st.logq[j] = 0.0
+        st.slots[j] = x
+        st.reveal_step[j] = gamma - j          # bookkeeping only: evaluation j + 1 of gamma wrote this slot
+        st.gumbel_gap[j] = gap
+        ids.append(int(x))
     return st, step_logits
 
 
@@ -224,6 +258,42 @@ def specdiff_round(model_p: Model, model_q: Model, ctx_ids, gamma: int, T: int,
     acc = accept_resample(lam, st.qrows, st.logq, st.slots, tau_p, tau_q, seed, rnd, b)
     emitted = [int(x) for x in st.slots[: acc.n]] + [acc.t]
     return RoundTrace(len(ctx_ids), st, acc, emitted, lam if keep else None, step_logits if keep else None)
+
+
+def sps_round(model_p: Model, model_a: Model, ctx_ids, gamma: int, tau_p: float, tau_q: float, seed: int, rnd: int,
+              b: int = 0, keep: bool = False) -> RoundTrace:
+    """One round of standard speculative decoding: autoregressive drafting, then the same verification,
+    acceptance and extra-token steps as Algorithm 1 (which differs from it only in how the draft is made)."""
+    ctx_ids = np.asarray(ctx_ids, dtype=np.int64)
+    st, step_logits = sps_draft(model_a, ctx_ids, gamma, tau_q, seed, rnd, b, keep_step_logits=keep)
+    lam = target_verify_logits(model_p, ctx_ids, st.slots)
+    acc = accept_resample(lam, st.qrows, st.logq, st.slots, tau_p, tau_q, seed, rnd, b)
+    emitted = [int(x) for x in st.slots[: acc.n]] + [acc.t]
+    return RoundTrace(len(ctx_ids), st, acc, emitted, lam if keep else None, step_logits if keep else None)
+
+
+def generate_with_sps_init(model_p: Model, model_q: Model, model_a: Model, prompt, gamma: int, T: int, gamma_sps: int,
+                           n_init: int, max_new: int, tau_p: float = 1.0, tau_q: float = 1.0, seed: int = 0,
+                           b: int = 0, keep: bool = False):
+    """Section "Sequence initialization": speculative-decoding rounds (drafter model_a, gamma_sps tokens per draft)
+    while fewer than n_init tokens exist, SpecDiff rounds (drafter model_q) after that.
+    Returns (all ids, list of RoundTrace, number of speculative-decoding rounds)."""
+    ids = [int(x) for x in prompt]
+    P = len(ids)
+    traces = []
+    rnd = 0
+    n_sps = 0
+    while len(ids) - P < max_new:
+        if len(ids) - P < n_init:
+            tr = sps_round(model_p, model_a, np.array(ids), gamma_sps, tau_p, tau_q, seed, rnd, b, keep)
+            n_sps += 1
+        else:
+            tr = specdiff_round(model_p, model_q, np.array(ids), gamma, T, tau_p, tau_q, seed, rnd, b, keep)
+        tr.emitted = tr.emitted[: max_new - (len(ids) - P)]
+        ids += tr.emitted
+        traces.append(tr)
+        rnd += 1
+    return np.array(ids, dtype=np.int64), traces, n_sps
 
 
 def generate(model_p: Model, model_q: Model, prompt, gamma: int, T: int, max_new: int,

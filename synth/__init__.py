@@ -56,6 +56,16 @@ class Workload:
     prompt_seed: int
     philox_seed: int
 
+    @property
+    def ar_drafter(self) -> ModelShape:
+        """Autoregressive drafter of the speculative-decoding warm start: the diffusion drafter's size, causal."""
+        d = self.drafter
+        return ModelShape(d.vocab, d.n_layer, d.d_model, d.n_head, d.n_ctx, True)
+
+    @property
+    def ar_weight_seed(self) -> int:
+        return self.weight_seed + 500
+
 
 def _wl(name, dtype, V, tl, td, th, ql, qd, qh, n_ctx, prompt, gamma, T, batch, max_new, seeds):
     return Workload(
