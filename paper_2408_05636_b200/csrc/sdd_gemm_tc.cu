@@ -712,14 +712,26 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
   }
   int bn = bn_hint;
   const long long mt = (M + BM - 1) / BM;
+  int splits = 1;
   if (bn != 32 && bn != 64 && bn != 128 && bn != 256) {
-    // the narrowest N tile whose grid still fits one wave (most CTAs without a second wave); 256 beyond that
-    bn = 256;
-    for (int cand : {32, 64, 128}) {
-      if (mt * ((N + cand - 1) / cand) <= SMS) { bn = cand; break; }
+    // Tile width (and K splits) by a cost model in SM clocks.  A CTA's main loop is bound by the fill rate of its
+    // shared memory (about 64 bytes per clock): (128 + bn) * 128 bytes per 64-wide k-block, i.e. 2 * (128 + bn) clocks,
+    // against 2 * bn clocks of tensor-core time.  CTAs that share an SM share that rate, so a grid costs
+    // ceil(CTAs / SMs) times one CTA; the epilogue adds a term that grows with the tile width.  Wide tiles with more
+    // K splits therefore beat narrow tiles whenever the grid would otherwise leave SMs idle.
+    double best = 0.0;
+    for (int cand : {256, 128, 64, 32}) {
+      const long long ctas1 = mt * ((N + cand - 1) / cand);
+      const int s = pick_splits(ctas1, 4);
+      const int kb_per = (total_kb + s - 1) / s;
+      const long long waves = (ctas1 * s + SMS - 1) / SMS;
+      double cost = (double)waves * (2.0 * (128 + cand) * kb_per + 600.0 + 8.0 * cand);
+      if (cand == 32 && epi != EPI_RESIDUAL && epi != EPI_STORE_F32) cost += (double)waves * 3000.0;   // no TMA store at this width
+      if (best == 0.0 || cost < best * 0.97) { best = cost; bn = cand; splits = s; }
     }
+  } else {
+    splits = pick_splits(mt * ((N + bn - 1) / bn), 4);
   }
-  const int splits = pick_splits(mt * ((N + bn - 1) / bn), 4);
   if ((e = get_tensor_map(A, a_cap, K, K, BM, BK, &ma)) != cudaSuccess) return e;
   if ((e = get_tensor_map(W, N, K, K, bn, BK, &mb)) != cudaSuccess) return e;
   ml = ma;
