@@ -124,6 +124,28 @@ int32_t sdd_step(sdd_ctx* ctx, int32_t* out_ids, int32_t* n_out);
  * either may be null. */
 int32_t sdd_ar_step(sdd_ctx* ctx, int32_t* out_ids, int32_t* n_out);
 
+/* Sequence initialisation (Section "Sequence initialization"; Table "walltime-metrics-prefix" samples the first 100
+ * tokens this way): standard speculative decoding with an AUTOREGRESSIVE drafter for the first tokens of a
+ * generation, SpecDiff rounds afterwards.  One such round is gamma_sps sequential evaluations of the drafter
+ * (Section "Preliminaries and Settings", paragraph "Speculative decoding": x_{i+j} ~ q_{i+j}(. | x_{1:i+j-1}), every
+ * q row stored) followed by the same verification, acceptance, extra-token and commit kernels as sdd_step.
+ *
+ * sdd_sps_workspace_bytes: bytes of the drafter's KV cache (+ a few ints) for params->batch sequences.
+ * sdd_sps_attach: ar_drafter is a causal model (sdd_model, causal = 1) with the target's vocabulary and dtype and
+ *   d_model <= the target's (it runs in the context's activation buffers); its weights stay owned by the caller and
+ *   must outlive the context.  workspace: device memory, 256-byte aligned, owned by the caller until sdd_destroy.
+ *   Must be called right after sdd_create (before any round: SDD_E_STATE otherwise); every prompt needs at least two
+ *   tokens (SDD_E_ARG); the drafter's position table must cover prompt + max_new + gamma (SDD_E_CTX_FULL).  Enqueues
+ *   the prefill of the drafter's cache on the context's stream.
+ * sdd_sps_step: one speculative-decoding round; 1 <= gamma_sps <= params.gamma (SDD_E_ARG).  out_ids is device int32
+ *   [batch][gamma_sps + 1] (-1 padded), n_out device int32 [batch]; either may be null.  The Philox round index is
+ *   shared with the other rounds; the draft draw of slot j uses the same stream as a SpecDiff round's slot j.
+ *   Allowed only while every round so far was a speculative-decoding round (the drafter's cache has no gaps then);
+ *   after the first sdd_step / sdd_draft_begin / sdd_ar_step it returns SDD_E_STATE. */
+int32_t sdd_sps_workspace_bytes(const sdd_model* ar_drafter, const sdd_params* params, uint64_t* out_bytes);
+int32_t sdd_sps_attach(sdd_ctx* ctx, const sdd_model* ar_drafter, void* workspace, uint64_t workspace_bytes);
+int32_t sdd_sps_step(sdd_ctx* ctx, int32_t gamma_sps, int32_t* out_ids, int32_t* n_out);
+
 /* Non-blocking progress read (host): rounds whose commit has been seen so far, and the smallest
  * number of generated tokens over the batch at that point.  Either pointer may be null. */
 int32_t sdd_progress(sdd_ctx* ctx, uint64_t* rounds_done, int32_t* min_emitted);

@@ -30,7 +30,8 @@ PROF_NAMES = ["gemm_drafter", "gemm_target", "head_drafter", "head_target", "att
 
 EXPORTS = [
     "sdd_workspace_bytes", "sdd_create", "sdd_draft_begin", "sdd_draft_step", "sdd_draft",
-    "sdd_verify_accept", "sdd_step", "sdd_ar_step", "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
+    "sdd_verify_accept", "sdd_step", "sdd_ar_step", "sdd_sps_workspace_bytes", "sdd_sps_attach", "sdd_sps_step",
+    "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
     "sdd_accept_logits_static", "sdd_debug_gemm_bf16", "sdd_debug_attention_bf16",
     "sdd_tap", "sdd_counters", "sdd_profile_begin", "sdd_profile_end", "sdd_sync_status", "sdd_destroy", "sdd_strerror", "sdd_last_cuda_error",
 ]
@@ -75,6 +76,9 @@ def lib() -> C.CDLL:
         L.sdd_verify_accept.argtypes = [vp, vp, vp]
         L.sdd_step.argtypes = [vp, vp, vp]
         L.sdd_ar_step.argtypes = [vp, vp, vp]
+        L.sdd_sps_workspace_bytes.argtypes = [C.POINTER(sdd_model), C.POINTER(sdd_params), C.POINTER(u64)]
+        L.sdd_sps_attach.argtypes = [vp, C.POINTER(sdd_model), vp, u64]
+        L.sdd_sps_step.argtypes = [vp, i32, vp, vp]
         L.sdd_progress.argtypes = [vp, C.POINTER(u64), C.POINTER(i32)]
         L.sdd_accept_scratch_bytes.argtypes = [i32, i32, i32]
         L.sdd_accept_scratch_bytes.restype = u64
@@ -271,6 +275,20 @@ class Session:
         if not hasattr(self, "ar_ids"):
             self.ar_ids = self.torch.empty(self.batch, dtype=self.torch.int32, device=self.device)
         _check(lib().sdd_ar_step(self.h, self.ar_ids.data_ptr(), self.n_out.data_ptr()), "sdd_ar_step")
+
+    def sdd_sps_attach(self, ar_drafter: DeviceModel):
+        """Attach the autoregressive drafter of the speculative-decoding warm start (right after construction)."""
+        n = C.c_uint64(0)
+        _check(lib().sdd_sps_workspace_bytes(C.byref(ar_drafter.c), C.byref(self.params), C.byref(n)), "sdd_sps_workspace_bytes")
+        self.ar_drafter = ar_drafter
+        self.ar_workspace = self.torch.empty(int(n.value), dtype=self.torch.uint8, device=self.device)
+        _check(lib().sdd_sps_attach(self.h, C.byref(ar_drafter.c), self.ar_workspace.data_ptr(), int(n.value)), "sdd_sps_attach")
+
+    def sdd_sps_step(self, gamma_sps: int):
+        """One speculative-decoding round with the attached drafter (emitted ids in self.out_ids[:, :gamma_sps + 1])."""
+        if getattr(self, "sps_ids", None) is None or self.sps_ids.shape[1] != gamma_sps + 1:
+            self.sps_ids = self.torch.empty(self.batch, gamma_sps + 1, dtype=self.torch.int32, device=self.device)
+        _check(lib().sdd_sps_step(self.h, gamma_sps, self.sps_ids.data_ptr(), self.n_out.data_ptr()), "sdd_sps_step")
 
     def sdd_sync_status(self): _check(lib().sdd_sync_status(self.h), "sdd_sync_status")
 

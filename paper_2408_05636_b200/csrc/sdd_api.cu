@@ -172,6 +172,11 @@ struct sdd_ctx {
   int runahead;
   int lcap;                    // padded rows per sequence of the current round's drafter forwards
   size_t act_elems, xf_elems;  // capacity (elements) of the xn / att buffers (mlp: 4x) and of xf
+  Net A;                       // autoregressive drafter of the speculative-decoding warm start (sdd_sps_attach)
+  bool has_ar;
+  void* ar_kv;                 // its KV cache [layer][batch][n_ctx][2][d] (layout as the target's)
+  int* ar_eff;                 // [batch] effective length of its evaluation in flight
+  bool sps_allowed;            // false once a round of another kind has run (the drafter's cache would have holes)
   bool cache_skip;             // SDD_CACHE_SKIP != 0 (default): skip drafter evaluations whose input did not change
   bool hilo;                   // SDD_HILO != 0 (default): hi/lo activation pairs in the target's MLP and LM head
   bool force_simt;             // SDD_GEMM=simt: run bf16 GEMMs on the CUDA-core kernel (cross-check)
@@ -342,6 +347,52 @@ static int forward_drafter(sdd_ctx* c) {
   return SDD_OK;
 }
 
+// Causal forward of network N over rows_per_seq new tokens per sequence against its KV cache `kv`; `len` holds the
+// per-sequence length that fixes the rows' positions (see TargetMode); the caller has written the embeddings to B.h.
+template <typename T>
+static int forward_causal(sdd_ctx* c, const Net& N, void* kv, const int* len, int mode, int rows_per_seq, bool lm_head,
+                          float* logits_out, bool hilo, int gcat, int hcat, int acat) {
+  const Buffers& B = c->B;
+  const Dims& D = c->D;
+  const long long rows = (long long)D.batch * rows_per_seq;
+  const size_t layer_elems = (size_t)D.batch * N.n_ctx * 2 * N.d;
+  const bool tc = use_tc<T>(c, N);
+  hilo = hilo && tc;
+  // tensor-core path: per layer the cache is K [B][n_ctx][d] followed by V^T [B][d][n_ctx];
+  // CUDA-core path: [B][n_ctx][K|V][d]
+  SDD_TRY((run_blocks<T>(c, N, rows, gcat, hilo, nullptr,
+    [&](int l, QkvDst* qd) -> bool {
+      if (!tc) return false;
+      __nv_bfloat16* kc = (__nv_bfloat16*)kv + (size_t)l * layer_elems;
+      qd->k_dst = kc; qd->vt_dst = kc + layer_elems / 2; qd->ctx_len = len; qd->rows_per_seq = rows_per_seq;
+      qd->mode = mode == TARGET_VERIFY ? 1 : 2; qd->d = N.d; qd->k_seq_rows = N.n_ctx; qd->vt_ld = N.n_ctx;
+      return true;
+    },
+    [&](int l) -> int {
+      T* cache = (T*)kv + (size_t)l * layer_elems;
+      if (tc) {
+        const __nv_bfloat16* kc = (const __nv_bfloat16*)cache;
+        SDD_LAUNCH(c, acat, launch_attn_tc((const __nv_bfloat16*)B.qkv, (long long)(c->act_elems / N.d), 3 * N.d, 0, kc,
+                                           (long long)D.batch * N.n_ctx, N.d, 0, N.n_ctx, kc + layer_elems / 2, N.n_ctx,
+                                           (__nv_bfloat16*)B.att, N.d, len, D.batch, N.n_head, N.d, D.gamma,
+                                           mode == TARGET_VERIFY ? 1 : 2, rows_per_seq, &B.rs->status, c->st));
+      } else {
+        SDD_LAUNCH(c, CAT_GLUE, launch_kv_append<T>((const T*)B.qkv, cache, len, D.batch, rows_per_seq, mode, N.n_ctx, N.d,
+                                                    c->st));
+        SDD_LAUNCH(c, acat, launch_attn_cached<T>((const T*)B.qkv, cache, (T*)B.att, len, D.batch, rows_per_seq, mode,
+                                                  N.n_ctx, N.n_head, N.d_head, c->st));
+      }
+      return SDD_OK;
+    })));
+  if (lm_head) {
+    T* xf_lo = hilo ? (T*)B.xf_lo : nullptr;
+    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, N.lnf_g, N.lnf_b, (T*)B.xf, rows, N.d, c->st, xf_lo));
+    SDD_TRY(gemm<T>(c, hcat, B.xf, c->xf_elems, N.wte, nullptr, rows, D.V, N.d, EPI_STORE_F32, logits_out, D.V, nullptr,
+                    xf_lo));
+  }
+  return SDD_OK;
+}
+
 // target forward over rows_per_seq new tokens per sequence against the KV cache
 template <typename T>
 static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) {
@@ -349,43 +400,32 @@ static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) 
   const Buffers& B = c->B;
   const Dims& D = c->D;
   if (rows_per_seq <= 0) return SDD_OK;
-  const long long rows = (long long)D.batch * rows_per_seq;
+  // a verification forward carries the round's own draft length (gamma + 1 rows); slot_ids is [batch][that length]
+  const int slot_stride = mode == TARGET_VERIFY ? rows_per_seq - 1 : D.gamma;
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_target<T>((const T*)P.wte, (const T*)P.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
-                                       D.batch, D.gamma, rows_per_seq, mode, P.d, B.h, c->st));
-  const size_t layer_elems = (size_t)D.batch * P.n_ctx * 2 * P.d;
-  const bool tc = use_tc<T>(c, P);
-  // tensor-core path: per layer the cache is K [B][n_ctx][d] followed by V^T [B][d][n_ctx];
-  // CUDA-core path: [B][n_ctx][K|V][d]
-  SDD_TRY((run_blocks<T>(c, P, rows, CAT_GEMM_P, tc && c->hilo, nullptr,
-    [&](int l, QkvDst* qd) -> bool {
-      if (!tc) return false;
-      __nv_bfloat16* kc = (__nv_bfloat16*)B.kv + (size_t)l * layer_elems;
-      qd->k_dst = kc; qd->vt_dst = kc + layer_elems / 2; qd->ctx_len = B.ctx_len; qd->rows_per_seq = rows_per_seq;
-      qd->mode = mode == TARGET_VERIFY ? 1 : 2; qd->d = P.d; qd->k_seq_rows = P.n_ctx; qd->vt_ld = P.n_ctx;
-      return true;
-    },
-    [&](int l) -> int {
-      T* cache = (T*)B.kv + (size_t)l * layer_elems;
-      if (tc) {
-        const __nv_bfloat16* kc = (const __nv_bfloat16*)cache;
-        SDD_LAUNCH(c, CAT_ATTN_P, launch_attn_tc((const __nv_bfloat16*)B.qkv, (long long)(c->act_elems / P.d), 3 * P.d, 0, kc,
-                                                 (long long)D.batch * P.n_ctx, P.d, 0, P.n_ctx, kc + layer_elems / 2, P.n_ctx,
-                                                 (__nv_bfloat16*)B.att, P.d, B.ctx_len, D.batch, P.n_head, P.d, D.gamma,
-                                                 mode == TARGET_VERIFY ? 1 : 2, rows_per_seq, &B.rs->status, c->st));
-      } else {
-        SDD_LAUNCH(c, CAT_GLUE, launch_kv_append<T>((const T*)B.qkv, cache, B.ctx_len, D.batch, rows_per_seq, mode, P.n_ctx, P.d,
-                                                    c->st));
-        SDD_LAUNCH(c, CAT_ATTN_P, launch_attn_cached<T>((const T*)B.qkv, cache, (T*)B.att, B.ctx_len, D.batch, rows_per_seq, mode,
-                                                        P.n_ctx, P.n_head, P.d_head, c->st));
-      }
-      return SDD_OK;
-    })));
-  if (lm_head) {
-    T* xf_lo = (tc && c->hilo) ? (T*)B.xf_lo : nullptr;
-    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, P.lnf_g, P.lnf_b, (T*)B.xf, rows, P.d, c->st, xf_lo));
-    SDD_TRY(gemm<T>(c, CAT_HEAD_P, B.xf, c->xf_elems, P.wte, nullptr, rows, D.V, P.d, EPI_STORE_F32, B.logits_p, D.V, nullptr,
-                    xf_lo));
-  }
+                                       D.batch, slot_stride, rows_per_seq, mode, P.d, B.h, c->st));
+  return forward_causal<T>(c, P, B.kv, B.ctx_len, mode, rows_per_seq, lm_head, B.logits_p, c->hilo, CAT_GEMM_P, CAT_HEAD_P,
+                           CAT_ATTN_P);
+}
+
+// One evaluation of the autoregressive drafter of a speculative-decoding round, producing the logits of slot j
+// (Section "Preliminaries and Settings", paragraph "Speculative decoding": gamma sequential evaluations of M_q).
+// Evaluation 0 feeds positions c-2 and c-1: after a round that accepted every draft the drafter has never seen the
+// last draft token, and recomputing position c-2 otherwise reproduces what the cache already holds.  Evaluation
+// j > 0 feeds draft j-1 at position c+j-1.  The logits go to the head of the logits_p buffer, which is free until
+// the verification forward.
+template <typename T>
+static int forward_ar_drafter(sdd_ctx* c, int gamma, int j) {
+  const Net& A = c->A;
+  const Buffers& B = c->B;
+  const Dims& D = c->D;
+  const int rows = j == 0 ? 2 : 1, off = j == 0 ? -1 : j;
+  SDD_LAUNCH(c, CAT_GLUE, launch_embed_ar<T>((const T*)A.wte, (const T*)A.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
+                                             D.batch, gamma, rows, off, A.d, B.h, c->ar_eff, c->st));
+  SDD_TRY(forward_causal<T>(c, A, c->ar_kv, c->ar_eff, TARGET_VERIFY, rows, true, B.logits_p, false, CAT_GEMM_Q, CAT_HEAD_Q,
+                            CAT_ATTN_Q));
+  SDD_LAUNCH(c, CAT_SAMPLE, launch_ar_sample(B.logits_p, rows, B.slot_ids, B.q_logits, B.logq, B.reveal_step, D.batch, gamma, j,
+                                             D.V, c->inv_tau_q, c->key, B.rs, c->st));
   return SDD_OK;
 }
 
@@ -493,6 +533,10 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
   c->steps_done = -1;
   c->rounds = 0;
   c->launches = 0;
+  c->has_ar = false;
+  c->ar_kv = nullptr;
+  c->ar_eff = nullptr;
+  c->sps_allowed = true;
   c->profiling = false;
   c->prof_used = 0;
   {
@@ -586,6 +630,7 @@ static int round_epilogue(sdd_ctx* c, int max_emitted) {
 
 int32_t sdd_draft_begin(sdd_ctx* c) {
   if (c == nullptr) return SDD_E_ARG;
+  c->sps_allowed = false;
   SDD_TRY(round_prologue(c));
   return enqueue_draft_begin(c);
 }
@@ -615,6 +660,7 @@ int32_t sdd_verify_accept(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
 int32_t sdd_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
   if (c == nullptr) return SDD_E_ARG;
   if (c->steps_done != -1) return SDD_E_STATE;
+  c->sps_allowed = false;
   if (!c->use_graph) {
     SDD_TRY(sdd_draft(c));
     return sdd_verify_accept(c, out_ids, n_out);
@@ -655,6 +701,7 @@ int32_t sdd_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
 int32_t sdd_ar_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
   if (c == nullptr) return SDD_E_ARG;
   if (c->steps_done != -1) return SDD_E_STATE;
+  c->sps_allowed = false;
   if (c->rounds >= (uint64_t)c->runahead)
     SDD_CUDA(cudaEventSynchronize(c->ev[(c->rounds - c->runahead) % c->ev.size()]));
   if (!c->use_graph || c->profiling) {
@@ -683,6 +730,101 @@ int32_t sdd_ar_step(sdd_ctx* c, int32_t* out_ids, int32_t* n_out) {
   SDD_CUDA(cudaGraphLaunch(it->second.exec, c->st));
   c->launches += it->second.launches;
   return round_epilogue(c, 1);
+}
+
+// ---- speculative-decoding warm start (Section "Sequence initialization") -------------------------
+static size_t ar_workspace(const Net& A, int batch, size_t esize) {
+  return align_up((size_t)A.n_layer * batch * A.n_ctx * 2 * A.d * esize, 256) + align_up((size_t)batch * 4, 256);
+}
+
+int32_t sdd_sps_workspace_bytes(const sdd_model* ar_drafter, const sdd_params* params, uint64_t* out_bytes) {
+  if (out_bytes == nullptr || params == nullptr || params->batch < 1) return SDD_E_ARG;
+  Net A;
+  SDD_TRY(parse_model(ar_drafter, 1, &A));
+  *out_bytes = ar_workspace(A, params->batch, A.dtype == SDD_BF16 ? 2 : 4);
+  return SDD_OK;
+}
+
+int32_t sdd_sps_attach(sdd_ctx* c, const sdd_model* ar_drafter, void* workspace, uint64_t workspace_bytes) {
+  if (c == nullptr || workspace == nullptr) return SDD_E_ARG;
+  if (c->rounds != 0 || c->steps_done != -1 || c->has_ar) return SDD_E_STATE;
+  Net A;
+  SDD_TRY(parse_model(ar_drafter, 1, &A));
+  // the drafter shares the activation buffers, which are sized for the target's verification rows
+  if (A.vocab != c->P.vocab || A.dtype != c->P.dtype || A.d > c->P.d) return SDD_E_SHAPE;
+  for (int p : c->prompt_len)
+    if (p < 2) return SDD_E_ARG;                       // its first evaluation feeds positions c-2 and c-1
+  if ((long long)c->D.max_prompt + c->D.max_new + c->D.gamma > A.n_ctx) return SDD_E_CTX_FULL;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || ar_workspace(A, c->D.batch, c->D.esize) > workspace_bytes)
+    return SDD_E_WORKSPACE;
+  c->A = A;
+  const size_t kv_bytes = (size_t)A.n_layer * c->D.batch * A.n_ctx * 2 * A.d * c->D.esize;
+  c->ar_kv = workspace;
+  c->ar_eff = (int*)((uint8_t*)workspace + align_up(kv_bytes, 256));
+  SDD_CUDA(cudaMemsetAsync(workspace, 0, ar_workspace(A, c->D.batch, c->D.esize), c->st));   // V^T past the valid positions must be finite
+  // prefill its cache with x_{0:c-2}, as for the target
+  const Buffers& B = c->B;
+  const int rows = c->D.max_prompt - 1;
+  int s = SDD_OK;
+  if (A.dtype == SDD_BF16) {
+    SDD_LAUNCH(c, CAT_GLUE, launch_embed_target<__nv_bfloat16>((const __nv_bfloat16*)A.wte, (const __nv_bfloat16*)A.wpe, B.tokens,
+                                                               c->D.tok_stride, B.ctx_len, B.slot_ids, c->D.batch, c->D.gamma,
+                                                               rows, TARGET_PREFILL, A.d, B.h, c->st));
+    s = forward_causal<__nv_bfloat16>(c, A, c->ar_kv, B.ctx_len, TARGET_PREFILL, rows, false, nullptr, false, CAT_GEMM_Q,
+                                      CAT_HEAD_Q, CAT_ATTN_Q);
+  } else {
+    SDD_LAUNCH(c, CAT_GLUE, launch_embed_target<float>((const float*)A.wte, (const float*)A.wpe, B.tokens, c->D.tok_stride,
+                                                       B.ctx_len, B.slot_ids, c->D.batch, c->D.gamma, rows, TARGET_PREFILL, A.d,
+                                                       B.h, c->st));
+    s = forward_causal<float>(c, A, c->ar_kv, B.ctx_len, TARGET_PREFILL, rows, false, nullptr, false, CAT_GEMM_Q, CAT_HEAD_Q,
+                              CAT_ATTN_Q);
+  }
+  if (s != SDD_OK) { c->ar_kv = nullptr; return s; }
+  c->has_ar = true;
+  return SDD_OK;
+}
+
+static int enqueue_sps_round(sdd_ctx* c, int gamma, int32_t* out_ids, int32_t* n_out) {
+  for (int j = 0; j < gamma; ++j)
+    SDD_TRY(c->P.dtype == SDD_BF16 ? forward_ar_drafter<__nv_bfloat16>(c, gamma, j) : forward_ar_drafter<float>(c, gamma, j));
+  return enqueue_verify_accept(c, gamma, out_ids, n_out);
+}
+
+// One round of standard speculative decoding with the attached autoregressive drafter: gamma_sps sequential drafter
+// evaluations, then the same verification, acceptance and commit kernels as a SpecDiff round.
+int32_t sdd_sps_step(sdd_ctx* c, int32_t gamma_sps, int32_t* out_ids, int32_t* n_out) {
+  if (c == nullptr) return SDD_E_ARG;
+  if (!c->has_ar || !c->sps_allowed || c->steps_done != -1) return SDD_E_STATE;
+  if (gamma_sps < 1 || gamma_sps > c->D.gamma) return SDD_E_ARG;
+  if (c->rounds >= (uint64_t)c->runahead)
+    SDD_CUDA(cudaEventSynchronize(c->ev[(c->rounds - c->runahead) % c->ev.size()]));
+  if (!c->use_graph || c->profiling) {
+    SDD_TRY(enqueue_sps_round(c, gamma_sps, out_ids, n_out));
+    return round_epilogue(c, gamma_sps + 1);
+  }
+  // keys of the other graphs: padded row counts (positive), 0 (autoregressive step), small negative (timing passes)
+  const auto key = std::make_tuple(-(1 << 24) - gamma_sps, (void*)out_ids, (void*)n_out);
+  auto it = c->graphs.find(key);
+  if (it == c->graphs.end()) {
+    const uint64_t l0 = c->launches;
+    SDD_CUDA(cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal));
+    const int s = enqueue_sps_round(c, gamma_sps, out_ids, n_out);
+    cudaGraph_t g = nullptr;
+    cudaError_t e = cudaStreamEndCapture(c->st, &g);
+    if (s != SDD_OK) { if (g) cudaGraphDestroy(g); return s; }
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamEndCapture");
+    sdd_ctx::GraphEntry ge;
+    ge.exec = nullptr;
+    ge.launches = c->launches - l0;
+    c->launches = l0;
+    e = cudaGraphInstantiate(&ge.exec, g, 0);
+    cudaGraphDestroy(g);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGraphInstantiate");
+    it = c->graphs.emplace(key, ge).first;
+  }
+  SDD_CUDA(cudaGraphLaunch(it->second.exec, c->st));
+  c->launches += it->second.launches;
+  return round_epilogue(c, gamma_sps + 1);
 }
 
 int32_t sdd_progress(sdd_ctx* c, uint64_t* rounds_done, int32_t* min_emitted) {

@@ -56,6 +56,32 @@ __global__ void embed_target_kernel(const T* __restrict__ wte, const T* __restri
   for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = to_f32(te[e]) + to_f32(pe[e]);
 }
 
+// Autoregressive drafter of a speculative-decoding round: row i of sequence b is position c + off - 1 + i, whose token
+// is a context token (position < c) or a draft of this round (slot position - c).  Block (0, b) also publishes the
+// evaluation's effective length c + off, which the other kernels of the evaluation take in place of ctx_len
+// (their rows then sit at positions eff - 1 + i, the convention of a verification forward).
+template <typename T>
+__global__ void embed_ar_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
+                                int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
+                                int gamma, int rows_per_seq, int off, int d, float* __restrict__ h,
+                                int* __restrict__ eff_len) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int i = blockIdx.x, b = blockIdx.y;
+  const int c = ctx_len[b];
+  if (i == 0 && threadIdx.x == 0) eff_len[b] = c + off;
+  const int pos = c + off - 1 + i;
+  float* __restrict__ dst = h + ((long long)b * rows_per_seq + i) * d;
+  if (pos < 0) {   // cannot happen for prompts of two or more tokens
+    for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = 0.f;
+    return;
+  }
+  const int tok = pos < c ? tokens[(long long)b * tok_stride + pos] : slot_ids[(long long)b * gamma + pos - c];
+  const T* __restrict__ te = wte + (long long)tok * d;
+  const T* __restrict__ pe = wpe + (long long)pos * d;
+  for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = to_f32(te[e]) + to_f32(pe[e]);
+}
+
 // ---------------------------------------------------------------------------------------------
 // LayerNorm (eps 1e-5): one warp per row, the row held in registers, mean then centred variance
 // ---------------------------------------------------------------------------------------------
@@ -162,6 +188,14 @@ cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, i
   return cudaGetLastError();
 }
 template <typename T>
+cudaError_t launch_embed_ar(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
+                            const int* slot_ids, int batch, int gamma, int rows_per_seq, int off, int d, float* h,
+                            int* eff_len, cudaStream_t st) {
+  launch_k(embed_ar_kernel<T>, dim3(rows_per_seq, batch), dim3(128), 0, st, wte, wpe, tokens, tok_stride, ctx_len, slot_ids,
+           gamma, rows_per_seq, off, d, h, eff_len);
+  return cudaGetLastError();
+}
+template <typename T>
 cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* out, long long rows, int d,
                              cudaStream_t st, T* out_lo, const int* skip) {
   if (rows <= 0) return cudaSuccess;
@@ -189,6 +223,8 @@ cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int bat
                                                int, int, float*, cudaStream_t, const int*);                             \
   template cudaError_t launch_embed_target<T>(const T*, const T*, const int*, int, const int*, const int*, int, int,    \
                                               int, int, int, float*, cudaStream_t);                                     \
+  template cudaError_t launch_embed_ar<T>(const T*, const T*, const int*, int, const int*, const int*, int, int, int,   \
+                                          int, int, float*, int*, cudaStream_t);                                        \
   template cudaError_t launch_layernorm<T>(const float*, const float*, const float*, T*, long long, int, cudaStream_t, \
                                            T*, const int*);                                                                         \
   template cudaError_t launch_layernorm_slots<T>(const float*, const float*, const float*, T*, const int*, int, int,    \

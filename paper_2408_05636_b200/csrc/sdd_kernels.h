@@ -57,6 +57,10 @@ cudaError_t launch_accept(const float* logits_p, const float* q_rows, const int*
 cudaError_t launch_commit(int* tokens, int tok_stride, int* ctx_len, int* n_emitted, const int* slot_ids,
                           const int* n_accept, const int* extra_token, int batch, int gamma, int max_new, RoundState* rs,
                           int* out_ids, int* n_out, volatile int* host_mirror, cudaStream_t st);
+// draw of slot j from the last of the rows_per_seq logit rows per sequence (autoregressive drafter)
+cudaError_t launch_ar_sample(const float* logits, int rows_per_seq, int* slot_ids, float* q_logits, float* logq,
+                             int* reveal_step, int batch, int gamma, int j, int V, float inv_tau_q, PhiloxKey key,
+                             const RoundState* rs, cudaStream_t st);
 cudaError_t launch_reset_slots(int* slot_ids, int* reveal_step, int n, int mask_id, RoundState* rs, cudaStream_t st);
 
 // ---- glue (sdd_glue.cu) ---------------------------------------------------------------------
@@ -68,6 +72,11 @@ template <typename T>
 cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                 const int* slot_ids, int batch, int gamma, int rows_per_seq, int mode, int d, float* h,
                                 cudaStream_t st);
+// rows of an autoregressive drafter's evaluation: positions ctx_len[b] + off - 1 + i; writes eff_len[b] = ctx_len[b] + off
+template <typename T>
+cudaError_t launch_embed_ar(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
+                            const int* slot_ids, int batch, int gamma, int rows_per_seq, int off, int d, float* h,
+                            int* eff_len, cudaStream_t st);
 // LayerNorm of `rows` rows of h (fp32, row stride d) into out (activation type); out_lo (optional) receives the
 // rounding remainder y - out so that (out, out_lo) carries y to about 16 significant bits
 template <typename T>

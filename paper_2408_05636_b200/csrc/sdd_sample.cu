@@ -249,26 +249,14 @@ __device__ __forceinline__ MaxSum block_maxsum(MaxSum ms, float* s_m, float* s_s
 constexpr int SAMPLE_THREADS = 512;
 
 // returns true in every CTA of a cluster whose slot was revealed by this step
-__device__ __forceinline__ bool unmask_sample_row(const float* __restrict__ step_logits,  // [B, gamma, V]
-                     int* __restrict__ slot_ids,             // [B, gamma]  (V = masked)
-                     float* __restrict__ q_logits,           // [B, gamma, V]
-                     float* __restrict__ logq,               // [B, gamma]
-                     int* __restrict__ reveal_step,          // [B, gamma]
-                     int gamma, int V, int k, float inv_tau_q, PhiloxKey key, const RoundState* __restrict__ rs) {
+// Gumbel-max draw of one slot by the cluster that owns it: x = argmax_v (z_v + G_v), z = src * inv_tau_q (arg-max of
+// src when greedy); the row z is stored to dst and log q(x) = z_x - logsumexp(z) to *logq_out.  `mark` goes to
+// *reveal_out (the denoising step, or the evaluation index of an autoregressive drafter).
+__device__ __forceinline__ void draw_slot(const float* __restrict__ src, float* __restrict__ dst, int* __restrict__ slot_out,
+                                          float* __restrict__ logq_out, int* __restrict__ reveal_out, int j, int b, int V,
+                                          int mark, float inv_tau_q, PhiloxKey key, uint32_t rnd) {
   cg::cluster_group cl = cg::this_cluster();
   const int rank = (int)cl.block_rank();
-  const int j = blockIdx.x / VC, b = blockIdx.y;
-  const uint32_t rnd = rs->round;
-  const long long row = (long long)b * gamma + j;
-  // every CTA of the cluster takes the same decision from the same inputs, before anyone writes the slot
-  if (slot_ids[row] != V) return false;  // already revealed: carried over unchanged
-  // reveal with probability 1/k: u = m * 2^-24 with m odd, so u < 1/k  <=>  m * k < 2^24 (exact, k <= 255)
-  const uint32_t wu = philox4x32_10(0u, (uint32_t)j, rnd, rng_c3(RNG_UNMASK, (uint32_t)k, (uint32_t)b), key).x;
-  const uint32_t m_odd = ((wu >> 9) << 1) | 1u;
-  if (!(m_odd * (uint32_t)k < (1u << 24))) return false;
-
-  const float* __restrict__ src = step_logits + row * V;
-  float* __restrict__ dst = q_logits + row * V;
   const bool greedy = inv_tau_q == 0.f;
   const uint32_t c3 = rng_c3(RNG_DRAFT, 0u, (uint32_t)b);
 
@@ -311,11 +299,30 @@ __device__ __forceinline__ bool unmask_sample_row(const float* __restrict__ step
   if (rank == 0 && threadIdx.x == 0) {
     const ArgMax win = cluster_merge_argmax(cl, &part, false);
     const float lse = greedy ? 0.f : cluster_merge_lse(cl, &part);
-    slot_ids[row] = win.i;
-    logq[row] = greedy ? 0.f : src[win.i] * inv_tau_q - lse;
-    reveal_step[row] = k;
+    *slot_out = win.i;
+    *logq_out = greedy ? 0.f : src[win.i] * inv_tau_q - lse;
+    *reveal_out = mark;
   }
   cl.sync();   // partials stay alive until rank 0 has read them
+}
+
+__device__ __forceinline__ bool unmask_sample_row(const float* __restrict__ step_logits,  // [B, gamma, V]
+                     int* __restrict__ slot_ids,             // [B, gamma]  (V = masked)
+                     float* __restrict__ q_logits,           // [B, gamma, V]
+                     float* __restrict__ logq,               // [B, gamma]
+                     int* __restrict__ reveal_step,          // [B, gamma]
+                     int gamma, int V, int k, float inv_tau_q, PhiloxKey key, const RoundState* __restrict__ rs) {
+  const int j = blockIdx.x / VC, b = blockIdx.y;
+  const uint32_t rnd = rs->round;
+  const long long row = (long long)b * gamma + j;
+  // every CTA of the cluster takes the same decision from the same inputs, before anyone writes the slot
+  if (slot_ids[row] != V) return false;  // already revealed: carried over unchanged
+  // reveal with probability 1/k: u = m * 2^-24 with m odd, so u < 1/k  <=>  m * k < 2^24 (exact, k <= 255)
+  const uint32_t wu = philox4x32_10(0u, (uint32_t)j, rnd, rng_c3(RNG_UNMASK, (uint32_t)k, (uint32_t)b), key).x;
+  const uint32_t m_odd = ((wu >> 9) << 1) | 1u;
+  if (!(m_odd * (uint32_t)k < (1u << 24))) return false;
+  draw_slot(step_logits + row * V, q_logits + row * V, slot_ids + row, logq + row, reveal_step + row, j, b, V, k, inv_tau_q,
+            key, rnd);
   return true;
 }
 
@@ -341,6 +348,20 @@ unmask_sample_kernel(const float* __restrict__ step_logits, int* __restrict__ sl
       rs->ticket = 0u;
     }
   }
+}
+
+// Draw of slot j by an autoregressive drafter (standard speculative decoding): the logits are the last of the
+// `rows_per_seq` rows the evaluation produced for each sequence; the slot is always written.  grid = (VC, batch).
+__global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(SAMPLE_THREADS)
+ar_sample_kernel(const float* __restrict__ logits, int rows_per_seq, int* __restrict__ slot_ids, float* __restrict__ q_logits,
+                 float* __restrict__ logq, int* __restrict__ reveal_step, int gamma, int j, int V, float inv_tau_q,
+                 PhiloxKey key, const RoundState* __restrict__ rs) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int b = blockIdx.y;
+  const long long row = (long long)b * gamma + j;
+  draw_slot(logits + ((long long)b * rows_per_seq + rows_per_seq - 1) * V, q_logits + row * V, slot_ids + row, logq + row,
+            reveal_step + row, j, b, V, gamma - j, inv_tau_q, key, rs->round);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -610,6 +631,14 @@ cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float*
   dim3 grid(VC * gamma, batch);
   launch_k(unmask_sample_kernel, dim3(grid), dim3(SAMPLE_THREADS), 0, st, step_logits, slot_ids, q_logits, logq, reveal_step, gamma, V, k,
                                                        inv_tau_q, key, rs, cache_skip);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_ar_sample(const float* logits, int rows_per_seq, int* slot_ids, float* q_logits, float* logq,
+                             int* reveal_step, int batch, int gamma, int j, int V, float inv_tau_q, PhiloxKey key,
+                             const RoundState* rs, cudaStream_t st) {
+  launch_k(ar_sample_kernel, dim3(VC, batch), dim3(SAMPLE_THREADS), 0, st, logits, rows_per_seq, slot_ids, q_logits, logq,
+           reveal_step, gamma, j, V, inv_tau_q, key, rs);
   return cudaGetLastError();
 }
 
