@@ -98,6 +98,7 @@ struct Buffers {
   float* h;                    // residual stream, fp32
   void *xn, *qkv, *att, *mlp, *xf;  // activations in the model dtype
   void *xn_lo, *mlp_lo, *xf_lo;  // rounding remainders of xn / mlp / xf (hi/lo pairs of the target's MLP and LM head)
+  float* h_s;                  // residual stream of the gamma slot rows [batch * gamma, d_q] (last drafter block)
   void* vt;                    // drafter V transposed [batch][d_q][lcap_max] (tensor-core path)
   void* kv;                    // target KV cache [layer][batch][n_ctx][2][d]
 };
@@ -146,6 +147,7 @@ static size_t carve(const Dims& D, const Net& P, const Net& Q, uint8_t* base, Bu
   b.xn_lo = take(mx(rq * Q.d, rp * P.d) * D.esize);
   b.mlp_lo = take(mx(rq * Q.d, rp * P.d) * 4 * D.esize);
   b.xf_lo = take(Bn * (G + 1) * mx(Q.d, P.d) * D.esize);
+  b.h_s = (float*)take(Bn * G * Q.d * 4);
   b.kv = take((size_t)P.n_layer * Bn * P.n_ctx * 2 * P.d * D.esize);
   if (B) *B = b;
   return off;
@@ -177,6 +179,9 @@ struct sdd_ctx {
   void* ar_kv;                 // its KV cache [layer][batch][n_ctx][2][d] (layout as the target's)
   int* ar_eff;                 // [batch] effective length of its evaluation in flight
   bool sps_allowed;            // false once a round of another kind has run (the drafter's cache would have holes)
+  int slot_prune;              // SDD_SLOT_PRUNE: 1 / 0 = the drafter's last block runs on the slot rows only / on all rows;
+                               // unset (-1): on for forwards of 2048 rows or more (below that the forward is bound by
+                               // launch latency and the extra gather launch costs what the smaller GEMMs save)
   bool cache_skip;             // SDD_CACHE_SKIP != 0 (default): skip drafter evaluations whose input did not change
   bool hilo;                   // SDD_HILO != 0 (default): hi/lo activation pairs in the target's MLP and LM head
   bool force_simt;             // SDD_GEMM=simt: run bf16 GEMMs on the CUDA-core kernel (cross-check)
@@ -281,19 +286,33 @@ static bool use_tc(const sdd_ctx* c, const Net& N) {
   } while (0)
 
 // one transformer block on `rows` rows; attention is issued by the caller-supplied functor
-template <typename T, typename QkvFn, typename AttnFn>
+// slot_rows > 0 (drafter): after the last block's attention only the slot rows go on (gathered by `gather` into the
+// head of the dead qkv buffer and into h_s), because nothing else reaches the LM head
+template <typename T, typename QkvFn, typename AttnFn, typename GatherFn>
 static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, bool hilo_mlp, const int* skip, QkvFn qkv_dst,
-                      AttnFn attn) {
+                      AttnFn attn, long long slot_rows, GatherFn gather) {
   const Buffers& B = c->B;
   const int d = N.d;
   for (int l = 0; l < N.n_layer; ++l) {
     const Layer& L = N.layers[l];
+    const bool pruned = slot_rows > 0 && l == N.n_layer - 1;
     SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln1_g, L.ln1_b, (T*)B.xn, rows, d, c->st, nullptr, skip));
     QkvDst qd = {};
     const bool fused = qkv_dst(l, &qd);
     SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_qkv, L.b_qkv, rows, 3 * d, d, fused ? EPI_QKV : EPI_STORE, B.qkv,
                     3 * d, fused ? &qd : nullptr, nullptr, nullptr, skip));
     SDD_TRY(attn(l));
+    if (pruned) {
+      SDD_TRY(gather());
+      SDD_TRY(gemm<T>(c, gcat, B.qkv, 3 * c->act_elems, L.w_o, L.b_o, slot_rows, d, d, EPI_RESIDUAL, B.h_s, d, nullptr, nullptr,
+                      nullptr, skip));
+      SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h_s, L.ln2_g, L.ln2_b, (T*)B.xn, slot_rows, d, c->st, nullptr, skip));
+      SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_fc1, L.b_fc1, slot_rows, 4 * d, d, EPI_GELU, B.mlp, 4 * d, nullptr,
+                      nullptr, nullptr, skip));
+      SDD_TRY(gemm<T>(c, gcat, B.mlp, 4 * c->act_elems, L.w_fc2, L.b_fc2, slot_rows, d, 4 * d, EPI_RESIDUAL, B.h_s, d, nullptr,
+                      nullptr, nullptr, skip));
+      break;
+    }
     SDD_TRY(gemm<T>(c, gcat, B.att, c->act_elems, L.w_o, L.b_o, rows, d, d, EPI_RESIDUAL, B.h, d, nullptr, nullptr, nullptr, skip));
     // hilo_mlp: the MLP's two products take their activations as hi/lo bf16 pairs (see sdd_gemm_tc.cu)
     T* xn_lo = hilo_mlp ? (T*)B.xn_lo : nullptr;
@@ -317,6 +336,8 @@ static int forward_drafter(sdd_ctx* c) {
   const long long rows = (long long)D.batch * lcap;
   // every kernel of the evaluation returns at once when the previous step revealed nothing (RoundState.skip_forward)
   const int* skip = &B.rs->skip_forward;
+  const long long slot_rows = (long long)D.batch * D.gamma;
+  const bool prune = c->slot_prune == 1 || (c->slot_prune < 0 && rows >= 2048);
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_drafter<T>((const T*)Q.wte, (const T*)Q.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
                                         D.batch, D.gamma, lcap, Q.d, B.h, c->st, skip));
   const bool tc = use_tc<T>(c, Q);
@@ -339,9 +360,18 @@ static int forward_drafter(sdd_ctx* c) {
                                                        Q.d_head, c->st, skip));
       }
       return SDD_OK;
+    },
+    prune ? slot_rows : 0,
+    [&]() -> int {
+      SDD_LAUNCH(c, CAT_GLUE, launch_gather_slots<T>((const T*)B.att, B.h, B.ctx_len, D.batch, D.gamma, lcap, Q.d, (T*)B.qkv,
+                                                     B.h_s, c->st, skip));
+      return SDD_OK;
     })));
-  SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm_slots<T>(B.h, Q.lnf_g, Q.lnf_b, (T*)B.xf, B.ctx_len, D.batch, D.gamma, lcap, Q.d, c->st,
-                                                         skip));
+  if (prune)
+    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h_s, Q.lnf_g, Q.lnf_b, (T*)B.xf, slot_rows, Q.d, c->st, nullptr, skip));
+  else
+    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm_slots<T>(B.h, Q.lnf_g, Q.lnf_b, (T*)B.xf, B.ctx_len, D.batch, D.gamma, lcap, Q.d,
+                                                           c->st, skip));
   SDD_TRY(gemm<T>(c, CAT_HEAD_Q, B.xf, c->xf_elems, Q.wte, nullptr, (long long)D.batch * D.gamma, D.V, Q.d, EPI_STORE_F32, B.step_logits, D.V,
                   nullptr, nullptr, nullptr, skip));
   return SDD_OK;
@@ -383,7 +413,8 @@ static int forward_causal(sdd_ctx* c, const Net& N, void* kv, const int* len, in
                                                   N.n_ctx, N.n_head, N.d_head, c->st));
       }
       return SDD_OK;
-    })));
+    },
+    0, []() -> int { return SDD_OK; })));
   if (lm_head) {
     T* xf_lo = hilo ? (T*)B.xf_lo : nullptr;
     SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, N.lnf_g, N.lnf_b, (T*)B.xf, rows, N.d, c->st, xf_lo));
@@ -548,6 +579,8 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
     c->force_simt = g != nullptr && strcmp(g, "simt") == 0;
     const char* cs = getenv("SDD_CACHE_SKIP");
     c->cache_skip = cs == nullptr || atoi(cs) != 0;
+    const char* sp = getenv("SDD_SLOT_PRUNE");
+    c->slot_prune = sp == nullptr ? -1 : (atoi(sp) != 0 ? 1 : 0);
     const char* hl = getenv("SDD_HILO");
     c->hilo = hl == nullptr || atoi(hl) != 0;
     const char* bn = getenv("SDD_GEMM_BN");

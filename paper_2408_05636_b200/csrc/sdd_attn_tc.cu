@@ -15,6 +15,7 @@
 // over it; with that the CTA needs 96 KB and two CTAs share an SM, one's soft-max overlapping the other's MMAs.
 // Waits are bounded exactly as in the GEMM kernel.
 #include <mutex>
+#include <type_traits>
 
 #include "sdd_kernels.h"
 #include "sdd_tc.cuh"
@@ -191,19 +192,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       // the 64 scores are read twice from TMEM (once for the maximum, once for the exponentials) instead of being
       // kept in 64 registers: two CTAs per SM need the kernel to stay near 100 registers
       uint32_t v[32];
-      float mx = -INFINITY;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
 #pragma unroll 1
       for (int cc = 0; cc < 2; ++cc) {
         tmem_ld32(t_lane + (uint32_t)(hf * 64 + cc * 32), v);
         if (full) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
+          for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(v[j]));
         } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (key0 + cc * 32 + j < key_limit) mx = fmaxf(mx, __uint_as_float(v[j]));
+            if (key0 + cc * 32 + j < key_limit) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(v[j]));
         }
       }
+      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       float* sm = s_max + (t & 1) * 256;
       sm[hf * 128 + r] = mx;
       named_bar_sync(2, 256);
@@ -211,29 +213,39 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const float m_new = fmaxf(m, mx * scale);
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
       const float corr = m == -INFINITY ? 0.f : ex2(m - m_use);
-      float sum = 0.f;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      // two copies of the loop, chosen by a real branch: the visibility tests cost a third of the issue slots when
+      // they are predicated into the common (unmasked) path
+      auto exp_pass = [&](auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;
 #pragma unroll 1
-      for (int cc = 0; cc < 2; ++cc) {
-        tmem_ld32(t_lane + (uint32_t)(hf * 64 + cc * 32), v);
+        for (int cc = 0; cc < 2; ++cc) {
+          tmem_ld32(t_lane + (uint32_t)(hf * 64 + cc * 32), v);
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          uint32_t pk[4];
+          for (int g = 0; g < 4; ++g) {
+            uint32_t pk[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int j0 = g * 8 + 2 * e;
-            float p0 = ex2(fmaf(__uint_as_float(v[j0]), scale, -m_use));
-            float p1 = ex2(fmaf(__uint_as_float(v[j0 + 1]), scale, -m_use));
-            if (!full) {
-              if (!(key0 + cc * 32 + j0 < key_limit)) p0 = 0.f;
-              if (!(key0 + cc * 32 + j0 + 1 < key_limit)) p1 = 0.f;
+            for (int e = 0; e < 4; ++e) {
+              const int j0 = g * 8 + 2 * e;
+              float p0 = ex2(fmaf(__uint_as_float(v[j0]), scale, -m_use));
+              float p1 = ex2(fmaf(__uint_as_float(v[j0 + 1]), scale, -m_use));
+              if (!FULL) {
+                if (!(key0 + cc * 32 + j0 < key_limit)) p0 = 0.f;
+                if (!(key0 + cc * 32 + j0 + 1 < key_limit)) p1 = 0.f;
+              }
+              sum4[e] += p0 + p1;
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+              pk[e] = *reinterpret_cast<uint32_t*>(&h2);
             }
-            sum += p0 + p1;
-            __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+            *reinterpret_cast<uint4*>(p_row + (((cc * 4 + g) ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
-          *reinterpret_cast<uint4*>(p_row + (((cc * 4 + g) ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
-      }
+      };
+      // tcgen05.ld is warp-collective: the branch must not split a warp (rows past the end and causal rows have
+      // their own key_limit), so the unmasked copy runs only when every lane of the warp sees the whole tile
+      if (__all_sync(0xffffffffu, full)) exp_pass(std::true_type{});
+      else exp_pass(std::false_type{});
+      const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       l = l * corr + sum;     // this thread's half of the row sum; the halves share m, so they add up at the end
       m = m_new;
       fence_async_smem();

@@ -122,6 +122,67 @@ __device__ __forceinline__ void layernorm_row(const float* __restrict__ src, con
   }
 }
 
+// Vector variant for the large forwards: every lane owns groups of four consecutive elements (16-byte loads of the
+// fp32 row and of the gain / bias, 8- or 16-byte stores), NV groups per lane, d = 4 * 32 * NV at most and a multiple
+// of 4; all pointers 16-byte aligned.
+template <typename T>
+__device__ __forceinline__ void store4(T* p, float a, float b, float c, float d);
+template <>
+__device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+template <>
+__device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+}
+
+template <typename T, int NV>
+__global__ void __launch_bounds__(128)
+layernorm_vec_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
+                     T* __restrict__ out, T* __restrict__ out_lo, long long rows, int d, const int* __restrict__ skip) {
+  pdl_wait();
+  pdl_launch_dependents();
+  if (skip != nullptr && *skip) return;
+  const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int lane = threadIdx.x & 31;
+  const float* __restrict__ src = h + row * d;
+  float4 x[NV];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int e = (i * 32 + lane) * 4;
+    x[i] = e < d ? *reinterpret_cast<const float4*>(src + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+    sum += (x[i].x + x[i].y) + (x[i].z + x[i].w);
+  }
+  const float mu = warp_sum(sum) / (float)d;
+  float var = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int e = (i * 32 + lane) * 4;
+    if (e < d) {
+      const float a = x[i].x - mu, b = x[i].y - mu, c = x[i].z - mu, dd = x[i].w - mu;
+      var += (a * a + b * b) + (c * c + dd * dd);
+    }
+  }
+  const float rstd = rsqrtf(warp_sum(var) / (float)d + LN_EPS);
+  T* __restrict__ dst = out + row * d;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int e = (i * 32 + lane) * 4;
+    if (e < d) {
+      const float4 gg = *reinterpret_cast<const float4*>(g + e), bb = *reinterpret_cast<const float4*>(bta + e);
+      const float y0 = (x[i].x - mu) * rstd * gg.x + bb.x, y1 = (x[i].y - mu) * rstd * gg.y + bb.y;
+      const float y2 = (x[i].z - mu) * rstd * gg.z + bb.z, y3 = (x[i].w - mu) * rstd * gg.w + bb.w;
+      store4<T>(dst + e, y0, y1, y2, y3);
+      if (out_lo != nullptr)   // second half of a hi/lo pair
+        store4<T>(out_lo + row * d + e, y0 - to_f32<T>(from_f32<T>(y0)), y1 - to_f32<T>(from_f32<T>(y1)),
+                  y2 - to_f32<T>(from_f32<T>(y2)), y3 - to_f32<T>(from_f32<T>(y3)));
+    }
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(128)
 layernorm_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
@@ -146,6 +207,25 @@ layernorm_slots_kernel(const float* __restrict__ h, const float* __restrict__ g,
   if (r >= batch * gamma) return;
   const int b = r / gamma, j = r - b * gamma;
   layernorm_row<T>(h + ((long long)b * L_cap + ctx_len[b] + j) * d, g, bta, out + (long long)r * d, nullptr, d);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Slot-row gather: after the drafter's last attention only the gamma slot rows of every sequence feed the LM head, so
+// the rest of that block runs on a compact copy: att_s[b*gamma + j] = att[b*L_cap + c_b + j], the same for h.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void gather_slots_kernel(const T* __restrict__ att, const float* __restrict__ h, const int* __restrict__ ctx_len,
+                                    int gamma, int L_cap, int d, T* __restrict__ att_s, float* __restrict__ h_s,
+                                    const int* __restrict__ skip) {
+  pdl_wait();
+  pdl_launch_dependents();
+  if (skip != nullptr && *skip) return;
+  const int j = blockIdx.x, b = blockIdx.y;
+  const long long src = ((long long)b * L_cap + ctx_len[b] + j) * d, dst = ((long long)b * gamma + j) * d;
+  for (int e = threadIdx.x; e < d; e += blockDim.x) {
+    att_s[dst + e] = att[src + e];
+    h_s[dst + e] = h[src + e];
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -200,7 +280,15 @@ cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* 
                              cudaStream_t st, T* out_lo, const int* skip) {
   if (rows <= 0) return cudaSuccess;
   if (d > LN_MAX_PER_LANE * 32) return cudaErrorInvalidValue;
-  launch_k(layernorm_kernel<T>, dim3((unsigned)((rows + 3) / 4)), dim3(128), 0, st, h, g, b, out, out_lo, rows, d, skip);
+  const dim3 grid((unsigned)((rows + 3) / 4));
+  const uintptr_t al = reinterpret_cast<uintptr_t>(h) | reinterpret_cast<uintptr_t>(g) | reinterpret_cast<uintptr_t>(b) |
+                       reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(out_lo);
+  if ((d & 3) == 0 && (al & 15u) == 0 && rows >= 64) {
+    if (d <= 1024) launch_k(layernorm_vec_kernel<T, 8>, grid, dim3(128), 0, st, h, g, b, out, out_lo, rows, d, skip);
+    else launch_k(layernorm_vec_kernel<T, 16>, grid, dim3(128), 0, st, h, g, b, out, out_lo, rows, d, skip);
+  } else {
+    launch_k(layernorm_kernel<T>, grid, dim3(128), 0, st, h, g, b, out, out_lo, rows, d, skip);
+  }
   return cudaGetLastError();
 }
 template <typename T>
@@ -208,6 +296,12 @@ cudaError_t launch_layernorm_slots(const float* h, const float* g, const float* 
                                    int gamma, int L_cap, int d, cudaStream_t st, const int* skip) {
   if (d > LN_MAX_PER_LANE * 32) return cudaErrorInvalidValue;
   launch_k(layernorm_slots_kernel<T>, dim3((batch * gamma + 3) / 4), dim3(128), 0, st, h, g, b, out, ctx_len, batch, gamma, L_cap, d, skip);
+  return cudaGetLastError();
+}
+template <typename T>
+cudaError_t launch_gather_slots(const T* att, const float* h, const int* ctx_len, int batch, int gamma, int L_cap, int d,
+                                T* att_s, float* h_s, cudaStream_t st, const int* skip) {
+  launch_k(gather_slots_kernel<T>, dim3(gamma, batch), dim3(128), 0, st, att, h, ctx_len, gamma, L_cap, d, att_s, h_s, skip);
   return cudaGetLastError();
 }
 template <typename T>
@@ -229,6 +323,8 @@ cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int bat
                                            T*, const int*);                                                                         \
   template cudaError_t launch_layernorm_slots<T>(const float*, const float*, const float*, T*, const int*, int, int,    \
                                                  int, int, cudaStream_t, const int*);                                   \
+  template cudaError_t launch_gather_slots<T>(const T*, const float*, const int*, int, int, int, int, T*, float*,       \
+                                              cudaStream_t, const int*);                                                \
   template cudaError_t launch_kv_append<T>(const T*, T*, const int*, int, int, int, int, int, cudaStream_t);
 SDD_INSTANTIATE_GLUE(float)
 SDD_INSTANTIATE_GLUE(__nv_bfloat16)

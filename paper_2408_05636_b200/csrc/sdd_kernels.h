@@ -86,6 +86,10 @@ cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* 
 template <typename T>
 cudaError_t launch_layernorm_slots(const float* h, const float* g, const float* b, T* out, const int* ctx_len, int batch,
                                    int gamma, int L_cap, int d, cudaStream_t st, const int* skip = nullptr);
+// compact copies of the gamma slot rows of every sequence: att_s / h_s [batch * gamma, d]
+template <typename T>
+cudaError_t launch_gather_slots(const T* att, const float* h, const int* ctx_len, int batch, int gamma, int L_cap, int d,
+                                T* att_s, float* h_s, cudaStream_t st, const int* skip = nullptr);
 // copy the K and V thirds of qkv rows into the cache: cache[b][pos][0|1][d]
 template <typename T>
 cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int batch, int rows_per_seq, int mode, int n_ctx,

@@ -18,7 +18,9 @@ def _ref(q, k, v, causal_from=None):
     return o.transpose(0, 1)
 
 
-@pytest.mark.parametrize("H,lens,gamma,lcap", [(2, [100], 16, 128), (3, [250, 37, 511], 16, 640), (12, [300], 32, 384)])
+# the last case: many CTAs (several waves), sequences whose last key tile is full or ragged
+@pytest.mark.parametrize("H,lens,gamma,lcap", [(2, [100], 16, 128), (3, [250, 37, 511], 16, 640), (12, [300], 32, 384),
+                                                (16, [700, 130, 250, 1000, 496, 129], 16, 1024)])
 def test_drafter_mode(H, lens, gamma, lcap):
     import paper_2408_05636_b200 as sdd
     B, d = len(lens), H * 64

@@ -38,6 +38,20 @@ def test_small_bf16_ragged_batch():
     s.close()
 
 
+def test_small_bf16_ragged_batch_slot_row_pruning(monkeypatch):
+    """The same batch with the drafter's last block restricted to the slot rows (what large forwards do)."""
+    import paper_2408_05636_b200 as sdd
+    monkeypatch.setenv("SDD_SLOT_PRUNE", "1")
+    wl = synth.scaled_workload(synth.WORKLOADS["small_bf16"], batch=3, T=3)
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 3, 200, wl.prompt_seed)
+    s = sdd.Session(dp, dq, prompts, [200, 90, 131], wl.gamma, 3, 40, 1.0, 1.0, wl.philox_seed)
+    log, stats = roundcheck.check_rounds(s, mp, mq, wl, 1, 1.0, 1.0, TOL)
+    print("near-ties:", log, "max logit err q/p:", stats["max_q_err"], stats["max_p_err"])
+    assert len(log) <= 2
+    s.close()
+
+
 def test_xl_bf16_one_round_reduced_T():
     """GPT-2-XL-shaped target (48L d1600 h25) with the 24L d1024 drafter, prompt 512, gamma 32; one round with
     T = 2 denoising evaluations (the oracle needs about 3 TFLOP in fp64 for this round)."""

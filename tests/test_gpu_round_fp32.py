@@ -60,6 +60,19 @@ def test_ragged_batch_with_truncation_and_perturbed_weights():
     s.close()
 
 
+def test_slot_row_pruning_of_the_last_drafter_block(monkeypatch):
+    """Forced on (it is chosen by size otherwise): after the drafter's last attention only the slot rows go through
+    the rest of the block.  Same stage-by-stage parity as the full forward, ragged batch, non-trivial biases."""
+    monkeypatch.setenv("SDD_SLOT_PRUNE", "1")
+    wl = synth.scaled_workload(synth.WORKLOADS["tiny_fp32"], batch=3)
+    mp, mq, dp, dq = roundcheck.build_pair(wl, bias_std=0.05, perturb_ln=True)
+    prompts = synth.prompt_ids(wl.target.vocab, 3, 40, wl.prompt_seed)
+    s = _session(wl, dp, dq, prompts, [40, 7, 1], max_new=9, gamma=5, T=3)
+    log, stats = roundcheck.check_rounds(s, mp, mq, wl, 3, 1.0, 1.0, TOL)
+    assert len(log) <= 1 and stats["max_q_err"] < TOL
+    s.close()
+
+
 def test_greedy_equals_autoregressive_greedy():
     import paper_2408_05636_b200 as sdd
     wl = synth.WORKLOADS["tiny_fp32"]
