@@ -38,6 +38,9 @@ constexpr int BK = 64;           // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int THREADS = 192;     // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
 
+// tensor maps of the epilogue's TMA stores: the output matrix and (fused QKV of the drafter) the transposed V tensor
+struct alignas(64) OutMaps { CUtensorMap out, vt; };
+
 // one stage = A tile + B tile (+ the lo tile of the activation operand: the A side unless SWAP)
 template <int BN, bool SWAP, bool HILO>
 constexpr int stage_bytes() { return BM * BK * 2 + BN * BK * 2 + (HILO ? (SWAP ? BN : BM) * BK * 2 : 0); }
@@ -127,6 +130,54 @@ __device__ __forceinline__ void epilogue_tma(uint32_t tmem_acc, int m0, int n0, 
         const uint32_t src = stage_u32 + buf * (128 * 128);
         if (f32) tma_reduce_add_2d(map_out, src, c0, m0);
         else tma_store_2d(map_out, src, n0 + (cc & ~1) * 32, m0);
+        tma_commit_group();
+      }
+      ++n_store;
+    }
+  }
+}
+
+// V tiles of the drafter's fused-QKV GEMM: the tile is written transposed ([feature][position]) into the staging
+// buffers -- 64 features x 128 positions per buffer, as two 128-byte-swizzled boxes of 64 positions -- and leaves
+// through two TMA tile stores per buffer.  The 128 rows of the tile are 128 consecutive positions of one sequence.
+// vt_row0: row of the tile's first feature in the V^T tensor; pos0: position of the tile's first row.
+template <int BN>
+__device__ __forceinline__ void epilogue_vt(uint32_t tmem_acc, int q, int lane, const float* bias_s,
+                                            const CUtensorMap* map_vt, uint8_t* stage_generic, uint32_t stage_u32,
+                                            int& n_store, int vt_row0, int pos0) {
+  const int rl = q * 32 + lane;               // row inside the tile = position offset
+  const bool is_issuer = threadIdx.x == 64;
+  constexpr int CHUNKS = BN / 32;
+  const int pl = rl & 63;
+  const uint32_t box_off = (uint32_t)(rl >> 6) * (64 * 128);       // positions 64..127 fill the second box
+  const uint32_t in_row = (uint32_t)(pl & 7) * 2u;
+  const uint32_t pchunk = (uint32_t)(pl >> 3);
+#pragma unroll 1
+  for (int cc = 0; cc < CHUNKS; ++cc) {
+    uint32_t v[32];
+    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
+    const int buf = (cc >> 1) & 1;
+    const bool first_of_buf = (cc & 1) == 0;
+    const bool last_of_buf = (cc & 1) == 1 || cc == CHUNKS - 1;
+    if (first_of_buf) {
+      if (is_issuer && n_store >= 2) tma_wait_group_read<1>();   // the stores that last used this buffer have read it
+      named_bar_sync(2, 128);
+    }
+    uint8_t* bp = stage_generic + buf * (128 * 128) + box_off;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const int jj = (cc & 1) * 32 + j;        // feature row inside the buffer
+      const float x = __uint_as_float(v[j]) + bias_s[cc * 32 + j];
+      *reinterpret_cast<__nv_bfloat16*>(bp + jj * 128 + ((pchunk ^ (uint32_t)(jj & 7)) << 4) + in_row) = __float2bfloat16_rn(x);
+    }
+    if (last_of_buf) {
+      fence_async_smem();
+      named_bar_sync(2, 128);
+      if (is_issuer) {
+        const uint32_t src = stage_u32 + buf * (128 * 128);
+        const int y = vt_row0 + (cc & ~1) * 32;
+        tma_store_2d(map_vt, src, pos0, y);
+        tma_store_2d(map_vt, src + 64 * 128, pos0 + 64, y);
         tma_commit_group();
       }
       ++n_store;
@@ -272,7 +323,7 @@ __device__ __forceinline__ void epilogue_manual(uint32_t tmem_acc, int m0, int n
 template <int BN, bool SWAP, bool HILO, bool DEEP>
 __global__ void __launch_bounds__(THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_out, int tma_out,
+               const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ OutMaps maps_out, int tma_out,
                int rows_a, int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out,
                void* __restrict__ out_lo, int ldc, int* status, const QkvDst qd, const int* __restrict__ skip) {
 
@@ -381,15 +432,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     float* bias_s = reinterpret_cast<float*>(generic_base + STAGES * STAGE_BYTES + 256);
     // tma_out == 2 (fused QKV): only tiles that lie wholly in the columns kept in place (Q, and K without a cache)
     // are plain row-major stores; the others scatter into the K cache / V^T and take the manual path
-    const bool use_tma = !SWAP && (tma_out == 1 || (tma_out == 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d)));
-    if (use_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);     // while the main loop runs
+    // tma_out == 3: also the tiles that lie wholly in V leave by TMA, transposed (drafter; 128-row tiles never
+    // straddle sequences there)
+    const bool use_tma = !SWAP && (tma_out == 1 || (tma_out >= 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d)));
+    const bool vt_tma = !SWAP && tma_out == 3 && n0 >= 2 * qd.d && n0 + BN <= rows_b;
+    if (use_tma || vt_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);     // while the main loop runs
     const bool ready = named_bar_and(1, 128, mbar_wait(tmem_full_bar, 0u, abort_flag, status));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ready && use_tma) {
       int n_store = 0;
-      epilogue_tma<BN>(tmem_base, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &map_out, generic_base, base,
+      epilogue_tma<BN>(tmem_base, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &maps_out.out, generic_base, base,
                        n_store);
       if (threadIdx.x == 64) tma_wait_group_read<0>();      // shared memory stays valid until the copies have read it
+    } else if (ready && vt_tma) {
+      int n_store = 0;
+      const int sb = m0 / qd.rows_per_seq;
+      epilogue_vt<BN>(tmem_base, q, lane, bias_s, &maps_out.vt, generic_base, base, n_store, sb * qd.d + (n0 - 2 * qd.d),
+                      m0 - sb * qd.rows_per_seq);
+      if (threadIdx.x == 64) tma_wait_group_read<0>();
     } else if (ready) {
       epilogue_manual<BN, SWAP>(tmem_base, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, split, qd);
     }
@@ -422,7 +482,7 @@ constexpr int persist_smem_bytes() {
 template <int BN, bool HILO>
 __global__ void __launch_bounds__(THREADS)
 gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                       const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_out, int tma_out,
+                       const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ OutMaps maps_out, int tma_out,
                        int rows_a, int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out,
                        void* __restrict__ out_lo, int ldc, int* status, const QkvDst qd, const int* __restrict__ skip,
                        int tiles_m, int tiles_n, int n_fastest) {
@@ -530,15 +590,19 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       const int m0 = (n_fastest ? tile / tiles_n : tile % tiles_m) * BM;
       const int n0 = (n_fastest ? tile % tiles_n : tile / tiles_m) * BN;
       float* bias_s = reinterpret_cast<float*>(generic_base + BAR_OFF + 512) + buf * BN;
-      const bool use_tma = tma_out == 1 || (tma_out == 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d));
-      if (use_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);            // while the tile's main loop runs
+      const bool use_tma = tma_out == 1 || (tma_out >= 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d));
+      const bool vt_tma = tma_out == 3 && n0 >= 2 * qd.d && n0 + BN <= rows_b;
+      if (use_tma || vt_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);  // while the tile's main loop runs
       const bool ready = named_bar_and(1, 128, mbar_wait(tfull_bar(buf), (uint32_t)(i >> 1) & 1u, abort_flag, status));
       if (!ready) break;
       fence_after_sync();
       const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
       if (use_tma)
-        epilogue_tma<BN>(acc, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &map_out,
+        epilogue_tma<BN>(acc, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &maps_out.out,
                          generic_base + STAGING_OFF, base + STAGING_OFF, n_store);
+      else if (vt_tma)
+        epilogue_vt<BN>(acc, q, lane, bias_s, &maps_out.vt, generic_base + STAGING_OFF, base + STAGING_OFF, n_store,
+                        (m0 / qd.rows_per_seq) * qd.d + (n0 - 2 * qd.d), m0 % qd.rows_per_seq);
       else
         epilogue_manual<BN, false>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, false, qd);
       // this thread's reads of the accumulator are complete (tcgen05.wait::ld inside tmem_ld32): hand it back
@@ -559,7 +623,7 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 // host side: tensor maps (cached per pointer / shape / box) and launch
 // ---------------------------------------------------------------------------------------------
 template <int BN, bool SWAP, bool HILO, bool DEEP>
-static cudaError_t launch_cfg2(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& mo,
+static cudaError_t launch_cfg2(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const OutMaps& mo,
                               int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias, void* out, void* out_lo,
                               int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits, const int* skip) {
   dim3 grid((rows_b + BN - 1) / BN, (rows_a + BM - 1) / BM, splits);
@@ -568,7 +632,7 @@ static cudaError_t launch_cfg2(const CUtensorMap& ma, const CUtensorMap& mb, con
   return cudaGetLastError();
 }
 template <int BN, bool SWAP, bool HILO>
-static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& mo,
+static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const OutMaps& mo,
                               int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias, void* out, void* out_lo,
                               int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits, const int* skip) {
   // more than two waves of CTAs: shallow rings, two CTAs per SM (needs 2 x BN TMEM columns <= 512: always true)
@@ -580,7 +644,7 @@ static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, cons
                                            qd, splits, skip);
 }
 template <int BN, bool HILO>
-static cudaError_t launch_persist(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const CUtensorMap& mo,
+static cudaError_t launch_persist(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const OutMaps& mo,
                                   int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias, void* out,
                                   void* out_lo, int ldc, int* status, cudaStream_t st, const QkvDst& qd, const int* skip) {
   const int tiles_m = (rows_a + BM - 1) / BM, tiles_n = (rows_b + BN - 1) / BN;
@@ -594,7 +658,7 @@ static cudaError_t launch_persist(const CUtensorMap& ma, const CUtensorMap& mb, 
 
 template <int BN, bool SWAP>
 static cudaError_t launch_hl(bool hilo, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml,
-                             const CUtensorMap& mo, int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias,
+                             const OutMaps& mo, int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias,
                              void* out, void* out_lo, int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits,
                              const int* skip) {
   if (hilo)
@@ -707,8 +771,10 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     if ((e = get_tensor_map(A, a_cap, K, K, bn, BK, &mb)) != cudaSuccess) return e;
     ml = mb;
     if (hilo && (e = get_tensor_map(A_lo, a_cap, K, K, bn, BK, &ml)) != cudaSuccess) return e;
-    if (bn == 32) return launch_hl<32, true>(hilo, ma, mb, ml, ma, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
-    return launch_hl<64, true>(hilo, ma, mb, ml, ma, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
+    OutMaps none;
+    none.out = ma; none.vt = ma;
+    if (bn == 32) return launch_hl<32, true>(hilo, ma, mb, ml, none, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
+    return launch_hl<64, true>(hilo, ma, mb, ml, none, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
   }
   int bn = bn_hint;
   const long long mt = (M + BM - 1) / BM;
@@ -737,15 +803,24 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
   ml = ma;
   if (hilo && (e = get_tensor_map(A_lo, a_cap, K, K, BM, BK, &ml)) != cudaSuccess) return e;
   // output through TMA where the layout allows 16-byte-aligned rows (see the kernel's epilogue)
-  CUtensorMap mo = ma;
+  OutMaps mo;
+  mo.out = ma; mo.vt = ma;
   int tma_out = 0;
   if (epi == EPI_RESIDUAL && (ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
-    if ((e = get_tensor_map(out, M, N, ldc, BM, 32, &mo, 4)) != cudaSuccess) return e;
+    if ((e = get_tensor_map(out, M, N, ldc, BM, 32, &mo.out, 4)) != cudaSuccess) return e;
     tma_out = 1;
   } else if ((epi == EPI_STORE || epi == EPI_GELU || epi == EPI_QKV) && out_lo == nullptr && bn >= 64 && (ldc & 7) == 0 &&
              (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
-    if ((e = get_tensor_map(out, M, N, ldc, BM, 64, &mo, 2)) != cudaSuccess) return e;
+    if ((e = get_tensor_map(out, M, N, ldc, BM, 64, &mo.out, 2)) != cudaSuccess) return e;
     tma_out = epi == EPI_QKV ? 2 : 1;   // fused QKV: per tile, see the kernel
+    // drafter (every row of a tile is a position of one sequence, all of them stored): V tiles by TMA too
+    if (epi == EPI_QKV && qd.mode == 0 && qd.vt_dst != nullptr && (M % BM) == 0 && (qd.rows_per_seq % BM) == 0 &&
+        (qd.vt_ld & 7) == 0 && (reinterpret_cast<uintptr_t>(qd.vt_dst) & 15u) == 0 && qd.rows_per_seq <= qd.vt_ld) {
+      if ((e = get_tensor_map(qd.vt_dst, (long long)(M / qd.rows_per_seq) * qd.d, qd.vt_ld, qd.vt_ld, 64, 64, &mo.vt, 2)) !=
+          cudaSuccess)
+        return e;
+      tma_out = 3;
+    }
   }
   // many 256-wide tiles and no K split: the persistent kernel (SDD_GEMM_PERSIST=0 switches it off)
   static const bool persist_on = [] { const char* e = getenv("SDD_GEMM_PERSIST"); return e == nullptr || atoi(e) != 0; }();

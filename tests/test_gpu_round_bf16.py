@@ -52,6 +52,22 @@ def test_small_bf16_ragged_batch_slot_row_pruning(monkeypatch):
     s.close()
 
 
+def test_small_bf16_batch12_sampled_sequences():
+    """Twelve sequences: the drafter forward has 4608 rows, which is where the large-forward code paths start (the
+    persistent GEMM with its fused-QKV tiles, V^T tiles stored by TMA, vector LayerNorm, slot-row pruning chosen by
+    size).  One round with T = 2; three of the twelve sequences are followed by the oracle."""
+    import paper_2408_05636_b200 as sdd
+    wl = synth.scaled_workload(synth.WORKLOADS["small_bf16"], batch=12, T=2)
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 12, 260, wl.prompt_seed)
+    plen = [260, 131, 250, 199, 260, 77, 240, 258, 129, 260, 200, 255]
+    s = sdd.Session(dp, dq, prompts, plen, wl.gamma, 2, 40, 1.0, 1.0, wl.philox_seed)
+    log, stats = roundcheck.check_rounds(s, mp, mq, wl, 1, 1.0, 1.0, TOL, seqs=[0, 5, 11])
+    print("near-ties:", log, "max logit err q/p:", stats["max_q_err"], stats["max_p_err"])
+    assert len(log) <= 2
+    s.close()
+
+
 def test_xl_bf16_one_round_reduced_T():
     """GPT-2-XL-shaped target (48L d1600 h25) with the 24L d1024 drafter, prompt 512, gamma 32; one round with
     T = 2 denoising evaluations (the oracle needs about 3 TFLOP in fp64 for this round)."""
