@@ -620,6 +620,171 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 }
 
 // ---------------------------------------------------------------------------------------------
+// CTA-pair variant of the persistent kernel (tcgen05 cta_group::2): a cluster of two CTAs on two SMs owns a 256 x 256
+// tile.  CTA r loads rows m0 + 128 r of A and rows n0 + 128 r of W (half of the B tile) into its own shared memory;
+// one thread of CTA 0 (the leader) issues MMAs that run on both SMs' tensor cores, each reading its own A half and
+// both B halves, and accumulating the CTA's 128 x 256 half of the result in its own TMEM.  Per 64-wide k-block a CTA
+// fills 32 KB instead of the 48 KB of a one-CTA 128 x 256 tile, which lifts the shared-memory-fill bound from 2/3 of
+// the tensor peak to the peak.  Every barrier is an mbarrier in one CTA's shared memory; what the other CTA has to
+// learn is forwarded by a thread with a remote arrive:
+//   full[s]   (leader only: 1 arrive + the bytes of both CTAs' copies) -- both producers name the leader's barrier in
+//             their TMA loads (cta_group::2 form); the leader's producer announces the bytes of both
+//   empty[s]  (both: 1 arrive) -- the leader's MMA thread commits once to its own barrier and once to the peer's
+//   tfull[b]  (both: 1 arrive) -- leader's commit locally; its epilogue thread 64 forwards it to the peer
+//   tempty[b] (leader: 256 arrives) -- the epilogue threads of both CTAs arrive on the leader's barrier
+// (with forwarding threads on the full / empty path the refill round trip exceeded what the ring covers and the
+// kernel ran at half speed)
+// The epilogues are those of the one-CTA kernels, applied by each CTA to its half.  The CTAs meet at a cluster
+// barrier before TMEM is freed, so that neither leaves while the other may still touch its shared memory.
+// ---------------------------------------------------------------------------------------------
+constexpr int PAIR_STAGE_BYTES = BM * BK * 2 + 128 * BK * 2;     // A tile + half of the 256-wide B tile: 32 KB
+constexpr int PAIR_STAGES = 6;
+constexpr int PAIR_STAGING_OFF = PAIR_STAGES * PAIR_STAGE_BYTES;
+constexpr int PAIR_BAR_OFF = PAIR_STAGING_OFF + 2 * 128 * 128;
+constexpr int PAIR_SMEM = PAIR_BAR_OFF + 512 + 1024 + 1024;       // barriers, one tile's bias, alignment slack
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    const __grid_constant__ OutMaps maps_out, int tma_out, int rows_a, int rows_b, int K, int epi,
+                    const float* __restrict__ bias, void* __restrict__ out, int ldc, int* status, const QkvDst qd,
+                    const int* __restrict__ skip, int tiles_m2, int tiles_n, int n_fastest) {
+  constexpr int BN = 256;
+  constexpr int STAGES = PAIR_STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* generic_base = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bar_base = base + PAIR_BAR_OFF;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(generic_base + PAIR_BAR_OFF + 8 * (2 * STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(generic_base + PAIR_BAR_OFF + 8 * (2 * STAGES + 4) + 8);
+  constexpr uint32_t TMEM_COLS = 512;                // two 256-column accumulators
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const uint32_t peer = rank ^ 1u;
+  const int num_kb = (K + BK - 1) / BK;
+  const int n_tiles = tiles_m2 * tiles_n;
+  const int pair = (int)(blockIdx.x >> 1), n_pairs = (int)(gridDim.x >> 1);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 256); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  cluster_sync_all();                                // both CTAs' barriers exist before anyone arrives remotely
+  if (warp == 1) tmem_alloc_pair(tmem_slot, TMEM_COLS);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+  pdl_launch_dependents();
+  const bool active = skip == nullptr || *skip == 0;   // the same value in both CTAs (read after the producer grid)
+
+  if (!active) {
+  } else if (warp == 0) {
+    if (lane == 0) {
+      long long it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+        const int m0 = (n_fastest ? tile / tiles_n : tile % tiles_m2) * (2 * BM) + (int)rank * BM;
+        const int n0 = (n_fastest ? tile % tiles_n : tile / tiles_m2) * BN + (int)rank * 128;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = (int)(it % STAGES);
+          const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+          if (!mbar_wait_cluster(empty_bar(s), ph ^ 1u, abort_flag, status)) { ok = false; break; }
+          if (leader) mbar_expect_tx(full_bar(s), 2u * (uint32_t)PAIR_STAGE_BYTES);   // both CTAs' bytes
+          const uint32_t lf = map_to_cta(full_bar(s), 0u);
+          const uint32_t sa = base + s * PAIR_STAGE_BYTES;
+          tma_load_2d_pair(sa, &map_a, lf, kb * BK, m0);
+          tma_load_2d_pair(sa + BM * BK * 2, &map_b, lf, kb * BK, n0);
+        }
+      }
+      if (leader && *abort_flag) {
+        // do not leave while copies into the pair's shared memory may still be in flight (the peer stays until the
+        // cluster barrier at the end, which the leader reaches after this)
+        for (long long j = it > STAGES ? it - STAGES : 0; j < it; ++j) {
+          const long long t0 = clock64();
+          while (!mbar_try_cluster(full_bar((int)(j % STAGES)), (uint32_t)(j / STAGES) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && leader) {
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      long long it = 0;
+      int i = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++i) {
+        const int buf = i & 1;
+        ok = mbar_wait_cluster(tempty_bar(buf), ((uint32_t)(i >> 1) & 1u) ^ 1u, abort_flag, status);   // drained in both CTAs
+        if (!ok) break;
+        fence_after_sync();
+        const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = (int)(it % STAGES);
+          ok = mbar_wait_cluster(full_bar(s), (uint32_t)(it / STAGES) & 1u, abort_flag, status);
+          if (!ok) break;
+          fence_after_sync();
+          const uint32_t sa = base + s * PAIR_STAGE_BYTES;
+          const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + BM * BK * 2);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_pair(acc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit_pair(empty_bar(s));                       // frees the stage in this CTA ...
+          umma_commit_pair(map_to_cta(empty_bar(s), peer));     // ... and in the peer
+        }
+        if (ok) umma_commit_pair(tfull_bar(buf));
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    int n_store = 0, i = 0;
+    const uint32_t leader_tempty0 = map_to_cta(tempty_bar(0), 0u);
+    for (int tile = pair; tile < n_tiles; tile += n_pairs, ++i) {
+      const int buf = i & 1;
+      const int m0 = (n_fastest ? tile / tiles_n : tile % tiles_m2) * (2 * BM) + (int)rank * BM;
+      const int n0 = (n_fastest ? tile % tiles_n : tile / tiles_m2) * BN;
+      float* bias_s = reinterpret_cast<float*>(generic_base + PAIR_BAR_OFF + 512);   // reused: the same threads read it last
+      const bool use_tma = tma_out == 1 || (tma_out >= 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d));
+      const bool vt_tma = tma_out == 3 && n0 >= 2 * qd.d && n0 + BN <= rows_b;
+      if (use_tma || vt_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);  // while the tile's main loop runs
+      const bool mine = mbar_wait_cluster(tfull_bar(buf), (uint32_t)(i >> 1) & 1u, abort_flag, status);
+      // the leader forwards "accumulator complete" to the peer's epilogue warps
+      if (leader && threadIdx.x == 64 && mine) mbar_arrive_remote(map_to_cta(tfull_bar(buf), peer));
+      const bool ready = named_bar_and(1, 128, mine);
+      if (!ready) break;
+      fence_after_sync();
+      const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
+      if (use_tma)
+        epilogue_tma<BN>(acc, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &maps_out.out,
+                         generic_base + PAIR_STAGING_OFF, base + PAIR_STAGING_OFF, n_store);
+      else if (vt_tma)
+        epilogue_vt<BN>(acc, q, lane, bias_s, &maps_out.vt, generic_base + PAIR_STAGING_OFF, base + PAIR_STAGING_OFF, n_store,
+                        (m0 / qd.rows_per_seq) * qd.d + (n0 - 2 * qd.d), m0 % qd.rows_per_seq);
+      else
+        epilogue_manual<BN, false>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, nullptr, ldc, false, qd);
+      // this thread's reads of the accumulator are complete (tcgen05.wait::ld inside tmem_ld32): hand it back
+      fence_before_sync();
+      mbar_arrive_remote(leader_tempty0 + 8u * (uint32_t)buf);
+    }
+    if (threadIdx.x == 64) tma_wait_group_read<0>();      // staging memory stays valid until the copies have read it
+  }
+  fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();                                // the peer's MMAs, copies and remote arrives are behind us
+  if (warp == 1) {
+    fence_after_sync();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side: tensor maps (cached per pointer / shape / box) and launch
 // ---------------------------------------------------------------------------------------------
 template <int BN, bool SWAP, bool HILO, bool DEEP>
@@ -692,8 +857,9 @@ cudaError_t tc_prepare_gemm() {
   if ((e = prepare_one<64, true>()) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(gemm_tc_persist_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 persist_smem_bytes<256, false>())) != cudaSuccess) return e;
-  return cudaFuncSetAttribute(gemm_tc_persist_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              persist_smem_bytes<256, true>());
+  if ((e = cudaFuncSetAttribute(gemm_tc_persist_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                persist_smem_bytes<256, true>())) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM);
 }
 
 static PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
@@ -776,7 +942,7 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     if (bn == 32) return launch_hl<32, true>(hilo, ma, mb, ml, none, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
     return launch_hl<64, true>(hilo, ma, mb, ml, none, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
   }
-  int bn = bn_hint;
+  int bn = bn_hint == 512 ? 256 : bn_hint;       // 512: the CTA-pair kernel on 256 x 256 tiles
   const long long mt = (M + BM - 1) / BM;
   int splits = 1;
   if (bn != 32 && bn != 64 && bn != 128 && bn != 256) {
@@ -820,6 +986,23 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
           cudaSuccess)
         return e;
       tma_out = 3;
+    }
+  }
+  // CTA pairs on 256 x 256 tiles for the large GEMMs (bn_hint 512 forces them, SDD_GEMM_PAIR=0 switches them off)
+  {
+    const char* pe = getenv("SDD_GEMM_PAIR");
+    const bool pair_on = pe == nullptr || atoi(pe) != 0;
+    const bool eligible = !hilo && out_lo == nullptr && (M % 256) == 0 && (N % 256) == 0 && (bn_hint == 512 || bn == 256);
+    if (bn_hint == 512 && !eligible) return cudaErrorInvalidValue;
+    if (eligible && (bn_hint == 512 || (pair_on && splits == 1 && mt * (N / 256) > 2 * SMS))) {
+      CUtensorMap mb_half;
+      if ((e = get_tensor_map(W, N, K, K, 128, BK, &mb_half)) != cudaSuccess) return e;
+      const int tiles_m2 = M / 256, tiles_n = N / 256;
+      const long long tiles = (long long)tiles_m2 * tiles_n;
+      const unsigned pairs = (unsigned)(tiles < SMS / 2 ? tiles : SMS / 2);
+      launch_k(gemm_tc_pair_kernel, dim3(2 * pairs), dim3(THREADS), (size_t)PAIR_SMEM, st, ma, mb_half, mo, tma_out, M, N, K, epi,
+               bias, out, ldc, status, qd, skip, tiles_m2, tiles_n, (long long)N * K * 2 <= (48ll << 20) ? 1 : 0);
+      return cudaGetLastError();
     }
   }
   // many 256-wide tiles and no K split: the persistent kernel (SDD_GEMM_PERSIST=0 switches it off)

@@ -26,6 +26,8 @@ CASES = [
     (400, 768, 3072, 0), (130, 50257, 128, 128),
     # many tiles: the persistent kernel with two TMEM accumulators (ragged M and N)
     (8200, 2000, 192, 0), (5000, 4096, 1024, 0),
+    # CTA pairs (n_tile 512): 256 x 256 tiles computed by two SMs, one tile / several tiles per pair / long K
+    (256, 256, 64, 512), (512, 768, 192, 512), (1024, 512, 1024, 512), (4864, 1024, 320, 512),
     # swapped orientation: M <= 64 rows
     (1, 128, 64, 0), (17, 768, 3072, 0), (17, 2304, 768, 0), (33, 1600, 1600, 0), (64, 777, 256, 0), (17, 50257, 768, 0),
 ]
