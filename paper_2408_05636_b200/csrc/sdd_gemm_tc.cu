@@ -756,7 +756,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       if (use_tma || vt_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);  // while the tile's main loop runs
       const bool mine = mbar_wait_cluster(tfull_bar(buf), (uint32_t)(i >> 1) & 1u, abort_flag, status);
       // the leader forwards "accumulator complete" to the peer's epilogue warps
-      if (leader && threadIdx.x == 64 && mine) mbar_arrive_remote(map_to_cta(tfull_bar(buf), peer));
+      if (leader && threadIdx.x == 64 && mine) mbar_arrive_remote_relaxed(map_to_cta(tfull_bar(buf), peer));
       const bool ready = named_bar_and(1, 128, mine);
       if (!ready) break;
       fence_after_sync();
@@ -771,7 +771,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         epilogue_manual<BN, false>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, nullptr, ldc, false, qd);
       // this thread's reads of the accumulator are complete (tcgen05.wait::ld inside tmem_ld32): hand it back
       fence_before_sync();
-      mbar_arrive_remote(leader_tempty0 + 8u * (uint32_t)buf);
+      mbar_arrive_remote_relaxed(leader_tempty0 + 8u * (uint32_t)buf);
     }
     if (threadIdx.x == 64) tma_wait_group_read<0>();      // staging memory stays valid until the copies have read it
   }
@@ -994,7 +994,8 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     const bool pair_on = pe == nullptr || atoi(pe) != 0;
     const bool eligible = !hilo && out_lo == nullptr && (M % 256) == 0 && (N % 256) == 0 && (bn_hint == 512 || bn == 256);
     if (bn_hint == 512 && !eligible) return cudaErrorInvalidValue;
-    if (eligible && (bn_hint == 512 || (pair_on && splits == 1 && mt * (N / 256) > 2 * SMS))) {
+    // (forwards of a few thousand rows gain nothing from pairs; measured at 4608 rows: 3 to 5 % slower)
+    if (eligible && (bn_hint == 512 || (pair_on && splits == 1 && M >= 8192 && mt * (N / 256) > 2 * SMS))) {
       CUtensorMap mb_half;
       if ((e = get_tensor_map(W, N, K, K, 128, BK, &mb_half)) != cudaSuccess) return e;
       const int tiles_m2 = M / 256, tiles_n = N / 256;
