@@ -110,7 +110,9 @@ int32_t sdd_draft(sdd_ctx* ctx);
  * the extra token, and the commit of n+1 tokens to every sequence's context.  Requires a finished
  * draft (SDD_E_STATE otherwise).  If non-null, out_ids (device int32 [batch, gamma+1]) receives
  * the tokens emitted this round (-1 padded) and n_out (device int32 [batch]) their count per
- * sequence (0 for a sequence that already has max_new tokens). */
+ * sequence (0 for a sequence that already has max_new tokens).  Both may also point to page-locked host memory
+ * that the device can address: the commit kernel then writes them over the bus, and they are complete for round r
+ * as soon as sdd_progress reports r + 1 rounds, without a stream synchronisation. */
 int32_t sdd_verify_accept(sdd_ctx* ctx, int32_t* out_ids, int32_t* n_out);
 
 /* One whole round = sdd_draft + sdd_verify_accept. */

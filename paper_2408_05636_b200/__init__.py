@@ -267,8 +267,13 @@ class Session:
     def sdd_verify_accept(self):
         _check(lib().sdd_verify_accept(self.h, self.out_ids.data_ptr(), self.n_out.data_ptr()), "sdd_verify_accept")
 
-    def sdd_step(self):
-        _check(lib().sdd_step(self.h, self.out_ids.data_ptr(), self.n_out.data_ptr()), "sdd_step")
+    def sdd_step(self, out_ids=None, n_out=None):
+        """One round.  out_ids [batch, gamma + 1] / n_out [batch] int32: where the emitted ids go (default: the
+        session's device tensors).  Page-locked host tensors work too (the commit kernel then writes the ids
+        straight into host memory; they are complete once sdd_progress() counts the round)."""
+        o = self.out_ids if out_ids is None else out_ids
+        n = self.n_out if n_out is None else n_out
+        _check(lib().sdd_step(self.h, o.data_ptr(), n.data_ptr()), "sdd_step")
 
     def sdd_ar_step(self):
         """One plain autoregressive token per sequence (emitted ids in self.ar_ids [batch])."""

@@ -62,38 +62,55 @@ constexpr int smem_bytes() {
 // epilogues (shared by the one-tile and the persistent kernel); called by the four epilogue warps, q = TMEM lane
 // quarter of the calling warp, tmem_acc = first column of the tile's accumulator
 // ---------------------------------------------------------------------------------------------
-// the four epilogue warps copy the tile's bias values to shared memory (zero past column N or without a bias)
+// A group of four epilogue warps (128 threads, one TMEM lane quarter each) and the 32-column chunks it drains.  The
+// one-CTA kernels have one group for the whole tile with two staging buffers; the pair kernel has two groups, each
+// with half of the tile's chunks, one staging buffer and named barriers of its own.
+struct EpiGroup {
+  int c_begin, c_end;    // chunks [c_begin, c_end) of the tile; c_begin is even
+  int nbuf;              // staging buffers of 16 KB at stage_generic: 1 or 2
+  int bar_id;            // named barrier of the group's 128 threads
+  int first_tid;         // first thread of the group; it issues the group's TMA stores
+};
+template <int BN>
+__device__ __forceinline__ EpiGroup whole_tile_group() { return EpiGroup{0, BN / 32, 2, 2, 64}; }
+
+// the group copies the bias values of its chunks to shared memory (zero past column N or without a bias)
+__device__ __forceinline__ void stage_bias(float* bias_s, const float* __restrict__ bias, int n0, int rows_b, const EpiGroup& eg) {
+  for (int c = eg.c_begin * 32 + (int)threadIdx.x - eg.first_tid; c < eg.c_end * 32; c += 128)
+    bias_s[c] = (bias != nullptr && n0 + c < rows_b) ? bias[n0 + c] : 0.f;
+  named_bar_sync(eg.bar_id, 128);
+}
 template <int BN>
 __device__ __forceinline__ void stage_bias(float* bias_s, const float* __restrict__ bias, int n0, int rows_b) {
-  for (int c = (int)threadIdx.x - 64; c < BN; c += 128) bias_s[c] = (bias != nullptr && n0 + c < rows_b) ? bias[n0 + c] : 0.f;
-  named_bar_sync(2, 128);
+  stage_bias(bias_s, bias, n0, rows_b, whole_tile_group<BN>());
 }
 
 template <int BN>
 __device__ __forceinline__ void epilogue_tma(uint32_t tmem_acc, int m0, int n0, int q, int lane, int epi,
                                              const float* bias_s, const CUtensorMap* map_out,
-                                             uint8_t* stage_generic, uint32_t stage_u32, int& n_store) {
+                                             uint8_t* stage_generic, uint32_t stage_u32, int& n_store,
+                                             const EpiGroup eg = whole_tile_group<BN>()) {
   // Output through shared memory and TMA: every thread writes its row's 128-byte piece of the tile into a
   // staging buffer (128-byte swizzle, so that the 32 rows of a warp spread over all banks), one thread issues a
   // tile store (bf16 outputs) or an add-reduce (fp32 residual stream; also correct under K splits).
   // bias_s: the tile's BN bias values in shared memory (zeros where there is no bias or no column).
   const int rl = q * 32 + lane;               // row inside the tile
   const int sw = rl & 7;
-  const bool is_issuer = threadIdx.x == 64;
+  const bool is_issuer = (int)threadIdx.x == eg.first_tid;
   const bool f32 = epi == EPI_RESIDUAL;
-  constexpr int CHUNKS = BN / 32;
   #pragma unroll 1
-  for (int cc = 0; cc < CHUNKS; ++cc) {
+  for (int cc = eg.c_begin; cc < eg.c_end; ++cc) {
     uint32_t v[32];
     tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
     const int c0 = n0 + cc * 32;
     // fp32: one 32-column chunk fills a 128-byte row; bf16: two chunks do
-    const int buf = f32 ? (cc & 1) : ((cc >> 1) & 1);
+    const int buf = eg.nbuf == 1 ? 0 : (f32 ? (cc & 1) : ((cc >> 1) & 1));
     const bool first_of_buf = f32 || (cc & 1) == 0;
-    const bool last_of_buf = f32 || (cc & 1) == 1 || cc == CHUNKS - 1;
+    const bool last_of_buf = f32 || (cc & 1) == 1 || cc == eg.c_end - 1;
     if (first_of_buf) {
-      if (is_issuer && n_store >= 2) tma_wait_group_read<1>();   // the store that last used this buffer has read it
-      named_bar_sync(2, 128);
+      // the store that last used this buffer has read it
+      if (is_issuer && n_store >= eg.nbuf) { if (eg.nbuf == 1) tma_wait_group_read<0>(); else tma_wait_group_read<1>(); }
+      named_bar_sync(eg.bar_id, 128);
     }
     uint8_t* row = stage_generic + buf * (128 * 128) + rl * 128;
     if (f32) {
@@ -125,7 +142,7 @@ __device__ __forceinline__ void epilogue_tma(uint32_t tmem_acc, int m0, int n0, 
     }
     if (last_of_buf) {
       fence_async_smem();
-      named_bar_sync(2, 128);
+      named_bar_sync(eg.bar_id, 128);
       if (is_issuer) {
         const uint32_t src = stage_u32 + buf * (128 * 128);
         if (f32) tma_reduce_add_2d(map_out, src, c0, m0);
@@ -144,24 +161,25 @@ __device__ __forceinline__ void epilogue_tma(uint32_t tmem_acc, int m0, int n0, 
 template <int BN>
 __device__ __forceinline__ void epilogue_vt(uint32_t tmem_acc, int q, int lane, const float* bias_s,
                                             const CUtensorMap* map_vt, uint8_t* stage_generic, uint32_t stage_u32,
-                                            int& n_store, int vt_row0, int pos0) {
+                                            int& n_store, int vt_row0, int pos0,
+                                            const EpiGroup eg = whole_tile_group<BN>()) {
   const int rl = q * 32 + lane;               // row inside the tile = position offset
-  const bool is_issuer = threadIdx.x == 64;
-  constexpr int CHUNKS = BN / 32;
+  const bool is_issuer = (int)threadIdx.x == eg.first_tid;
   const int pl = rl & 63;
   const uint32_t box_off = (uint32_t)(rl >> 6) * (64 * 128);       // positions 64..127 fill the second box
   const uint32_t in_row = (uint32_t)(pl & 7) * 2u;
   const uint32_t pchunk = (uint32_t)(pl >> 3);
 #pragma unroll 1
-  for (int cc = 0; cc < CHUNKS; ++cc) {
+  for (int cc = eg.c_begin; cc < eg.c_end; ++cc) {
     uint32_t v[32];
     tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
-    const int buf = (cc >> 1) & 1;
+    const int buf = eg.nbuf == 1 ? 0 : ((cc >> 1) & 1);
     const bool first_of_buf = (cc & 1) == 0;
-    const bool last_of_buf = (cc & 1) == 1 || cc == CHUNKS - 1;
+    const bool last_of_buf = (cc & 1) == 1 || cc == eg.c_end - 1;
     if (first_of_buf) {
-      if (is_issuer && n_store >= 2) tma_wait_group_read<1>();   // the stores that last used this buffer have read it
-      named_bar_sync(2, 128);
+      // the stores that last used this buffer have read it
+      if (is_issuer && n_store >= eg.nbuf) { if (eg.nbuf == 1) tma_wait_group_read<0>(); else tma_wait_group_read<1>(); }
+      named_bar_sync(eg.bar_id, 128);
     }
     uint8_t* bp = stage_generic + buf * (128 * 128) + box_off;
 #pragma unroll
@@ -172,7 +190,7 @@ __device__ __forceinline__ void epilogue_vt(uint32_t tmem_acc, int q, int lane, 
     }
     if (last_of_buf) {
       fence_async_smem();
-      named_bar_sync(2, 128);
+      named_bar_sync(eg.bar_id, 128);
       if (is_issuer) {
         const uint32_t src = stage_u32 + buf * (128 * 128);
         const int y = vt_row0 + (cc & ~1) * 32;
@@ -188,11 +206,12 @@ __device__ __forceinline__ void epilogue_vt(uint32_t tmem_acc, int q, int lane, 
 template <int BN, bool SWAP>
 __device__ __forceinline__ void epilogue_manual(uint32_t tmem_acc, int m0, int n0, int q, int lane, int rows_a, int rows_b,
                                                 int epi, const float* __restrict__ bias, void* __restrict__ out,
-                                                void* __restrict__ out_lo, int ldc, bool split, const QkvDst& qd) {
+                                                void* __restrict__ out_lo, int ldc, bool split, const QkvDst& qd,
+                                                int c_begin = 0, int c_end = BN / 32) {
   const int r = m0 + q * 32 + lane;          // index along the A operand's rows
   const bool r_ok = r < rows_a;
 #pragma unroll 1
-  for (int cc = 0; cc < BN / 32; ++cc) {
+  for (int cc = c_begin; cc < c_end; ++cc) {
     uint32_t v[32];
     tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
     const int c0 = n0 + cc * 32;             // index along the B operand's rows
@@ -631,10 +650,11 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 //             their TMA loads (cta_group::2 form); the leader's producer announces the bytes of both
 //   empty[s]  (both: 1 arrive) -- the leader's MMA thread commits once to its own barrier and once to the peer's
 //   tfull[b]  (both: 1 arrive) -- leader's commit locally; its epilogue thread 64 forwards it to the peer
-//   tempty[b] (leader: 256 arrives) -- the epilogue threads of both CTAs arrive on the leader's barrier
+//   tempty[b] (leader: 512 arrives) -- the epilogue threads of both CTAs arrive on the leader's barrier
 // (with forwarding threads on the full / empty path the refill round trip exceeded what the ring covers and the
 // kernel ran at half speed)
-// The epilogues are those of the one-CTA kernels, applied by each CTA to its half.  The CTAs meet at a cluster
+// The epilogues are those of the one-CTA kernels, applied by each CTA to its half; eight epilogue warps in two groups
+// (columns 0..127 and 128..255, one staging buffer each), because the main loop of a tile is a third shorter here.  The CTAs meet at a cluster
 // barrier before TMEM is freed, so that neither leaves while the other may still touch its shared memory.
 // ---------------------------------------------------------------------------------------------
 constexpr int PAIR_STAGE_BYTES = BM * BK * 2 + 128 * BK * 2;     // A tile + half of the 256-wide B tile: 32 KB
@@ -643,7 +663,9 @@ constexpr int PAIR_STAGING_OFF = PAIR_STAGES * PAIR_STAGE_BYTES;
 constexpr int PAIR_BAR_OFF = PAIR_STAGING_OFF + 2 * 128 * 128;
 constexpr int PAIR_SMEM = PAIR_BAR_OFF + 512 + 1024 + 1024;       // barriers, one tile's bias, alignment slack
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS)
+constexpr int PAIR_THREADS = 320;   // warp 0: TMA, warp 1: MMA (leader) + TMEM owner, warps 2-5 and 6-9: two epilogue groups
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PAIR_THREADS)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ OutMaps maps_out, int tma_out, int rows_a, int rows_b, int K, int epi,
                     const float* __restrict__ bias, void* __restrict__ out, int ldc, int* status, const QkvDst qd,
@@ -672,7 +694,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 256); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 512); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -743,7 +765,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       }
     }
   } else {
+    // two groups of four warps; each drains half of the tile's columns through a staging buffer of its own
     const int q = warp & 3;
+    const int grp = (warp - 2) >> 2;
+    const EpiGroup eg{grp * 4, grp * 4 + 4, 1, 2 + grp, 64 + grp * 128};
+    uint8_t* stage_g = generic_base + PAIR_STAGING_OFF + grp * (128 * 128);
+    const uint32_t stage_u = base + PAIR_STAGING_OFF + grp * (128 * 128);
     int n_store = 0, i = 0;
     const uint32_t leader_tempty0 = map_to_cta(tempty_bar(0), 0u);
     for (int tile = pair; tile < n_tiles; tile += n_pairs, ++i) {
@@ -753,27 +780,28 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       float* bias_s = reinterpret_cast<float*>(generic_base + PAIR_BAR_OFF + 512);   // reused: the same threads read it last
       const bool use_tma = tma_out == 1 || (tma_out >= 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d));
       const bool vt_tma = tma_out == 3 && n0 >= 2 * qd.d && n0 + BN <= rows_b;
-      if (use_tma || vt_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);  // while the tile's main loop runs
+      if (use_tma || vt_tma) stage_bias(bias_s, bias, n0, rows_b, eg);  // while the tile's main loop runs
       const bool mine = mbar_wait_cluster(tfull_bar(buf), (uint32_t)(i >> 1) & 1u, abort_flag, status);
       // the leader forwards "accumulator complete" to the peer's epilogue warps
       if (leader && threadIdx.x == 64 && mine) mbar_arrive_remote_relaxed(map_to_cta(tfull_bar(buf), peer));
-      const bool ready = named_bar_and(1, 128, mine);
+      const bool ready = named_bar_and(4 + grp, 128, mine);
       if (!ready) break;
       fence_after_sync();
       const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
       if (use_tma)
-        epilogue_tma<BN>(acc, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &maps_out.out,
-                         generic_base + PAIR_STAGING_OFF, base + PAIR_STAGING_OFF, n_store);
+        epilogue_tma<BN>(acc, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &maps_out.out, stage_g, stage_u,
+                         n_store, eg);
       else if (vt_tma)
-        epilogue_vt<BN>(acc, q, lane, bias_s, &maps_out.vt, generic_base + PAIR_STAGING_OFF, base + PAIR_STAGING_OFF, n_store,
-                        (m0 / qd.rows_per_seq) * qd.d + (n0 - 2 * qd.d), m0 % qd.rows_per_seq);
+        epilogue_vt<BN>(acc, q, lane, bias_s, &maps_out.vt, stage_g, stage_u, n_store,
+                        (m0 / qd.rows_per_seq) * qd.d + (n0 - 2 * qd.d), m0 % qd.rows_per_seq, eg);
       else
-        epilogue_manual<BN, false>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, nullptr, ldc, false, qd);
+        epilogue_manual<BN, false>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, nullptr, ldc, false, qd, eg.c_begin,
+                                   eg.c_end);
       // this thread's reads of the accumulator are complete (tcgen05.wait::ld inside tmem_ld32): hand it back
       fence_before_sync();
       mbar_arrive_remote_relaxed(leader_tempty0 + 8u * (uint32_t)buf);
     }
-    if (threadIdx.x == 64) tma_wait_group_read<0>();      // staging memory stays valid until the copies have read it
+    if ((int)threadIdx.x == eg.first_tid) tma_wait_group_read<0>();   // staging memory stays valid until the copies have read it
   }
   fence_before_sync();
   __syncthreads();
@@ -988,20 +1016,21 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
       tma_out = 3;
     }
   }
-  // CTA pairs on 256 x 256 tiles for the large GEMMs (bn_hint 512 forces them, SDD_GEMM_PAIR=0 switches them off)
+  // CTA pairs on 256 x 256 tiles for the large GEMMs (bn_hint 512 forces them, SDD_GEMM_PAIR=0 switches them off, =2 drops the size rule)
   {
     const char* pe = getenv("SDD_GEMM_PAIR");
     const bool pair_on = pe == nullptr || atoi(pe) != 0;
+    const bool pair_any_size = pe != nullptr && atoi(pe) == 2;      // tests: pairs wherever they are eligible
     const bool eligible = !hilo && out_lo == nullptr && (M % 256) == 0 && (N % 256) == 0 && (bn_hint == 512 || bn == 256);
     if (bn_hint == 512 && !eligible) return cudaErrorInvalidValue;
     // (forwards of a few thousand rows gain nothing from pairs; measured at 4608 rows: 3 to 5 % slower)
-    if (eligible && (bn_hint == 512 || (pair_on && splits == 1 && M >= 8192 && mt * (N / 256) > 2 * SMS))) {
+    if (eligible && (bn_hint == 512 || (pair_on && splits == 1 && (M >= 8192 || pair_any_size) && mt * (N / 256) > 2 * SMS))) {
       CUtensorMap mb_half;
       if ((e = get_tensor_map(W, N, K, K, 128, BK, &mb_half)) != cudaSuccess) return e;
       const int tiles_m2 = M / 256, tiles_n = N / 256;
       const long long tiles = (long long)tiles_m2 * tiles_n;
       const unsigned pairs = (unsigned)(tiles < SMS / 2 ? tiles : SMS / 2);
-      launch_k(gemm_tc_pair_kernel, dim3(2 * pairs), dim3(THREADS), (size_t)PAIR_SMEM, st, ma, mb_half, mo, tma_out, M, N, K, epi,
+      launch_k(gemm_tc_pair_kernel, dim3(2 * pairs), dim3(PAIR_THREADS), (size_t)PAIR_SMEM, st, ma, mb_half, mo, tma_out, M, N, K, epi,
                bias, out, ldc, status, qd, skip, tiles_m2, tiles_n, (long long)N * K * 2 <= (48ll << 20) ? 1 : 0);
       return cudaGetLastError();
     }

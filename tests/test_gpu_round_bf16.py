@@ -52,11 +52,15 @@ def test_small_bf16_ragged_batch_slot_row_pruning(monkeypatch):
     s.close()
 
 
-def test_small_bf16_batch12_sampled_sequences():
+@pytest.mark.parametrize("pairs", ["1", "2"])
+def test_small_bf16_batch12_sampled_sequences(pairs, monkeypatch):
     """Twelve sequences: the drafter forward has 4608 rows, which is where the large-forward code paths start (the
     persistent GEMM with its fused-QKV tiles, V^T tiles stored by TMA, vector LayerNorm, slot-row pruning chosen by
-    size).  One round with T = 2; three of the twelve sequences are followed by the oracle."""
+    size).  One round with T = 2; three of the twelve sequences are followed by the oracle.  pairs = 2: the GEMMs that
+    are eligible run on CTA pairs although the forward is smaller than the size rule asks (fused-QKV, GELU and
+    residual epilogues of the pair kernel inside a round)."""
     import paper_2408_05636_b200 as sdd
+    monkeypatch.setenv("SDD_GEMM_PAIR", pairs)
     wl = synth.scaled_workload(synth.WORKLOADS["small_bf16"], batch=12, T=2)
     mp, mq, dp, dq = roundcheck.build_pair(wl)
     prompts = synth.prompt_ids(wl.target.vocab, 12, 260, wl.prompt_seed)
