@@ -278,10 +278,16 @@ def run_ours(args):
         kernels[n] = {"share": round(cat_ms[n] / total_ms, 4), "launches": cat_n[n],
                       "avg_us": round(cat_ms[n] * 1e3 / cat_n[n], 2), "bound": bound, "achieved": round(ach, 3),
                       "peak": peak, "unit": unit, "frac": round(ach / peak, 5)}
+    # DRAM bytes per launch of the drafter's GEMMs from the ncu capture summarised in
+    # profiles/gemm_drafter_traffic_small_bf16.txt (mean of the four GEMMs of a block; valid for the headline workload
+    # and for the GEMM kernel as captured)
+    traffic_bytes = {"gemm_drafter": 4.71e6} if wl.name == WORKLOAD and not (args.gamma or args.T) else {}
     dom = max(kernels, key=lambda n: kernels[n]["share"])
     roofline = {"kernel": dom, "bound": kernels[dom]["bound"], "achieved": kernels[dom]["achieved"],
                 "peak": kernels[dom]["peak"], "unit": kernels[dom]["unit"], "frac": kernels[dom]["frac"],
-                "traffic": None, "peak_source": f"of {peaks['source']}",
+                "traffic": traffic_bytes.get(dom), "traffic_unit": "bytes per launch (ncu dram read + write)",
+                "algorithmic_flops_per_launch": round(cat_work[dom] / max(1, cat_n[dom])),
+                "peak_source": f"of {peaks['source']}",
                 "timing": f"CUDA-event pairs around every launch in a separate pass of {prof_rounds} rounds"}
     sess.close()
 
