@@ -353,7 +353,11 @@ def run_ours(args):
     rows, g4 = 64, 32
     acc = microbench.accept(rows, g4, V, 0.5, iters=20, warmup=3)
     accept_roof = {"bound": "hbm", "achieved": round(acc["gbs"], 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                   "frac": round(acc["gbs"] / peaks["hbm_gbs"], 4), "traffic": None, "ms": round(acc["us"] * 1e-3, 4),
+                   "frac": round(acc["gbs"] / peaks["hbm_gbs"], 4),
+                   # ncu capture of the 16-row case scaled by 4 (profiles/accept_kernels_16x32x50257.txt): statistics pass
+                   # 209.08 + 3.7 MB, acceptance pass 6.69 MB per 16 rows; algorithmic bytes 836.3 MB
+                   "traffic": round(4 * (209.08e6 + 3.7e6 + 6.69e6)), "traffic_unit": "bytes per call (two launches)",
+                   "ms": round(acc["us"] * 1e-3, 4),
                    "launches_per_call": 2,
                    "workload": f"{rows} rows x gamma {g4} x V {V} fp32 logits, inputs 0.84 GB > L2",
                    "mean_accepted": acc["mean_accepted"], "peak_source": f"of {peaks['source']}"}
