@@ -14,6 +14,7 @@
 // completed (only then is the stage handed back to the producer), so the first half of P (keys 0..63) is written
 // over it; with that the CTA needs 96 KB and two CTAs share an SM, one's soft-max overlapping the other's MMAs.
 // Waits are bounded exactly as in the GEMM kernel.
+#include <cstdlib>
 #include <mutex>
 #include <type_traits>
 
@@ -34,6 +35,10 @@ constexpr int AT_KV_STAGES = 2;
 constexpr int AT_BAR_OFF = AT_Q_BYTES + AT_P_BYTES + AT_KV_STAGES * AT_STAGE_BYTES;   // 96 KB: two CTAs per SM
 constexpr int AT_SMEM = AT_BAR_OFF + 1024 + 128 + 3 * 1024;   // barriers, then the soft-max exchange arrays
 constexpr uint32_t AT_TMEM_COLS = 256;              // S: columns 0..127, PV: columns 128..191
+// key-split launches add a receive area for the other CTAs' partial states (it must not lie over tiles that this CTA
+// may still be using when a faster CTA sends): at most 136 rows of 64 floats plus their m and l
+constexpr int AT_RECV_OFF = AT_BAR_OFF + 3328;
+constexpr int AT_SMEM_SPLIT = AT_RECV_OFF + 36 * 1024 + 1024;
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -53,12 +58,25 @@ struct AttnParams {
   int d;                // model width = rows of one sequence in the V^T tensor
   int* status;
   const int* skip;      // may be null; *skip != 0: return at once (skipped drafter evaluation)
+  int kv_split;         // > 1 (unmasked mode, small grids): a cluster of kv_split CTAs shares the key tiles of one query
+                        // tile (CTA r takes tiles r, r + kv_split, ...); the partial soft-max states are merged row slice by
+                        // row slice, one slice per CTA
 };
+
+// stores into the shared memory of another CTA of the cluster (address from map_to_cta); they complete asynchronously
+// and are visible to that CTA after the next cluster barrier
+__device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, float a, float b, float c, float d) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
 
 __global__ void __launch_bounds__(AT_THREADS, 2)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_vt, const AttnParams prm) {
-  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int kv_split = prm.kv_split, kv_rank = (int)blockIdx.x % kv_split;   // cluster = kv_split consecutive CTAs in x
+  const int qt = (int)blockIdx.x / kv_split, h = blockIdx.y, b = blockIdx.z;
   pdl_wait();   // ctx_len and Q / K / V^T come from earlier kernels
   pdl_launch_dependents();
   if (prm.skip != nullptr && *prm.skip) return;
@@ -77,6 +95,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   else n_keys_cta = last_valid + 1;
   if (n_keys_cta > prm.k_rows_per_seq) n_keys_cta = prm.k_rows_per_seq;
   const int num_kt = (n_keys_cta + 127) / 128;
+  const int my_kt = kv_rank < num_kt ? (num_kt - kv_rank + kv_split - 1) / kv_split : 0;   // key tiles of this CTA
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -105,18 +124,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (lane == 0 && my_kt > 0) {
       mbar_expect_tx(q_full, AT_Q_BYTES);
       tma_load_2d(sQ, &map_q, q_full, prm.q_col0 + h * AT_DH, b * prm.q_rows_per_seq + q0);
       int issued = 0;
-      for (int t = 0; t < num_kt; ++t) {
-        const int s = t & 1;
-        if (!mbar_wait(kv_empty(s), ((uint32_t)(t >> 1) & 1u) ^ 1u, abort_flag, prm.status)) break;
+      for (int it = 0; it < my_kt; ++it) {
+        const int t = kv_rank + it * kv_split;      // key tile; `it` counts this CTA's iterations (stages, phases)
+        const int s = it & 1;
+        if (!mbar_wait(kv_empty(s), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag, prm.status)) break;
         mbar_expect_tx(kv_full(s), AT_STAGE_BYTES);
         tma_load_2d(sK(s), &map_k, kv_full(s), prm.k_col0 + h * AT_DH, b * prm.k_rows_per_seq + t * 128);
         tma_load_2d(sVT(s), &map_vt, kv_full(s), t * 128, b * prm.d + h * AT_DH);
         tma_load_2d(sVT(s) + 64 * 64 * 2, &map_vt, kv_full(s), t * 128 + 64, b * prm.d + h * AT_DH);
-        issued = t + 1;
+        issued = it + 1;
       }
       if (*abort_flag) {   // do not leave while copies into this CTA's shared memory may be in flight
         long long t0 = clock64();
@@ -127,13 +147,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
     }
+    if (kv_split > 1) { __syncwarp(); cluster_sync_all(); }   // see the soft-max warps
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (lane == 0 && my_kt > 0) {
       constexpr uint32_t idesc_s = make_idesc<128>();
       constexpr uint32_t idesc_pv = make_idesc<64>();
       bool ok = mbar_wait(q_full, 0u, abort_flag, prm.status);
       const uint64_t dq = make_smem_desc(sQ);
-      for (int t = 0; t < num_kt && ok; ++t) {
+      for (int t = 0; t < my_kt && ok; ++t) {        // t: this CTA's iteration (the key tile does not matter here)
         const int s = t & 1;
         ok = mbar_wait(kv_full(s), (uint32_t)(t >> 1) & 1u, abort_flag, prm.status);
         if (!ok) break;
@@ -156,6 +177,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         umma_commit(kv_empty(s));
       }
     }
+    if (kv_split > 1) { __syncwarp(); cluster_sync_all(); }
   } else {
     // soft-max warps 2..9: two threads per query row.  Warp w reads TMEM lane quarter w & 3; warps 2..5 take key
     // columns 0..63 of the tile (and output columns 0..31), warps 6..9 key columns 64..127 (output columns 32..63).
@@ -179,14 +201,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     for (int j = 0; j < AT_DH / 2; ++j) o[j] = 0.f;
     const int sw = r & 7;
     bool ok = true;
-    for (int t = 0; t < num_kt; ++t) {
-      ok = __all_sync(0xffffffffu, mbar_wait(s_full, (uint32_t)t & 1u, abort_flag, prm.status));
-      ok = named_bar_and(1, 256, ok);                  // also orders the reuse of s_max[t & 1] (last read at tile t - 2)
+    for (int it = 0; it < my_kt; ++it) {
+      const int t = kv_rank + it * kv_split;           // key tile; `it` counts this CTA's iterations (stages, phases)
+      ok = __all_sync(0xffffffffu, mbar_wait(s_full, (uint32_t)it & 1u, abort_flag, prm.status));
+      ok = named_bar_and(1, 256, ok);                  // also orders the reuse of s_max[it & 1] (last read two iterations ago)
       if (!ok) break;
       fence_after_sync();
       const int key0 = t * 128 + hf * 64;
       // this thread's 64 probabilities are one row of a P k-block: block 0 lies over the stage's (consumed) K tile
-      uint8_t* p_row = gbase + (hf == 0 ? AT_Q_BYTES + AT_P_BYTES + (t & 1) * AT_STAGE_BYTES : AT_Q_BYTES) + r * 128;
+      uint8_t* p_row = gbase + (hf == 0 ? AT_Q_BYTES + AT_P_BYTES + (it & 1) * AT_STAGE_BYTES : AT_Q_BYTES) + r * 128;
       // rows that see all of their 64 keys skip the per-entry visibility test
       const bool full = key0 + 64 <= key_limit;
       // the 64 scores are read twice from TMEM (once for the maximum, once for the exponentials) instead of being
@@ -206,7 +229,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      float* sm = s_max + (t & 1) * 256;
+      float* sm = s_max + (it & 1) * 256;
       sm[hf * 128 + r] = mx;
       named_bar_sync(2, 256);
       mx = fmaxf(mx, sm[(hf ^ 1) * 128 + r]);
@@ -250,7 +273,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       m = m_new;
       fence_async_smem();
       mbar_arrive(p_ready);
-      ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)t & 1u, abort_flag, prm.status));
+      ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)it & 1u, abort_flag, prm.status));
       if (!ok) break;
       fence_after_sync();
       tmem_ld32(t_lane + 128u + (uint32_t)(hf * 32), v);
@@ -261,7 +284,59 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (ok) {
       s_l[hf * 128 + r] = l;
       named_bar_sync(2, 256);
-      l += s_l[(hf ^ 1) * 128 + r];
+      l += s_l[(hf ^ 1) * 128 + r];                    // the row sum over this CTA's key tiles
+    }
+    bool writes_row = kv_split == 1;
+    if (kv_split > 1) {
+      // Merge of the cluster's partial soft-max states (m, l, o).  The 128 rows are dealt out to the CTAs in slices of
+      // sz rows; every thread sends its row's state to the CTA that owns the row (asynchronous remote stores into the
+      // receive area behind the kernel's other shared memory), one cluster barrier, then the owner's thread of
+      // that row adds up what it received.  recv_o[src][row in slice][64], recv_m / recv_l[src][row in slice].
+      const int sz = (128 + kv_split - 1) / kv_split;
+      const int owner = r / sz, rloc = r - owner * sz;
+      float* recv_o = reinterpret_cast<float*>(gbase + AT_RECV_OFF);
+      float* recv_m = recv_o + kv_split * sz * AT_DH;
+      float* recv_l = recv_m + kv_split * sz;
+      const bool have = ok && my_kt > 0;
+      if (owner != kv_rank) {
+        const int slot = kv_rank * sz + rloc;
+        if (hf == 0) {
+          st_cluster_f32(map_to_cta(smem_u32(recv_m + slot), (uint32_t)owner), have ? m : -INFINITY);
+          st_cluster_f32(map_to_cta(smem_u32(recv_l + slot), (uint32_t)owner), l);
+        }
+        if (have) {
+          const uint32_t dst = map_to_cta(smem_u32(recv_o + slot * AT_DH + hf * 32), (uint32_t)owner);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) st_cluster_v4(dst + 16u * j, o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        }
+      }
+      cluster_sync_all();
+      if (owner == kv_rank && ok) {
+        writes_row = true;
+        float mx = have ? m : -INFINITY;
+        for (int p = 0; p < kv_split; ++p)
+          if (p != kv_rank) mx = fmaxf(mx, recv_m[p * sz + rloc]);
+        const float w0 = (have && m != -INFINITY) ? ex2(m - mx) : 0.f;
+        l *= w0;
+#pragma unroll
+        for (int j = 0; j < AT_DH / 2; ++j) o[j] *= w0;
+        for (int p = 0; p < kv_split; ++p) {
+          if (p == kv_rank) continue;
+          const float mp = recv_m[p * sz + rloc];
+          if (mp == -INFINITY) continue;               // that CTA had no key tile (or no visible key) for this row
+          const float wp = ex2(mp - mx);
+          l = fmaf(recv_l[p * sz + rloc], wp, l);
+          const float4* src = reinterpret_cast<const float4*>(recv_o + (p * sz + rloc) * AT_DH + hf * 32);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float4 x = src[j];
+            o[4 * j] = fmaf(x.x, wp, o[4 * j]); o[4 * j + 1] = fmaf(x.y, wp, o[4 * j + 1]);
+            o[4 * j + 2] = fmaf(x.z, wp, o[4 * j + 2]); o[4 * j + 3] = fmaf(x.w, wp, o[4 * j + 3]);
+          }
+        }
+      }
+    }
+    if (ok && writes_row) {
       if (valid) {
         const float inv = 1.f / l;
         __nv_bfloat16* dst = prm.out + ((long long)b * prm.q_rows_per_seq + i) * prm.ld_out + h * AT_DH + hf * 32;
@@ -289,7 +364,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 }  // namespace tc
 
 cudaError_t tc_prepare_attn() {
-  return cudaFuncSetAttribute(tc::attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AT_SMEM);
+  return cudaFuncSetAttribute(tc::attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AT_SMEM_SPLIT);
 }
 
 cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q_ld, int q_col0, const __nv_bfloat16* k,
@@ -311,8 +386,25 @@ cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q
   AttnParams p;
   p.out = out; p.ld_out = ld_out; p.ctx_len = ctx_len; p.mode = mode; p.gamma = gamma;
   p.q_rows_per_seq = q_rows_per_seq; p.k_rows_per_seq = k_rows_per_seq; p.q_col0 = q_col0; p.k_col0 = k_col0;
-  p.d = d; p.status = status; p.skip = skip;
+  p.d = d; p.status = status; p.skip = skip; p.kv_split = 1;
   dim3 grid((q_rows_per_seq + 127) / 128, n_head, batch);
+  // Unmasked attention on a grid that leaves most SMs idle (one sequence): the key tiles of a query tile are shared out
+  // over a cluster of CTAs, which shortens the chain of dependent tiles per CTA; CTA 0 merges the partial states.
+  // As many CTAs per query tile as there are key tiles (at most 8) while the grid fits one CTA per SM.
+  // SDD_ATTN_SPLIT=0 switches it off.
+  if (mode == 0) {
+    const char* e = getenv("SDD_ATTN_SPLIT");
+    const long long ctas = (long long)grid.x * grid.y * grid.z;
+    int split = (q_rows_per_seq + 127) / 128;
+    if (split > 8) split = 8;
+    while (split > 1 && ctas * split > 148) --split;       // one CTA per SM with the receive area
+    if ((e == nullptr || atoi(e) != 0) && split > 1) {
+      p.kv_split = split;
+      grid.x *= split;
+      launch_k_cluster(attn_tc_kernel, grid, dim3(AT_THREADS), AT_SMEM_SPLIT, st, (unsigned)split, mq, mk, mv, p);
+      return cudaGetLastError();
+    }
+  }
   launch_k(attn_tc_kernel, dim3(grid), dim3(AT_THREADS), AT_SMEM, st, mq, mk, mv, p);
   return cudaGetLastError();
 }
