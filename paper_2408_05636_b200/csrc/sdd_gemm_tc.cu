@@ -488,25 +488,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // accumulators live in TMEM, so the MMA warp fills one while the epilogue warps drain the other; the operand ring
 // runs on across tile boundaries.  Extra barriers: tmem_full[2] (MMA -> epilogue), tmem_empty[2] (epilogue -> MMA).
 // ---------------------------------------------------------------------------------------------
-template <int BN, bool HILO>
+// SWAP (the LM heads: a few tokens against 50257 weight rows): the tiles are 128 weight rows each and the kernel is a
+// weight stream; what the persistent form buys there is that the loads run on while a tile's epilogue stores.
+template <int BN, bool HILO, bool SWAP = false>
 constexpr int persist_stages() {
-  constexpr int s = (227 * 1024 - 2 * 128 * 128 - 1024 - 1024 - 512 - 2048) / stage_bytes<BN, false, HILO>();
+  constexpr int s = (227 * 1024 - 2 * 128 * 128 - 1024 - 1024 - 512 - 2048) / stage_bytes<BN, SWAP, HILO>();
   return s > 8 ? 8 : s;
 }
-template <int BN, bool HILO>
+template <int BN, bool HILO, bool SWAP = false>
 constexpr int persist_smem_bytes() {
-  return persist_stages<BN, HILO>() * stage_bytes<BN, false, HILO>() + 2 * 128 * 128 + 1024 + 512 + 2048;
+  return persist_stages<BN, HILO, SWAP>() * stage_bytes<BN, SWAP, HILO>() + 2 * 128 * 128 + 1024 + 512 + 2048;
 }
 
-template <int BN, bool HILO>
+template <int BN, bool HILO, bool SWAP = false>
 __global__ void __launch_bounds__(THREADS)
 gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                        const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ OutMaps maps_out, int tma_out,
                        int rows_a, int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out,
                        void* __restrict__ out_lo, int ldc, int* status, const QkvDst qd, const int* __restrict__ skip,
                        int tiles_m, int tiles_n, int n_fastest) {
-  constexpr int STAGES = persist_stages<BN, HILO>();
-  constexpr int STAGE_BYTES = stage_bytes<BN, false, HILO>();
+  constexpr int STAGES = persist_stages<BN, HILO, SWAP>();
+  constexpr int STAGE_BYTES = stage_bytes<BN, SWAP, HILO>();
   constexpr int LO_OFF = BM * BK * 2 + BN * BK * 2;
   constexpr int STAGING_OFF = STAGES * STAGE_BYTES;
   constexpr int BAR_OFF = STAGING_OFF + 2 * 128 * 128;
@@ -557,7 +559,7 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
           const uint32_t sa = base + s * STAGE_BYTES;
           tma_load_2d(sa, &map_a, full_bar(s), kb * BK, m0);
           tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), kb * BK, n0);
-          if (HILO) tma_load_2d(sa + LO_OFF, &map_lo, full_bar(s), kb * BK, m0);
+          if (HILO) tma_load_2d(sa + LO_OFF, &map_lo, full_bar(s), kb * BK, SWAP ? n0 : m0);   // the activation side
         }
       }
       if (*abort_flag) {
@@ -593,8 +595,11 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
           if (HILO) {
             const uint64_t dl = make_smem_desc(sa + LO_OFF);
 #pragma unroll
-            for (int k = 0; k < BK / UMMA_K; ++k)
-              umma(acc, dl + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc, 1u);
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+              const uint64_t o = (uint64_t)(k * UMMA_K * 2 / 16);
+              if (SWAP) umma(acc, da + o, dl + o, idesc, 1u);
+              else umma(acc, dl + o, db + o, idesc, 1u);
+            }
           }
           umma_commit(empty_bar(s));
         }
@@ -609,14 +614,16 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       const int m0 = (n_fastest ? tile / tiles_n : tile % tiles_m) * BM;
       const int n0 = (n_fastest ? tile % tiles_n : tile / tiles_m) * BN;
       float* bias_s = reinterpret_cast<float*>(generic_base + BAR_OFF + 512) + buf * BN;
-      const bool use_tma = tma_out == 1 || (tma_out >= 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d));
-      const bool vt_tma = tma_out == 3 && n0 >= 2 * qd.d && n0 + BN <= rows_b;
+      const bool use_tma = !SWAP && (tma_out == 1 || (tma_out >= 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d)));
+      const bool vt_tma = !SWAP && tma_out == 3 && n0 >= 2 * qd.d && n0 + BN <= rows_b;
       if (use_tma || vt_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);  // while the tile's main loop runs
       const bool ready = named_bar_and(1, 128, mbar_wait(tfull_bar(buf), (uint32_t)(i >> 1) & 1u, abort_flag, status));
       if (!ready) break;
       fence_after_sync();
       const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
-      if (use_tma)
+      if (SWAP)
+        epilogue_manual<BN, true>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, false, qd);
+      else if (use_tma)
         epilogue_tma<BN>(acc, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &maps_out.out,
                          generic_base + STAGING_OFF, base + STAGING_OFF, n_store);
       else if (vt_tma)
@@ -849,6 +856,18 @@ static cudaError_t launch_persist(const CUtensorMap& ma, const CUtensorMap& mb, 
   return cudaGetLastError();
 }
 
+template <int BN, bool HILO>
+static cudaError_t launch_persist_swap(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const OutMaps& mo,
+                                       int rows_a, int rows_b, int K, int epi, const float* bias, void* out, void* out_lo,
+                                       int ldc, int* status, cudaStream_t st, const QkvDst& qd, const int* skip) {
+  const int tiles_m = (rows_a + BM - 1) / BM, tiles_n = (rows_b + BN - 1) / BN;
+  const long long tiles = (long long)tiles_m * tiles_n;
+  const unsigned grid = (unsigned)(tiles < 148 ? tiles : 148);
+  launch_k(gemm_tc_persist_kernel<BN, HILO, true>, dim3(grid), dim3(THREADS), persist_smem_bytes<BN, HILO, true>(), st, ma, mb, ml,
+           mo, 0, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n, 0);
+  return cudaGetLastError();
+}
+
 template <int BN, bool SWAP>
 static cudaError_t launch_hl(bool hilo, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml,
                              const OutMaps& mo, int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias,
@@ -887,6 +906,11 @@ cudaError_t tc_prepare_gemm() {
                                 persist_smem_bytes<256, false>())) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(gemm_tc_persist_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 persist_smem_bytes<256, true>())) != cudaSuccess) return e;
+#define SDD_PREP_PS(BN_, HL_)                                                                                              \
+  if ((e = cudaFuncSetAttribute(gemm_tc_persist_kernel<BN_, HL_, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
+                                persist_smem_bytes<BN_, HL_, true>())) != cudaSuccess) return e;
+  SDD_PREP_PS(32, false) SDD_PREP_PS(32, true) SDD_PREP_PS(64, false) SDD_PREP_PS(64, true)
+#undef SDD_PREP_PS
   return cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM);
 }
 
@@ -967,6 +991,18 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     if (hilo && (e = get_tensor_map(A_lo, a_cap, K, K, bn, BK, &ml)) != cudaSuccess) return e;
     OutMaps none;
     none.out = ma; none.vt = ma;
+    // many weight tiles (the LM heads): the persistent kernel keeps the weight stream going across tiles
+    // (SDD_GEMM_PERSIST=0 switches it off)
+    {
+      const char* pe = getenv("SDD_GEMM_PERSIST");
+      if ((pe == nullptr || atoi(pe) != 0) && splits == 1 && (N + BM - 1) / BM > 2 * SMS) {
+        if (bn == 32)
+          return hilo ? launch_persist_swap<32, true>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip)
+                      : launch_persist_swap<32, false>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip);
+        return hilo ? launch_persist_swap<64, true>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip)
+                    : launch_persist_swap<64, false>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip);
+      }
+    }
     if (bn == 32) return launch_hl<32, true>(hilo, ma, mb, ml, none, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
     return launch_hl<64, true>(hilo, ma, mb, ml, none, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
   }
