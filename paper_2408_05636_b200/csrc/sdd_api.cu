@@ -290,13 +290,15 @@ static bool use_tc(const sdd_ctx* c, const Net& N) {
 // head of the dead qkv buffer and into h_s), because nothing else reaches the LM head
 template <typename T, typename QkvFn, typename AttnFn, typename GatherFn>
 static int run_blocks(sdd_ctx* c, const Net& N, long long rows, int gcat, bool hilo_mlp, const int* skip, QkvFn qkv_dst,
-                      AttnFn attn, long long slot_rows, GatherFn gather) {
+                      AttnFn attn, long long slot_rows, GatherFn gather, bool first_ln_done = false) {
   const Buffers& B = c->B;
   const int d = N.d;
   for (int l = 0; l < N.n_layer; ++l) {
     const Layer& L = N.layers[l];
     const bool pruned = slot_rows > 0 && l == N.n_layer - 1;
-    SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln1_g, L.ln1_b, (T*)B.xn, rows, d, c->st, nullptr, skip));
+    // first_ln_done: the embedding kernel has already written the first block's LayerNorm to xn
+    if (!(l == 0 && first_ln_done))
+      SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, L.ln1_g, L.ln1_b, (T*)B.xn, rows, d, c->st, nullptr, skip));
     QkvDst qd = {};
     const bool fused = qkv_dst(l, &qd);
     SDD_TRY(gemm<T>(c, gcat, B.xn, c->act_elems, L.w_qkv, L.b_qkv, rows, 3 * d, d, fused ? EPI_QKV : EPI_STORE, B.qkv,
@@ -339,7 +341,8 @@ static int forward_drafter(sdd_ctx* c) {
   const long long slot_rows = (long long)D.batch * D.gamma;
   const bool prune = c->slot_prune == 1 || (c->slot_prune < 0 && rows >= 2048);
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_drafter<T>((const T*)Q.wte, (const T*)Q.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
-                                        D.batch, D.gamma, lcap, Q.d, B.h, c->st, skip));
+                                        D.batch, D.gamma, lcap, Q.d, B.h, c->st, skip, Q.layers[0].ln1_g, Q.layers[0].ln1_b,
+                                        (T*)B.xn));
   const bool tc = use_tc<T>(c, Q);
   SDD_TRY((run_blocks<T>(c, Q, rows, CAT_GEMM_Q, false, skip,
     [&](int, QkvDst* qd) -> bool {
@@ -366,7 +369,8 @@ static int forward_drafter(sdd_ctx* c) {
       SDD_LAUNCH(c, CAT_GLUE, launch_gather_slots<T>((const T*)B.att, B.h, B.ctx_len, D.batch, D.gamma, lcap, Q.d, (T*)B.qkv,
                                                      B.h_s, c->st, skip));
       return SDD_OK;
-    })));
+    },
+    true)));
   if (prune)
     SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h_s, Q.lnf_g, Q.lnf_b, (T*)B.xf, slot_rows, Q.d, c->st, nullptr, skip));
   else

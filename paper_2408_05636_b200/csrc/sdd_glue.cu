@@ -8,24 +8,76 @@ namespace sdd {
 // drafter rows: sequence b owns rows b*L_cap .. b*L_cap + L_cap - 1; row i is context token i for
 // i < c, draft slot i - c for c <= i < c + gamma, and zero padding beyond.
 // ---------------------------------------------------------------------------------------------
+constexpr int EMB_THREADS = 128;
+constexpr int EMB_MAX_PER_THREAD = 16;   // d_model <= 2048
+constexpr float EMB_LN_EPS = 1e-5f;      // the LayerNorm epsilon (same value as below)
+
+// sum over the 128 threads of an embedding block (every thread gets the result)
+__device__ __forceinline__ float emb_block_sum(float v, float* red) {
+  v = warp_sum(v);
+  __syncthreads();                       // red may still be read from the previous call
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  return (red[0] + red[1]) + (red[2] + red[3]);
+}
+
+// The embedding kernels also apply the first block's LayerNorm to the row they have just built (xn != nullptr), which
+// saves that launch: x holds the thread's elements e = tid + 128 k of the row.
 template <typename T>
-__global__ void embed_drafter_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
-                                     int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
-                                     int gamma, int L_cap, int d, float* __restrict__ h, const int* __restrict__ skip) {
+__device__ __forceinline__ void emb_layernorm_store(const float (&x)[EMB_MAX_PER_THREAD], int d, const float* __restrict__ g,
+                                                    const float* __restrict__ bta, T* __restrict__ xn_row) {
+  __shared__ float red[4];
+  float sum = 0.f;
+#pragma unroll
+  for (int k = 0; k < EMB_MAX_PER_THREAD; ++k) sum += (int)threadIdx.x + EMB_THREADS * k < d ? x[k] : 0.f;
+  const float mu = emb_block_sum(sum, red) / (float)d;
+  float var = 0.f;
+#pragma unroll
+  for (int k = 0; k < EMB_MAX_PER_THREAD; ++k) {
+    const float cdev = (int)threadIdx.x + EMB_THREADS * k < d ? x[k] - mu : 0.f;
+    var += cdev * cdev;
+  }
+  const float rstd = rsqrtf(emb_block_sum(var, red) / (float)d + EMB_LN_EPS);
+#pragma unroll
+  for (int k = 0; k < EMB_MAX_PER_THREAD; ++k) {
+    const int e = (int)threadIdx.x + EMB_THREADS * k;
+    if (e < d) xn_row[e] = from_f32<T>((x[k] - mu) * rstd * g[e] + bta[e]);
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(EMB_THREADS)
+embed_drafter_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
+                     int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
+                     int gamma, int L_cap, int d, float* __restrict__ h, const int* __restrict__ skip,
+                     const float* __restrict__ ln_g, const float* __restrict__ ln_b, T* __restrict__ xn) {
   pdl_wait();
   pdl_launch_dependents();
   if (skip != nullptr && *skip) return;
   const int i = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
-  float* __restrict__ dst = h + ((long long)b * L_cap + i) * d;
-  if (i >= c + gamma) {
-    for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = 0.f;
-    return;
+  const long long row = (long long)b * L_cap + i;
+  float* __restrict__ dst = h + row * d;
+  float x[EMB_MAX_PER_THREAD];
+  if (i >= c + gamma) {                      // padding row: zeros (its LayerNorm is the LayerNorm bias)
+#pragma unroll
+    for (int k = 0; k < EMB_MAX_PER_THREAD; ++k) x[k] = 0.f;
+  } else {
+    const int tok = i < c ? tokens[(long long)b * tok_stride + i] : slot_ids[(long long)b * gamma + (i - c)];
+    const T* __restrict__ te = wte + (long long)tok * d;
+    const T* __restrict__ pe = wpe + (long long)i * d;
+#pragma unroll
+    for (int k = 0; k < EMB_MAX_PER_THREAD; ++k) {
+      const int e = (int)threadIdx.x + EMB_THREADS * k;
+      x[k] = e < d ? to_f32(te[e]) + to_f32(pe[e]) : 0.f;
+    }
   }
-  const int tok = i < c ? tokens[(long long)b * tok_stride + i] : slot_ids[(long long)b * gamma + (i - c)];
-  const T* __restrict__ te = wte + (long long)tok * d;
-  const T* __restrict__ pe = wpe + (long long)i * d;
-  for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = to_f32(te[e]) + to_f32(pe[e]);
+#pragma unroll
+  for (int k = 0; k < EMB_MAX_PER_THREAD; ++k) {
+    const int e = (int)threadIdx.x + EMB_THREADS * k;
+    if (e < d) dst[e] = x[k];
+  }
+  if (xn != nullptr) emb_layernorm_store<T>(x, d, ln_g, ln_b, xn + row * d);
 }
 
 // target rows: sequence b owns rows b*rows_per_seq ..; VERIFY: row j = [last context token, drafts] at
@@ -253,9 +305,10 @@ __global__ void kv_append_kernel(const T* __restrict__ qkv, T* __restrict__ cach
 template <typename T>
 cudaError_t launch_embed_drafter(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                  const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st,
-                                 const int* skip) {
-  launch_k(embed_drafter_kernel<T>, dim3(dim3(L_cap, batch)), dim3(128), 0, st, wte, wpe, tokens, tok_stride, ctx_len, slot_ids, gamma,
-                                                              L_cap, d, h, skip);
+                                 const int* skip, const float* ln_g, const float* ln_b, T* xn) {
+  if (d > EMB_THREADS * EMB_MAX_PER_THREAD) return cudaErrorInvalidValue;
+  launch_k(embed_drafter_kernel<T>, dim3(L_cap, batch), dim3(EMB_THREADS), 0, st, wte, wpe, tokens, tok_stride, ctx_len, slot_ids,
+           gamma, L_cap, d, h, skip, ln_g, ln_b, xn);
   return cudaGetLastError();
 }
 template <typename T>
@@ -314,7 +367,8 @@ cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int bat
 
 #define SDD_INSTANTIATE_GLUE(T)                                                                                          \
   template cudaError_t launch_embed_drafter<T>(const T*, const T*, const int*, int, const int*, const int*, int, int,   \
-                                               int, int, float*, cudaStream_t, const int*);                             \
+                                               int, int, float*, cudaStream_t, const int*, const float*, const float*,  \
+                                               T*);                                                                     \
   template cudaError_t launch_embed_target<T>(const T*, const T*, const int*, int, const int*, const int*, int, int,    \
                                               int, int, int, float*, cudaStream_t);                                     \
   template cudaError_t launch_embed_ar<T>(const T*, const T*, const int*, int, const int*, const int*, int, int, int,   \

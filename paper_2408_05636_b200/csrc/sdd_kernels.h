@@ -67,7 +67,8 @@ cudaError_t launch_reset_slots(int* slot_ids, int* reveal_step, int n, int mask_
 template <typename T>
 cudaError_t launch_embed_drafter(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                  const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st,
-                                 const int* skip = nullptr);
+                                 const int* skip = nullptr, const float* ln_g = nullptr, const float* ln_b = nullptr,
+                                 T* xn = nullptr);   // xn != null: also xn = LayerNorm(h; ln_g, ln_b), the first block's
 template <typename T>
 cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                 const int* slot_ids, int batch, int gamma, int rows_per_seq, int mode, int d, float* h,
