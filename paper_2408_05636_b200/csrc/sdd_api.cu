@@ -537,6 +537,9 @@ int32_t sdd_workspace_bytes(const sdd_model* target, const sdd_model* drafter, c
   return SDD_OK;
 }
 
+static int load_prompts(sdd_ctx* c, const int32_t* prompt_ids, int32_t prompt_stride, const int32_t* prompt_len, int max_prompt);
+static int prefill_ar_drafter(sdd_ctx* c);
+
 int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_params* params,
                    const int32_t* prompt_ids, int32_t prompt_stride, const int32_t* prompt_len, void* workspace,
                    uint64_t workspace_bytes, sdd_ctx** out) {
@@ -611,27 +614,61 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
     SDD_CUDA(tc_prepare_gemm());
     SDD_CUDA(tc_prepare_attn());
   }
-  // zero the small state and the activations (padding rows must stay finite), then load the prompts
-  const Buffers& B = c->B;
-  const size_t state_bytes = (size_t)((uint8_t*)B.step_logits - (uint8_t*)workspace);
-  SDD_CUDA(cudaMemsetAsync(workspace, 0, state_bytes, c->st));
-  const size_t act_bytes = (size_t)((uint8_t*)B.kv - (uint8_t*)B.h);
-  SDD_CUDA(cudaMemsetAsync(B.h, 0, act_bytes, c->st));
   // the tensor-core attention multiplies masked probabilities (exact zeros) with whatever the V^T cache holds
   // past the valid positions, so that memory must be finite
-  SDD_CUDA(cudaMemsetAsync(B.kv, 0, (size_t)c->P.n_layer * params->batch * c->P.n_ctx * 2 * c->P.d * c->D.esize, c->st));
+  SDD_CUDA(cudaMemsetAsync(c->B.kv, 0, (size_t)c->P.n_layer * params->batch * c->P.n_ctx * 2 * c->P.d * c->D.esize, c->st));
+  s = load_prompts(c, prompt_ids, prompt_stride, prompt_len, max_prompt);
+  if (s != SDD_OK) return s;
+  guard.c = nullptr;
+  *out = c;
+  return SDD_OK;
+}
+
+// start of a generation: zero the small state and the activations (padding rows must stay finite), load the prompts,
+// prefill the target's KV cache with x_{0:c-2}
+static int load_prompts(sdd_ctx* c, const int32_t* prompt_ids, int32_t prompt_stride, const int32_t* prompt_len, int max_prompt) {
+  const Buffers& B = c->B;
+  const int batch = c->D.batch;
+  const size_t state_bytes = (size_t)((uint8_t*)B.step_logits - (uint8_t*)B.rs);
+  SDD_CUDA(cudaMemsetAsync(B.rs, 0, state_bytes, c->st));
+  const size_t act_bytes = (size_t)((uint8_t*)B.kv - (uint8_t*)B.h);
+  SDD_CUDA(cudaMemsetAsync(B.h, 0, act_bytes, c->st));
   SDD_CUDA(cudaMemcpy2DAsync(B.tokens, (size_t)c->D.tok_stride * 4, prompt_ids, (size_t)prompt_stride * 4,
-                             (size_t)max_prompt * 4, params->batch, cudaMemcpyDeviceToDevice, c->st));
-  SDD_CUDA(cudaMemcpyAsync(B.ctx_len, prompt_len, (size_t)params->batch * 4, cudaMemcpyHostToDevice, c->st));
-  // prefill the target's KV cache with x_{0:c-2}
+                             (size_t)max_prompt * 4, batch, cudaMemcpyDeviceToDevice, c->st));
+  SDD_CUDA(cudaMemcpyAsync(B.ctx_len, prompt_len, (size_t)batch * 4, cudaMemcpyHostToDevice, c->st));
   c->D.max_prompt = max_prompt;
+  int s;
   if (c->P.dtype == SDD_BF16) s = forward_target<__nv_bfloat16>(c, TARGET_PREFILL, max_prompt - 1, false);
   else s = forward_target<float>(c, TARGET_PREFILL, max_prompt - 1, false);
   if (s != SDD_OK) return s;
   // prompt_len is host memory owned by the caller: make sure the copy above has consumed it
   SDD_CUDA(cudaStreamSynchronize(c->st));
-  guard.c = nullptr;
-  *out = c;
+  return SDD_OK;
+}
+
+// A new generation in the same context: same models, parameters, workspace and captured graphs; new prompts.
+int32_t sdd_reset(sdd_ctx* c, const int32_t* prompt_ids, int32_t prompt_stride, const int32_t* prompt_len) {
+  if (c == nullptr || prompt_ids == nullptr || prompt_len == nullptr) return SDD_E_ARG;
+  if (c->steps_done != -1) return SDD_E_STATE;
+  const int batch = c->D.batch;
+  int max_prompt = 0;
+  for (int b = 0; b < batch; ++b) {
+    if (prompt_len[b] < 1 || prompt_len[b] > prompt_stride) return SDD_E_ARG;
+    if (c->has_ar && prompt_len[b] < 2) return SDD_E_ARG;
+    if (prompt_len[b] > max_prompt) max_prompt = prompt_len[b];
+  }
+  if ((long long)max_prompt + c->D.max_new + c->D.gamma > c->D.tok_stride) return SDD_E_CTX_FULL;
+  if (c->has_ar && (long long)max_prompt + c->D.max_new + c->D.gamma > c->A.n_ctx) return SDD_E_CTX_FULL;
+  // everything enqueued for the old generation has to be over before the host-side round bookkeeping restarts
+  SDD_CUDA(cudaStreamSynchronize(c->st));
+  c->rounds = 0;
+  c->steps_done = -1;
+  c->sps_allowed = true;
+  c->prompt_len.assign(prompt_len, prompt_len + batch);
+  c->c_ub = c->prompt_len;
+  memset(c->mirror, 0, (2 + 2 * (size_t)batch) * sizeof(int));
+  SDD_TRY(load_prompts(c, prompt_ids, prompt_stride, prompt_len, max_prompt));
+  if (c->has_ar) SDD_TRY(prefill_ar_drafter(c));
   return SDD_OK;
 }
 
@@ -799,7 +836,15 @@ int32_t sdd_sps_attach(sdd_ctx* c, const sdd_model* ar_drafter, void* workspace,
   c->ar_kv = workspace;
   c->ar_eff = (int*)((uint8_t*)workspace + align_up(kv_bytes, 256));
   SDD_CUDA(cudaMemsetAsync(workspace, 0, ar_workspace(A, c->D.batch, c->D.esize), c->st));   // V^T past the valid positions must be finite
-  // prefill its cache with x_{0:c-2}, as for the target
+  int s = prefill_ar_drafter(c);
+  if (s != SDD_OK) { c->ar_kv = nullptr; return s; }
+  c->has_ar = true;
+  return SDD_OK;
+}
+
+// prefill of the autoregressive drafter's cache with x_{0:c-2}, as for the target
+static int prefill_ar_drafter(sdd_ctx* c) {
+  const Net& A = c->A;
   const Buffers& B = c->B;
   const int rows = c->D.max_prompt - 1;
   int s = SDD_OK;
@@ -816,9 +861,7 @@ int32_t sdd_sps_attach(sdd_ctx* c, const sdd_model* ar_drafter, void* workspace,
     s = forward_causal<float>(c, A, c->ar_kv, B.ctx_len, TARGET_PREFILL, rows, false, nullptr, false, CAT_GEMM_Q, CAT_HEAD_Q,
                               CAT_ATTN_Q);
   }
-  if (s != SDD_OK) { c->ar_kv = nullptr; return s; }
-  c->has_ar = true;
-  return SDD_OK;
+  return s;
 }
 
 static int enqueue_sps_round(sdd_ctx* c, int gamma, int32_t* out_ids, int32_t* n_out) {

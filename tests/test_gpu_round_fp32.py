@@ -73,6 +73,35 @@ def test_slot_row_pruning_of_the_last_drafter_block(monkeypatch):
     s.close()
 
 
+def test_reset_equals_fresh_context():
+    """sdd_reset starts a new generation in the same context (graphs and workspace kept): the tokens must be those of
+    a fresh context on the same prompts, also after a generation that left longer sequences in the caches."""
+    import paper_2408_05636_b200 as sdd
+    wl = synth.scaled_workload(synth.WORKLOADS["tiny_fp32"], batch=2)
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    p1 = synth.prompt_ids(wl.target.vocab, 2, 40, wl.prompt_seed)
+    p2 = synth.prompt_ids(wl.target.vocab, 2, 40, wl.prompt_seed + 1)
+    s = _session(wl, dp, dq, p1, [40, 33], max_new=20, gamma=5, T=3)
+    s.generate()
+    with pytest.raises(sdd.SddError):                      # not in the middle of a round
+        s.sdd_draft_begin()
+        s.sdd_reset(p2, [12, 25])
+    for _ in range(3):
+        s.sdd_draft_step()
+    s.sdd_verify_accept()
+    s.sdd_reset(p2, [12, 25])
+    toks_a, len_a = s.generate()
+    rounds_a, _ = s.sdd_counters()
+    s.close()
+    f = _session(wl, dp, dq, p2, [12, 25], max_new=20, gamma=5, T=3)
+    toks_b, len_b = f.generate()
+    rounds_b, _ = f.sdd_counters()
+    f.close()
+    assert np.array_equal(len_a, len_b) and rounds_a == rounds_b
+    for b in range(2):
+        assert np.array_equal(toks_a[b, : len_a[b]], toks_b[b, : len_b[b]])
+
+
 def test_greedy_equals_autoregressive_greedy():
     import paper_2408_05636_b200 as sdd
     wl = synth.WORKLOADS["tiny_fp32"]
