@@ -2,11 +2,12 @@
 //
 // One CTA owns 128 query rows of one head of one sequence and walks over the keys in tiles of 128:
 //   S  = Q K^T          tcgen05.mma, 128 x 128 fp32 accumulator in TMEM (Q, K tiles via TMA, K-major)
-//   P  = exp2(S - max)  eight soft-max warps, two threads per query row (tcgen05.ld gives a thread its row);
+//   P  = exp2(S - m)    eight soft-max warps, two threads per query row (tcgen05.ld gives a thread its row), each an
+//                       independent online soft-max over its 64 keys of the tile with its own reference maximum m;
 //                       P is written as bf16 into shared memory in the 128-byte-swizzled K-major layout
-//   PV = P V            tcgen05.mma with V^T tiles ([d_head, keys], keys contiguous) as the second operand,
-//                       64-column fp32 accumulator in TMEM, folded into the per-thread output row with the
-//                       usual online-soft-max correction.
+//   PV = P V            tcgen05.mma with V^T tiles ([d_head, keys], keys contiguous) as the second operand; one
+//                       64-column fp32 accumulator per half of the key tile, accumulating over the tiles in TMEM and
+//                       rescaled there (tcgen05.ld / st) when a thread moves its reference maximum.
 // The same kernel serves the drafter (no mask: every row sees every row of its sequence) and the target
 // (row at position p sees cache positions 0..p).  V is consumed transposed, which the QKV GEMM's epilogue
 // produces for free; that keeps both MMAs on K-major operands.
@@ -34,7 +35,7 @@ constexpr int AT_STAGE_BYTES = AT_K_BYTES + AT_VT_BYTES;
 constexpr int AT_KV_STAGES = 2;
 constexpr int AT_BAR_OFF = AT_Q_BYTES + AT_P_BYTES + AT_KV_STAGES * AT_STAGE_BYTES;   // 96 KB: two CTAs per SM
 constexpr int AT_SMEM = AT_BAR_OFF + 1024 + 128 + 3 * 1024;   // barriers, then the soft-max exchange arrays
-constexpr uint32_t AT_TMEM_COLS = 256;              // S: columns 0..127, PV: columns 128..191
+constexpr uint32_t AT_TMEM_COLS = 256;              // S: columns 0..127, PV accumulators: 128..191 and 192..255
 // key-split launches add a receive area for the other CTAs' partial states (it must not lie over tiles that this CTA
 // may still be using when a faster CTA sends): at most 136 rows of 64 floats plus their m and l
 constexpr int AT_RECV_OFF = AT_BAR_OFF + 3328;
@@ -166,12 +167,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         ok = mbar_wait(p_ready, (uint32_t)t & 1u, abort_flag, prm.status);
         if (!ok) break;
         fence_after_sync();
+        // one accumulator per half of the key tile (columns 128..191: keys 0..63, 192..255: keys 64..127); both add up
+        // over the CTA's tiles in TMEM
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb) {
           const uint64_t dp = make_smem_desc(kb == 0 ? sK(s) : sP);
           const uint64_t dv = make_smem_desc(sVT(s) + kb * (64 * 64 * 2));
 #pragma unroll
-          for (int k = 0; k < 4; ++k) umma(tmem_base + 128u, dp + 2u * k, dv + 2u * k, idesc_pv, (kb | k) ? 1u : 0u);
+          for (int k = 0; k < 4; ++k)
+            umma(tmem_base + 128u + (uint32_t)(kb * 64), dp + 2u * k, dv + 2u * k, idesc_pv, (t | k) ? 1u : 0u);
         }
         umma_commit(pv_full);
         umma_commit(kv_empty(s));
@@ -196,30 +200,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     float* s_max = reinterpret_cast<float*>(gbase + AT_BAR_OFF + 128);          // [2 tile parities][2 halves][128 rows]
     float* s_l = s_max + 2 * 2 * 128;                                            // [2 halves][128 rows]
     float m = -INFINITY, l = 0.f;
-    float o[AT_DH / 2];
-#pragma unroll
-    for (int j = 0; j < AT_DH / 2; ++j) o[j] = 0.f;
     const int sw = r & 7;
     bool ok = true;
+    // The two threads of a row are independent online soft-maxes over "their" 64 keys of every tile: own reference
+    // maximum m, own sum l, own accumulator in TMEM (P_half x V_half).  The accumulator is rescaled in place, and only
+    // when the thread's maximum has grown by more than 2^8 since its reference was set (the probabilities are then
+    // bounded by 256, exact arithmetic otherwise unchanged), so the common tile has no fold, no exchange between the
+    // halves and no barrier among the warps.  The halves are combined once, after the last tile.
+    const uint32_t t_acc = t_lane + 128u + (uint32_t)(hf * 64);
+    uint32_t v[32];
     for (int it = 0; it < my_kt; ++it) {
       const int t = kv_rank + it * kv_split;           // key tile; `it` counts this CTA's iterations (stages, phases)
       ok = __all_sync(0xffffffffu, mbar_wait(s_full, (uint32_t)it & 1u, abort_flag, prm.status));
-      ok = named_bar_and(1, 256, ok);                  // also orders the reuse of s_max[it & 1] (last read two iterations ago)
       if (!ok) break;
       fence_after_sync();
       const int key0 = t * 128 + hf * 64;
       // this thread's 64 probabilities are one row of a P k-block: block 0 lies over the stage's (consumed) K tile
       uint8_t* p_row = gbase + (hf == 0 ? AT_Q_BYTES + AT_P_BYTES + (it & 1) * AT_STAGE_BYTES : AT_Q_BYTES) + r * 128;
-      // rows that see all of their 64 keys skip the per-entry visibility test
-      const bool full = key0 + 64 <= key_limit;
-      // the 64 scores are read twice from TMEM (once for the maximum, once for the exponentials) instead of being
-      // kept in 64 registers: two CTAs per SM need the kernel to stay near 100 registers
-      uint32_t v[32];
+      // tcgen05.ld / st are warp-collective: every branch around them is taken by whole warps
+      const bool full_w = __all_sync(0xffffffffu, key0 + 64 <= key_limit);
+      // the 64 scores are read twice from TMEM (once for the maximum, once for the exponentials) instead of being kept
+      // in 64 registers: two CTAs per SM need the kernel to stay below 100 registers
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
 #pragma unroll 1
       for (int cc = 0; cc < 2; ++cc) {
         tmem_ld32(t_lane + (uint32_t)(hf * 64 + cc * 32), v);
-        if (full) {
+        if (full_w) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(v[j]));
         } else {
@@ -228,63 +234,91 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             if (key0 + cc * 32 + j < key_limit) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(v[j]));
         }
       }
-      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      float* sm = s_max + (it & 1) * 256;
-      sm[hf * 128 + r] = mx;
-      named_bar_sync(2, 256);
-      mx = fmaxf(mx, sm[(hf ^ 1) * 128 + r]);
-      const float m_new = fmaxf(m, mx * scale);
-      const float m_use = m_new == -INFINITY ? 0.f : m_new;
-      const float corr = m == -INFINITY ? 0.f : ex2(m - m_use);
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-      // two copies of the loop, chosen by a real branch: the visibility tests cost a third of the issue slots when
-      // they are predicated into the common (unmasked) path
-      auto exp_pass = [&](auto full_tag) {
-        constexpr bool FULL = decltype(full_tag)::value;
-#pragma unroll 1
-        for (int cc = 0; cc < 2; ++cc) {
-          tmem_ld32(t_lane + (uint32_t)(hf * 64 + cc * 32), v);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale;     // -inf: no visible key
+      if (__any_sync(0xffffffffu, mx > m + 8.f)) {
+        // new reference for every lane of the warp (exact maximum); the accumulator and the sum follow it
+        const float m_new = fmaxf(m, mx);
+        const float corr = (m == -INFINITY || m_new == -INFINITY) ? 0.f : ex2(m - m_new);
+        if (it > 0) {
+          ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)(it - 1) & 1u, abort_flag, prm.status));
+          if (!ok) break;
+          fence_after_sync();
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint32_t pk[4];
+          for (int hh = 0; hh < 2; ++hh) {
+            tmem_ld32(t_acc + (uint32_t)(hh * 32), v);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int j0 = g * 8 + 2 * e;
-              float p0 = ex2(fmaf(__uint_as_float(v[j0]), scale, -m_use));
-              float p1 = ex2(fmaf(__uint_as_float(v[j0 + 1]), scale, -m_use));
-              if (!FULL) {
-                if (!(key0 + cc * 32 + j0 < key_limit)) p0 = 0.f;
-                if (!(key0 + cc * 32 + j0 + 1 < key_limit)) p1 = 0.f;
-              }
-              sum4[e] += p0 + p1;
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-              pk[e] = *reinterpret_cast<uint32_t*>(&h2);
-            }
-            *reinterpret_cast<uint4*>(p_row + (((cc * 4 + g) ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * corr);
+            tmem_st32(t_acc + (uint32_t)(hh * 32), v);
           }
         }
+        l *= corr;
+        m = m_new;
+      }
+      // P(t) may overwrite P(t-1) once PV(t-1) has read it (long done by now)
+      if (it > 0) {
+        ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)(it - 1) & 1u, abort_flag, prm.status));
+        if (!ok) break;
+      }
+      const float m_use = m == -INFINITY ? 0.f : m;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      auto exp_chunk = [&](auto full_tag, int cc) {
+        constexpr bool FULL = decltype(full_tag)::value;
+        tmem_ld32(t_lane + (uint32_t)(hf * 64 + cc * 32), v);
+        const uint32_t (&x)[32] = v;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int j0 = g * 8 + 2 * e;
+            float p0 = ex2(fmaf(__uint_as_float(x[j0]), scale, -m_use));
+            float p1 = ex2(fmaf(__uint_as_float(x[j0 + 1]), scale, -m_use));
+            if (!FULL) {
+              if (!(key0 + cc * 32 + j0 < key_limit)) p0 = 0.f;
+              if (!(key0 + cc * 32 + j0 + 1 < key_limit)) p1 = 0.f;
+            }
+            sum4[e] += p0 + p1;
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+          }
+          *reinterpret_cast<uint4*>(p_row + (((cc * 4 + g) ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
       };
-      // tcgen05.ld is warp-collective: the branch must not split a warp (rows past the end and causal rows have
-      // their own key_limit), so the unmasked copy runs only when every lane of the warp sees the whole tile
-      if (__all_sync(0xffffffffu, full)) exp_pass(std::true_type{});
-      else exp_pass(std::false_type{});
-      const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-      l = l * corr + sum;     // this thread's half of the row sum; the halves share m, so they add up at the end
-      m = m_new;
+      // two copies, chosen by a real (warp-uniform) branch: the visibility tests cost a third of the issue slots when
+      // they are predicated into the common unmasked path
+      if (full_w) { exp_chunk(std::true_type{}, 0); exp_chunk(std::true_type{}, 1); }
+      else { exp_chunk(std::false_type{}, 0); exp_chunk(std::false_type{}, 1); }
+      l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      fence_before_sync();          // accumulator reads / writes above are ordered before the MMA that follows the arrive
       fence_async_smem();
       mbar_arrive(p_ready);
-      ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)it & 1u, abort_flag, prm.status));
-      if (!ok) break;
-      fence_after_sync();
-      tmem_ld32(t_lane + 128u + (uint32_t)(hf * 32), v);
-#pragma unroll
-      for (int j = 0; j < 32; ++j) o[j] = fmaf(o[j], corr, __uint_as_float(v[j]));
     }
+    if (ok && my_kt > 0) ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)(my_kt - 1) & 1u, abort_flag, prm.status));
     ok = named_bar_and(1, 256, ok);
+    float o[AT_DH / 2];                                // this thread's 32 output columns (unnormalised)
+#pragma unroll
+    for (int j = 0; j < AT_DH / 2; ++j) o[j] = 0.f;
     if (ok) {
+      // combine the two halves of every row: common maximum, weights, sum; this thread's 32 output columns from both
+      // halves' accumulators
+      fence_after_sync();
+      float* s_m = s_max;                              // [2 halves][128 rows]
+      s_m[hf * 128 + r] = m;
       s_l[hf * 128 + r] = l;
       named_bar_sync(2, 256);
-      l += s_l[(hf ^ 1) * 128 + r];                    // the row sum over this CTA's key tiles
+      const float m_o = s_m[(hf ^ 1) * 128 + r], l_o = s_l[(hf ^ 1) * 128 + r];
+      const float mm = fmaxf(m, m_o);
+      const float w_me = m == -INFINITY ? 0.f : ex2(m - mm), w_o = m_o == -INFINITY ? 0.f : ex2(m_o - mm);
+      l = l * w_me + l_o * w_o;
+      m = mm;
+      if (my_kt > 0) {
+        tmem_ld32(t_lane + 128u + (uint32_t)(hf * 64 + hf * 32), v);           // own half's accumulator
+#pragma unroll
+        for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(v[j]) * w_me;
+        tmem_ld32(t_lane + 128u + (uint32_t)((hf ^ 1) * 64 + hf * 32), v);     // the other half's
+#pragma unroll
+        for (int j = 0; j < 32; ++j) o[j] = fmaf(__uint_as_float(v[j]), w_o, o[j]);
+      }
     }
     bool writes_row = kv_split == 1;
     if (kv_split > 1) {
