@@ -657,7 +657,7 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 //             their TMA loads (cta_group::2 form); the leader's producer announces the bytes of both
 //   empty[s]  (both: 1 arrive) -- the leader's MMA thread commits once to its own barrier and once to the peer's
 //   tfull[b]  (both: 1 arrive) -- leader's commit locally; its epilogue thread 64 forwards it to the peer
-//   tempty[b] (leader: 512 arrives) -- the epilogue threads of both CTAs arrive on the leader's barrier
+//   tempty[b] (leader: 16 arrives) -- the epilogue warps of both CTAs arrive on the leader's barrier
 // (with forwarding threads on the full / empty path the refill round trip exceeded what the ring covers and the
 // kernel ran at half speed)
 // The epilogues are those of the one-CTA kernels, applied by each CTA to its half; eight epilogue warps in two groups
@@ -701,7 +701,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 512); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 16); }   // one arrive per epilogue warp of the pair
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -804,9 +804,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       else
         epilogue_manual<BN, false>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, nullptr, ldc, false, qd, eg.c_begin,
                                    eg.c_end);
-      // this thread's reads of the accumulator are complete (tcgen05.wait::ld inside tmem_ld32): hand it back
+      // the warp's reads of the accumulator are complete (tcgen05.wait::ld inside tmem_ld32): hand it back, one arrive
+      // per warp
       fence_before_sync();
-      mbar_arrive_remote_relaxed(leader_tempty0 + 8u * (uint32_t)buf);
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote_relaxed(leader_tempty0 + 8u * (uint32_t)buf);
     }
     if ((int)threadIdx.x == eg.first_tid) tma_wait_group_read<0>();   // staging memory stays valid until the copies have read it
   }
