@@ -5,6 +5,11 @@
 // (cp.async.bulk.tensor, one elected producer thread), consumed by tcgen05.mma issued from one elected
 // thread, and the finished accumulator is read back with tcgen05.ld by four epilogue warps.
 //
+// Three kernels share the epilogues: gemm_tc_kernel (one tile per CTA; single-wave grids, K splits),
+// gemm_tc_persist_kernel (one CTA per SM walks over tiles with two accumulators; many-tile grids and the LM heads) and
+// gemm_tc_pair_kernel (two CTAs of a cluster share a 256 x 256 tile, tcgen05 cta_group::2; the largest GEMMs).  The host
+// picks the kernel, the tile width and the K splits (launch_gemm_tc).
+//
 // Orientation.  NORMAL: MMA-M axis = activation rows, MMA-N axis = output features (large-M GEMMs of
 // the drafter).  SWAP: MMA-M axis = output features (rows of W), MMA-N axis = tokens -- for the target's
 // verification forward, where only gamma+1 tokens exist and the kernel is a weight-streaming pass; the
