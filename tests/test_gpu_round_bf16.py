@@ -26,62 +26,31 @@ def test_small_bf16_two_rounds():
 def test_small_bf16_whole_rounds_as_the_benchmark_runs_them():
     """The headline configuration through sdd_step, i.e. in the launch configuration the benchmark times (one CUDA
     graph per round, programmatic dependent launches, skipped evaluations, key-split attention): three rounds, checked
-    on what a finished round leaves behind.  The state of the slots at denoising step k follows from the reveal steps
-    (a slot revealed at a step > k already had its final id, the others were [MASK]), so the stored q rows of the
-    slots revealed at two sampled steps per round are compared with the oracle's drafter evaluation of that state;
-    the target logits, the acceptance, the extra token and the commit are checked in full."""
+    on what a finished round leaves behind (roundcheck.check_whole_rounds)."""
     import paper_2408_05636_b200 as sdd
-    from oracle import philox as px
-    from oracle import specdiff as sd
-    from oracle.transformer import drafter_slot_logits, target_verify_logits
-    from tests import parity
     wl = synth.WORKLOADS["small_bf16"]
     mp, mq, dp, dq = roundcheck.build_pair(wl)
     prompts = synth.prompt_ids(wl.target.vocab, 1, wl.prompt_len, wl.prompt_seed)
     s = sdd.Session(dp, dq, prompts, [wl.prompt_len], wl.gamma, wl.T, wl.max_new, 1.0, 1.0, wl.philox_seed)
-    G, V = wl.gamma, wl.target.vocab
-    log = []
-    worst_q = worst_p = 0.0
-    for rnd in range(3):
-        toks = s.tap_numpy(sdd.TAP_TOKENS).reshape(1, s.tok_stride)[0]
-        c = int(s.tap_numpy(sdd.TAP_CTX_LEN)[0])
-        ctx = toks[:c].astype(np.int64)
-        s.sdd_step()
-        slots = s.tap_numpy(sdd.TAP_DRAFT_IDS).reshape(1, G)[0].astype(np.int64)
-        reveal = s.tap_numpy(sdd.TAP_REVEAL_STEP).reshape(1, G)[0]
-        qrows = s.tap_numpy(sdd.TAP_Q_LOGITS).reshape(1, G, V)[0]
-        logq = s.tap_numpy(sdd.TAP_LOGQ).reshape(1, G)[0]
-        lam = s.tap_numpy(sdd.TAP_LOGITS_P).reshape(1, G + 1, V)[0]
-        n_acc = int(s.tap_numpy(sdd.TAP_N_ACCEPT)[0])
-        extra = int(s.tap_numpy(sdd.TAP_EXTRA_TOKEN)[0])
-        prob = s.tap_numpy(sdd.TAP_ACCEPT_PROB).reshape(1, G)[0]
-        assert np.all(slots != V) and np.all((reveal >= 1) & (reveal <= wl.T))
-        steps = sorted(set(int(k) for k in reveal), reverse=True)
-        for k in (steps[0], steps[len(steps) // 2]):             # the first revealing step and a later one
-            state = np.where(reveal > k, slots, V)
-            ref = drafter_slot_logits(mq, ctx, state)
-            for j in np.nonzero(reveal == k)[0]:
-                z = qrows[j].astype(np.float64)
-                worst_q = max(worst_q, float(np.abs(z - ref[j]).max()))
-                x, gap = sd.argmax_with_gap(z + px.vocab_gumbels(wl.philox_seed, px.DRAFT, rnd, 0, int(j), 0, V))
-                if x != slots[j]:
-                    assert gap < parity.GAP_BAND
-                    log.append(("draft-near-tie", rnd, int(j), int(slots[j]), int(x), float(gap)))
-                assert abs(logq[j] - (z[slots[j]] - sd.logsumexp(z))) < 1e-5
-                # the reveal test of this slot: passed at step k, failed at every earlier step k' > k
-                for kk in range(wl.T, k - 1, -1):
-                    u = px.scalar_uniform(wl.philox_seed, px.UNMASK, rnd, kk, int(j), 0)
-                    assert (u < 1.0 / kk) == (kk == k)
-        ref_p = target_verify_logits(mp, ctx, slots)
-        worst_p = max(worst_p, float(np.abs(lam - ref_p).max()))
-        parity.check_accept(lam, qrows, logq, slots, 1.0, 1.0, wl.philox_seed, rnd, 0, n_acc, extra, prob, log)
-        toks2 = s.tap_numpy(sdd.TAP_TOKENS).reshape(1, s.tok_stride)[0]
-        c2 = int(s.tap_numpy(sdd.TAP_CTX_LEN)[0])
-        want = [int(x) for x in slots[:n_acc]] + [extra]
-        assert c2 == c + n_acc + 1 and list(toks2[c:c2]) == want
-        assert list(s.out_ids.cpu().numpy()[0, : n_acc + 1]) == want
+    log, worst_q, worst_p = roundcheck.check_whole_rounds(s, mp, mq, wl, 3, TOL, seqs=[0])
     print("near-ties:", log, "max logit err q/p:", worst_q, worst_p)
-    assert worst_q < TOL and worst_p < TOL and len(log) <= 2
+    assert len(log) <= 2
+    s.close()
+
+
+def test_xl_bf16_b16_one_round_sampled_sequence():
+    """The serving configuration at full size (48-layer d1600 target, 24-layer d1024 drafter, 16 sequences with
+    1024-token prompts, gamma 16, T 8), one round through sdd_step as the benchmark runs it: CTA-pair GEMMs,
+    persistent GEMMs, slot-row pruning.  One sequence of the sixteen is followed by the oracle: one sampled drafter
+    state, the target logits, the acceptance and the commit."""
+    import paper_2408_05636_b200 as sdd
+    wl = synth.WORKLOADS["xl_bf16_b16"]
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, wl.batch, wl.prompt_len, wl.prompt_seed)
+    s = sdd.Session(dp, dq, prompts, [wl.prompt_len] * wl.batch, wl.gamma, wl.T, wl.max_new, 1.0, 1.0, wl.philox_seed)
+    log, worst_q, worst_p = roundcheck.check_whole_rounds(s, mp, mq, wl, 1, TOL, seqs=[9], n_sampled_steps=1)
+    print("near-ties:", log, "max logit err q/p:", worst_q, worst_p)
+    assert len(log) <= 1
     s.close()
 
 
