@@ -103,6 +103,23 @@ def test_small_bf16_batch12_sampled_sequences(pairs, monkeypatch):
     s.close()
 
 
+@pytest.mark.parametrize("gamma,T", [(64, 32), (32, 16)])
+def test_small_bf16_sweep_corner_whole_rounds(gamma, T):
+    """The serving sweep's largest draft length and step count (gamma 64, T 32) and its middle point, on the
+    GPT-2-small-shaped pair with two sequences of different lengths: two rounds through sdd_step.  65 (33) target rows
+    per sequence, 64 (32) slot rows per LM head, many evaluations that reveal nothing (skipped), reveal steps spread
+    over 1..T.  Both sequences are followed by the oracle on two sampled denoising states per round."""
+    import paper_2408_05636_b200 as sdd
+    wl = synth.scaled_workload(synth.WORKLOADS["small_bf16"], batch=2, gamma=gamma, T=T)
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 2, 300, wl.prompt_seed)
+    s = sdd.Session(dp, dq, prompts, [300, 171], gamma, T, 4 * (gamma + 1), 1.0, 1.0, wl.philox_seed)
+    log, worst_q, worst_p = roundcheck.check_whole_rounds(s, mp, mq, wl, 2, TOL, seqs=[0, 1])
+    print("near-ties:", log, "max logit err q/p:", worst_q, worst_p)
+    assert len(log) <= 2
+    s.close()
+
+
 def test_xl_bf16_one_round_reduced_T():
     """GPT-2-XL-shaped target (48L d1600 h25) with the 24L d1024 drafter, prompt 512, gamma 32; one round with
     T = 2 denoising evaluations (the oracle needs about 3 TFLOP in fp64 for this round)."""
