@@ -56,7 +56,9 @@ enum { SDD_FP32 = 0, SDD_BF16 = 1 };
  *   then lnf_g[d] lnf_b[d].                       (n_tensors = 2 + 12 * n_layer + 2)
  * Linear weights are [out_features, in_features] row-major (y = x W^T + b).  With dtype ==
  * SDD_BF16 the matrices (wte, wpe, w_*) are bf16 and the vectors (ln*, b_*) are fp32; with
- * SDD_FP32 everything is fp32.  All pointers must be 16-byte aligned. */
+ * SDD_FP32 everything is fp32.  All pointers must be 16-byte aligned.  The tensors are borrowed and must
+ * not change while a context that uses them has work queued: kernels read weight tiles before they wait for
+ * the work ahead of them in the stream. */
 typedef struct {
   int32_t vocab, n_layer, d_model, n_head, n_ctx;
   int32_t causal; /* 1 = autoregressive target, 0 = masked-diffusion drafter */
@@ -213,7 +215,9 @@ int32_t sdd_accept_logits_static(const float* logits_p, const float* logits_q, c
  *   A_lo (may be null) second half of a hi/lo activation pair, same shape as A: the product uses A + A_lo
  *        (how the target's MLP and LM head carry their activations to about 16 significant bits)
  *   out_lo (may be null; epilogues 0 and 1) receives bf16(x - bf16(x)) next to out = bf16(x)
- * K must be a multiple of 8; A, A_lo and W 16-byte aligned. */
+ * K must be a multiple of 8; A, A_lo and W 16-byte aligned.  W must be complete in memory when the call is made (not
+ * the output of work still running on `stream`): like the weights of a model it is fetched before the kernel waits
+ * for the work ahead of it in the stream. */
 int32_t sdd_debug_gemm_bf16(const void* A, int64_t a_rows_capacity, const void* W, const float* bias, int32_t M,
                             int32_t N, int32_t K, int32_t epilogue, void* out, int32_t ldc, int32_t n_tile,
                             int32_t use_tensor_cores, int32_t* status_word, void* stream, const void* A_lo,

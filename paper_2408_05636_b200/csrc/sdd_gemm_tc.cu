@@ -389,24 +389,51 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
-  // everything above touched only shared / tensor memory; global inputs may still be in production
+  // Everything above touched only shared / tensor memory; the activations may still be in production.  The weight
+  // operand (B, or A in the swapped orientation) is never written while the library runs, so the first fill of the
+  // ring with weight tiles starts here, under the tail of the kernel ahead in the stream: the bytes are announced
+  // without an arrive, the stage's arrive follows with the activation tiles after the wait.  The early look at the
+  // skip flag only decides whether to fetch ahead; a stale value costs time, not correctness.
+  constexpr uint32_t W_BYTES = (SWAP ? BM : BN) * BK * 2;
+  int n_pre = 0;
+  if (threadIdx.x == 0 && (skip == nullptr || *reinterpret_cast<const volatile int*>(skip) == 0)) {
+    n_pre = min(num_kb, STAGES);
+    for (int kb = 0; kb < n_pre; ++kb) {
+      mbar_expect_tx_only(full_bar(kb), W_BYTES);
+      const uint32_t sa = base + kb * STAGE_BYTES;
+      if (SWAP) tma_load_2d(sa, &map_a, full_bar(kb), (kb0 + kb) * BK, m0);
+      else tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(kb), (kb0 + kb) * BK, n0);
+    }
+  }
   pdl_wait();
   pdl_launch_dependents();
   // launches of a drafter evaluation do nothing when the evaluation is skipped (they still free their TMEM below)
   const bool active = skip == nullptr || *skip == 0;
 
   if (!active) {
+    // weight tiles fetched ahead must have landed before the CTA gives its shared memory back
+    for (int kb = 0; kb < n_pre; ++kb) {
+      mbar_arrive(full_bar(kb));
+      const long long t0 = clock64();
+      while (!mbar_try(full_bar(kb), 0u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+    }
   } else if (warp == 0) {
     if (lane == 0) {
       int issued = 0;
       for (int kb = 0; kb < num_kb; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, status)) break;
-        mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES);
         const uint32_t sa = base + s * STAGE_BYTES;
-        tma_load_2d(sa, &map_a, full_bar(s), (kb0 + kb) * BK, m0);
-        tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), (kb0 + kb) * BK, n0);
+        if (kb < n_pre) {
+          mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES - W_BYTES);      // the weight tile is already on its way
+          if (SWAP) tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), (kb0 + kb) * BK, n0);
+          else tma_load_2d(sa, &map_a, full_bar(s), (kb0 + kb) * BK, m0);
+        } else {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, status)) break;
+          mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES);
+          tma_load_2d(sa, &map_a, full_bar(s), (kb0 + kb) * BK, m0);
+          tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), (kb0 + kb) * BK, n0);
+        }
         if (HILO) tma_load_2d(sa + LO_OFF, &map_lo, full_bar(s), (kb0 + kb) * BK, SWAP ? n0 : m0);
         issued = kb + 1;
       }
@@ -544,11 +571,33 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // the first ring fill of weight tiles starts before the wait for the kernel ahead (see gemm_tc_kernel)
+  constexpr uint32_t W_BYTES = (SWAP ? BM : BN) * BK * 2;
+  int n_pre = 0;
+  if (threadIdx.x == 0 && (int)blockIdx.x < n_tiles && (skip == nullptr || *reinterpret_cast<const volatile int*>(skip) == 0)) {
+    const long long mine = (long long)((n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * num_kb;
+    n_pre = (int)(mine < STAGES ? mine : STAGES);
+    for (int j = 0; j < n_pre; ++j) {
+      const int tile = (int)blockIdx.x + (j / num_kb) * (int)gridDim.x, kb = j % num_kb;
+      const int m0 = (n_fastest ? tile / tiles_n : tile % tiles_m) * BM;
+      const int n0 = (n_fastest ? tile % tiles_n : tile / tiles_m) * BN;
+      mbar_expect_tx_only(full_bar(j), W_BYTES);
+      const uint32_t sa = base + j * STAGE_BYTES;
+      if (SWAP) tma_load_2d(sa, &map_a, full_bar(j), kb * BK, m0);
+      else tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(j), kb * BK, n0);
+    }
+  }
   pdl_wait();
   pdl_launch_dependents();
   const bool active = skip == nullptr || *skip == 0;
 
   if (!active) {
+    // weight tiles fetched ahead must have landed before the CTA gives its shared memory back
+    for (int j = 0; j < n_pre; ++j) {
+      mbar_arrive(full_bar(j));
+      const long long t0 = clock64();
+      while (!mbar_try(full_bar(j), 0u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+    }
   } else if (warp == 0) {
     if (lane == 0) {
       long long it = 0;
@@ -559,11 +608,17 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = (int)(it % STAGES);
           const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, status)) { ok = false; break; }
-          mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES);
           const uint32_t sa = base + s * STAGE_BYTES;
-          tma_load_2d(sa, &map_a, full_bar(s), kb * BK, m0);
-          tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), kb * BK, n0);
+          if (it < n_pre) {
+            mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES - W_BYTES);    // the weight tile is already on its way
+            if (SWAP) tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), kb * BK, n0);
+            else tma_load_2d(sa, &map_a, full_bar(s), kb * BK, m0);
+          } else {
+            if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, status)) { ok = false; break; }
+            mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES);
+            tma_load_2d(sa, &map_a, full_bar(s), kb * BK, m0);
+            tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), kb * BK, n0);
+          }
           if (HILO) tma_load_2d(sa + LO_OFF, &map_lo, full_bar(s), kb * BK, SWAP ? n0 : m0);   // the activation side
         }
       }
