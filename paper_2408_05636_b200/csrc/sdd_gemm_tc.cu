@@ -208,7 +208,7 @@ __device__ __forceinline__ void epilogue_vt(uint32_t tmem_acc, int q, int lane, 
   }
 }
 
-template <int BN, bool SWAP>
+template <int BN, bool SWAP, bool ROLL = false>
 __device__ __forceinline__ void epilogue_manual(uint32_t tmem_acc, int m0, int n0, int q, int lane, int rows_a, int rows_b,
                                                 int epi, const float* __restrict__ bias, void* __restrict__ out,
                                                 void* __restrict__ out_lo, int ldc, bool split, const QkvDst& qd,
@@ -305,38 +305,50 @@ __device__ __forceinline__ void epilogue_manual(uint32_t tmem_acc, int m0, int n
       }
     } else {
       // out[c][r]: c = token, r = feature; consecutive lanes write consecutive features
+      // ROLL: a rolled loop over the valid tokens only.  Unrolled 32 times, this body (every epilogue kind, the
+      // cache arithmetic of the fused QKV) is tens of kilobytes of straight-line code; a CTA of the one-tile kernel
+      // runs through it once, and the few-CTA weight-streaming launches then spend their time fetching instructions
+      // (100 KB -> 14 KB of code per kernel).  v[] is then indexed dynamically, i.e. it passes through local memory
+      // (32 words per thread).  The persistent kernel repeats its epilogue tile after tile and keeps the unrolled form.
       const float bv = (bias != nullptr && r_ok) ? bias[r] : 0.f;
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const int c = c0 + j;
-        if (r_ok && c < rows_b) {
-          float x = __uint_as_float(v[j]) + bv;
-          const long long o = (long long)c * ldc + r;
-          if (epi == EPI_QKV) {
-            if (r < qd.d || (r < 2 * qd.d && qd.k_dst == nullptr)) {
-              reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(x);
-            } else {
-              const int sb = c / qd.rows_per_seq, si = c - sb * qd.rows_per_seq;
-              const int cl = qd.ctx_len[sb];
-              const int pos = qd.mode == 1 ? cl - 1 + si : si;
-              if (qd.mode != 2 || si < cl - 1) {
-                if (r < 2 * qd.d) {
-                  if (pos < qd.k_seq_rows)
-                    qd.k_dst[((long long)sb * qd.k_seq_rows + pos) * qd.d + (r - qd.d)] = __float2bfloat16_rn(x);
-                } else if (pos < qd.vt_ld) {
-                  qd.vt_dst[((long long)sb * qd.d + (r - 2 * qd.d)) * qd.vt_ld + pos] = __float2bfloat16_rn(x);
-                }
+      auto put = [&](int c, float acc) {
+        float x = acc + bv;
+        const long long o = (long long)c * ldc + r;
+        if (epi == EPI_QKV) {
+          if (r < qd.d || (r < 2 * qd.d && qd.k_dst == nullptr)) {
+            reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(x);
+          } else {
+            const int sb = c / qd.rows_per_seq, si = c - sb * qd.rows_per_seq;
+            const int cl = qd.ctx_len[sb];
+            const int pos = qd.mode == 1 ? cl - 1 + si : si;
+            if (qd.mode != 2 || si < cl - 1) {
+              if (r < 2 * qd.d) {
+                if (pos < qd.k_seq_rows)
+                  qd.k_dst[((long long)sb * qd.k_seq_rows + pos) * qd.d + (r - qd.d)] = __float2bfloat16_rn(x);
+              } else if (pos < qd.vt_ld) {
+                qd.vt_dst[((long long)sb * qd.d + (r - 2 * qd.d)) * qd.vt_ld + pos] = __float2bfloat16_rn(x);
               }
             }
-          } else if (epi == EPI_STORE || epi == EPI_GELU) {
-            if (epi == EPI_GELU) x = gelu_tanh_fast(x);
-            const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-            reinterpret_cast<__nv_bfloat16*>(out)[o] = hi;
-            if (out_lo != nullptr) reinterpret_cast<__nv_bfloat16*>(out_lo)[o] = __float2bfloat16_rn(x - __bfloat162float(hi));
           }
-          else if (epi == EPI_RESIDUAL) { if (split) atomicAdd(reinterpret_cast<float*>(out) + o, x); else reinterpret_cast<float*>(out)[o] += x; }
-          else reinterpret_cast<float*>(out)[o] = x;
+        } else if (epi == EPI_STORE || epi == EPI_GELU) {
+          if (epi == EPI_GELU) x = gelu_tanh_fast(x);
+          const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+          reinterpret_cast<__nv_bfloat16*>(out)[o] = hi;
+          if (out_lo != nullptr) reinterpret_cast<__nv_bfloat16*>(out_lo)[o] = __float2bfloat16_rn(x - __bfloat162float(hi));
         }
+        else if (epi == EPI_RESIDUAL) { if (split) atomicAdd(reinterpret_cast<float*>(out) + o, x); else reinterpret_cast<float*>(out)[o] += x; }
+        else reinterpret_cast<float*>(out)[o] = x;
+      };
+      if (ROLL) {
+        const int jn = rows_b - c0 < 32 ? rows_b - c0 : 32;
+        if (r_ok) {
+#pragma unroll 1
+          for (int j = 0; j < jn; ++j) put(c0 + j, __uint_as_float(v[j]));
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (r_ok && c0 + j < rows_b) put(c0 + j, __uint_as_float(v[j]));
       }
     }
   }
@@ -502,7 +514,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                       m0 - sb * qd.rows_per_seq);
       if (threadIdx.x == 64) tma_wait_group_read<0>();
     } else if (ready) {
-      epilogue_manual<BN, SWAP>(tmem_base, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, split, qd);
+      epilogue_manual<BN, SWAP, SWAP>(tmem_base, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, split, qd);
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
