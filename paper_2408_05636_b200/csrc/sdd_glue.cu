@@ -193,12 +193,20 @@ template <typename T, int NV>
 __global__ void __launch_bounds__(128)
 layernorm_vec_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
                      T* __restrict__ out, T* __restrict__ out_lo, long long rows, int d, const int* __restrict__ skip) {
+  // gain and bias are weights (never written while the library runs): fetched before the wait for the kernel ahead
+  const int lane = threadIdx.x & 31;
+  float4 gg[NV], bb[NV];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int e = (i * 32 + lane) * 4;
+    if (e < d) { gg[i] = *reinterpret_cast<const float4*>(g + e); bb[i] = *reinterpret_cast<const float4*>(bta + e); }
+    else { gg[i] = make_float4(0.f, 0.f, 0.f, 0.f); bb[i] = gg[i]; }
+  }
   pdl_wait();
   pdl_launch_dependents();
   if (skip != nullptr && *skip) return;
   const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
   if (row >= rows) return;
-  const int lane = threadIdx.x & 31;
   const float* __restrict__ src = h + row * d;
   float4 x[NV];
   float sum = 0.f;
@@ -224,9 +232,8 @@ layernorm_vec_kernel(const float* __restrict__ h, const float* __restrict__ g, c
   for (int i = 0; i < NV; ++i) {
     const int e = (i * 32 + lane) * 4;
     if (e < d) {
-      const float4 gg = *reinterpret_cast<const float4*>(g + e), bb = *reinterpret_cast<const float4*>(bta + e);
-      const float y0 = (x[i].x - mu) * rstd * gg.x + bb.x, y1 = (x[i].y - mu) * rstd * gg.y + bb.y;
-      const float y2 = (x[i].z - mu) * rstd * gg.z + bb.z, y3 = (x[i].w - mu) * rstd * gg.w + bb.w;
+      const float y0 = (x[i].x - mu) * rstd * gg[i].x + bb[i].x, y1 = (x[i].y - mu) * rstd * gg[i].y + bb[i].y;
+      const float y2 = (x[i].z - mu) * rstd * gg[i].z + bb[i].z, y3 = (x[i].w - mu) * rstd * gg[i].w + bb[i].w;
       store4<T>(dst + e, y0, y1, y2, y3);
       if (out_lo != nullptr)   // second half of a hi/lo pair
         store4<T>(out_lo + row * d + e, y0 - to_f32<T>(from_f32<T>(y0)), y1 - to_f32<T>(from_f32<T>(y1)),
