@@ -16,7 +16,7 @@ Readings of the paper taken here (the paper is silent or garbled on each):
     the network's categorical for that slot; revealed slots never change again.
   * The drafter takes tokens only (no time-step input).
   * q_j in the acceptance ratio is the distribution slot j's token was actually drawn
-    from (the logits of the step that revealed it, "the logits of which are stored").
+    from: the logits of the step that revealed it, kept from then on (Section "SpecDiff: Formulation").
   * gamma+1 target rows: row j is the distribution after context ∘ draft[0:j].
   * "r > p/q  => reject" is evaluated as: accept iff u <= min(1, p/q), in log space.
   * "if n < i + gamma" in Algorithm 1 means n < gamma.
@@ -25,8 +25,8 @@ Readings of the paper taken here (the paper is silent or garbled on each):
   * temperature tau divides the logits; tau = 0 is greedy decoding (the setting of every
     result the paper reports).
   * the last round's emission is truncated to `max_new`.
-  * "Sequence initialization" names standard speculative decoding for "the initial few tokens" (the evaluation
-    says the first 100) and nothing more.  Taken here: whole speculative-decoding rounds with an autoregressive
+  * Section "Sequence initialization" names standard speculative decoding for the start of a sequence (the
+    evaluation: its first 100 tokens) and nothing more.  Taken here: whole speculative-decoding rounds with an autoregressive
     drafter run while fewer than `n_init` tokens have been generated; the round that crosses `n_init` is kept
     whole; the rounds share one round counter (and so one random stream layout) with the diffusion rounds.
 MDLM-faithfulness of the unmasking rule: parity unpinned (MDLM's sampler is not available).
@@ -158,7 +158,7 @@ def sps_draft(model_a: Model, ctx_ids: np.ndarray, gamma: int, tau_q: float, see
 
 
 # ----------------------------------------------------------------------------------
-# acceptance and the extra token (Algorithm 1, from "Determine the number of accepted guesses")
+# acceptance and the extra token (Algorithm 1, from the acceptance block to the return statement)
 # ----------------------------------------------------------------------------------
 
 def q_probs(qrow: np.ndarray, draft_id: int, tau_q: float) -> np.ndarray:
@@ -215,6 +215,17 @@ def accept_resample(lam: np.ndarray, qrows: np.ndarray, logq: np.ndarray, draft_
     n = 0
     while n < gamma and us[n] <= ratio[n]:
         n += 1
+    t, gap, score = extra_token(lam, qrows, draft_ids, n, tau_p, tau_q, seed, rnd, b)
+    return AcceptResult(n, t, ratio, us, logp, sum_min, gap, score if keep_scores else None)
+
+
+def extra_token(lam: np.ndarray, qrows: np.ndarray, draft_ids: np.ndarray, n: int, tau_p: float, tau_q: float,
+                seed: int, rnd: int, b: int):
+    """The token that follows n accepted drafts (Algorithm 1, the block that adjusts the distribution): for
+    n < gamma a draw from norm(max(0, p_n - q_n)), for n == gamma a draw from p_gamma.
+    Returns (token, top-2 gap of the Gumbel scores, scores)."""
+    gamma, V = qrows.shape
+    lam = np.asarray(lam, dtype=np.float64)
     if n < gamma:
         p = p_probs(lam[n], tau_p)
         q = q_probs(qrows[n], int(draft_ids[n]), tau_q)
@@ -232,7 +243,7 @@ def accept_resample(lam: np.ndarray, qrows: np.ndarray, logq: np.ndarray, draft_
         else:
             score = lam[gamma]
     t, gap = argmax_with_gap(score)
-    return AcceptResult(n, t, ratio, us, logp, sum_min, gap, score if keep_scores else None)
+    return t, gap, score
 
 
 # ----------------------------------------------------------------------------------

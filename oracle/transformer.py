@@ -99,7 +99,7 @@ def drafter_slot_logits(model_q: Model, ctx_ids: np.ndarray, slot_ids: np.ndarra
 
 
 def target_verify_logits(model_p: Model, ctx_ids: np.ndarray, draft_ids: np.ndarray) -> np.ndarray:
-    """The gamma+1 target distributions of Algorithm 1 ("Run M_p in parallel"), as logits:
+    """The gamma+1 target distributions of Algorithm 1 (its parallel evaluation of M_p), as logits:
     row j is the next-token logits after x_{0:c-1} ∘ draft[0:j], j = 0..gamma; fp64 [gamma+1, V].
     Written as the plain definition: one causal forward over all c+gamma tokens."""
     c, g = len(ctx_ids), len(draft_ids)
