@@ -44,7 +44,10 @@ enum {
   SDD_E_CUDA = -5,       /* a CUDA runtime / driver call failed (see sdd_last_cuda_error)      */
   SDD_E_TIMEOUT = -6,    /* a bounded device-side wait ran out; the device stays usable        */
   SDD_E_UNIMPL = -7,     /* option combination not implemented                                 */
-  SDD_E_STATE = -8       /* call order violated (e.g. verify before draft)                     */
+  SDD_E_STATE = -8,      /* call order violated (e.g. verify before draft)                     */
+  SDD_E_INDEX = -9       /* a token id outside [0, vocab) reached the device (prompt or draft ids):
+                            it was replaced by a zero embedding / a rejected draft, never used as an
+                            index; reported by sdd_sync_status                                     */
 };
 
 enum { SDD_FP32 = 0, SDD_BF16 = 1 };
@@ -86,6 +89,8 @@ int32_t sdd_workspace_bytes(const sdd_model* target, const sdd_model* drafter, c
 
 /* Set up one generation (Section "Preliminaries": prefix x_{1:i} in, next n tokens out).
  *   prompt_ids : device int32 [batch, prompt_stride], row b holds prompt_len[b] ids in [0, vocab)
+ *                (the host cannot see them: an id outside that range becomes a zero embedding row on
+ *                the device and sdd_sync_status returns SDD_E_INDEX)
  *   prompt_len : host int32 [batch], each >= 1
  *   workspace  : device memory, 256-byte aligned, >= sdd_workspace_bytes(); zeroed by this call
  * Also enqueues the target's prefill of x_{0:c-2} into its KV cache.  *out receives the context
@@ -104,7 +109,7 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
  * SDD_E_CTX_FULL / SDD_E_ARG as for sdd_create. */
 int32_t sdd_reset(sdd_ctx* ctx, const int32_t* prompt_ids, int32_t prompt_stride, const int32_t* prompt_len);
 
-/* Drafting (Algorithm 1, "Take T diffusion steps to generate the draft" and "x ~ q^0"):
+/* Drafting (Algorithm 1, the loop over the T diffusion steps and the draw of the draft from q^0):
  *   sdd_draft_begin : all gamma slots <- [MASK]
  *   sdd_draft_step  : one denoising evaluation k = T, T-1, ... : drafter forward over
  *                     context ∘ slots, LM head on the slot rows, then each still-masked slot is
@@ -116,7 +121,7 @@ int32_t sdd_draft_begin(sdd_ctx* ctx);
 int32_t sdd_draft_step(sdd_ctx* ctx);
 int32_t sdd_draft(sdd_ctx* ctx);
 
-/* Verification and acceptance (Algorithm 1 from "Run M_p in parallel" to "Return"): one causal,
+/* Verification and acceptance (Algorithm 1 from the parallel evaluation of M_p to its return statement): one causal,
  * KV-cached target forward over [last context token, draft_1..draft_gamma], the acceptance test,
  * the extra token, and the commit of n+1 tokens to every sequence's context.  Requires a finished
  * draft (SDD_E_STATE otherwise).  If non-null, out_ids (device int32 [batch, gamma+1]) receives
@@ -173,7 +178,10 @@ int32_t sdd_progress(sdd_ctx* ctx, uint64_t* rounds_done, int32_t* min_emitted);
  *   accept_prob fp32 [rows, gamma]      out: min(1, p/q) of every row (also past the rejection)
  *   scratch   device, >= sdd_accept_scratch_bytes(rows, gamma, V) bytes, 16-byte aligned
  * logits_p and logits_q must be 16-byte aligned.  Row b uses Philox sequence index b and round
- * index `round`.  rows <= 65535, gamma <= 256, temp_p and temp_q both 0 (greedy) or both > 0. */
+ * index `round`, of which the low 32 bits are used (the Philox counter word that carries the round
+ * is 32 bits wide; the rounds of a context are counted in 32 bits too).  rows <= 65535,
+ * gamma <= 256, temp_p and temp_q both 0 (greedy) or both > 0.  A draft id outside [0, V) is never
+ * used as an index: that sequence gets n_accept = -1 and out_ids all -1. */
 uint64_t sdd_accept_scratch_bytes(int32_t rows, int32_t gamma, int32_t V);
 int32_t sdd_accept_logits(const float* logits_p, const float* logits_q, const int32_t* draft_ids,
                           int32_t rows, int32_t gamma, int32_t V, float temp_p, float temp_q,
@@ -241,6 +249,13 @@ int32_t sdd_debug_attention_bf16(const void* q, int64_t q_rows_total, int32_t q_
                                  int32_t batch, int32_t n_head, int32_t gamma, int32_t mode, int32_t q_rows_per_seq,
                                  int32_t* status_word, void* stream);
 
+/* Diagnostic: one CTA with the tensor-core kernels' role layout (copy producer, MMA issuer, epilogue warps, TMEM
+ * allocation) whose consumer waits on a barrier that nothing arrives on, with the kernels' own bounded wait and a
+ * limit of limit_cycles SM clocks (1 .. 2e9).  The wait runs out, the CTA raises its abort flag and *status_word =
+ * 1, every role leaves its loop, TMEM is freed and the kernel returns: the path a stuck copy or MMA would take in
+ * the GEMM and attention kernels, exercised without a fault.  status_word: device int32, must be 0 before the call. */
+int32_t sdd_debug_wait_timeout(int64_t limit_cycles, int32_t* status_word, void* stream);
+
 /* Read-only device views into the workspace, for inspection and tests. */
 enum {
   SDD_TAP_TOKENS = 0,      /* int32 [batch, tok_stride] context ids (prompt + emitted);
@@ -256,7 +271,9 @@ enum {
   SDD_TAP_N_ACCEPT = 9,    /* int32 [batch]                                                     */
   SDD_TAP_EXTRA_TOKEN = 10,/* int32 [batch]                                                     */
   SDD_TAP_N_EMITTED = 11,  /* int32 [batch]             tokens generated so far                 */
-  SDD_TAP_STATUS = 12      /* int32 [1]                 device status word (0 = ok)             */
+  SDD_TAP_STATUS = 12,     /* int32 [1]                 device status word (0 = ok)             */
+  SDD_TAP_EVALS = 13       /* int32 [2]                 drafter evaluations of this generation that
+                              ran / that were skipped because the step before revealed nothing  */
 };
 int32_t sdd_tap(sdd_ctx* ctx, int32_t what, const void** dev_ptr, uint64_t* bytes);
 

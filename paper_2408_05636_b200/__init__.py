@@ -19,11 +19,11 @@ LIB_PATH = os.path.join(_HERE, "libsdd.so")
 
 SDD_OK = 0
 SDD_E_ARG, SDD_E_SHAPE, SDD_E_WORKSPACE, SDD_E_CTX_FULL = -1, -2, -3, -4
-SDD_E_CUDA, SDD_E_TIMEOUT, SDD_E_UNIMPL, SDD_E_STATE = -5, -6, -7, -8
+SDD_E_CUDA, SDD_E_TIMEOUT, SDD_E_UNIMPL, SDD_E_STATE, SDD_E_INDEX = -5, -6, -7, -8, -9
 SDD_FP32, SDD_BF16 = 0, 1
 
 (TAP_TOKENS, TAP_CTX_LEN, TAP_DRAFT_IDS, TAP_STEP_LOGITS, TAP_Q_LOGITS, TAP_LOGQ, TAP_REVEAL_STEP,
- TAP_LOGITS_P, TAP_ACCEPT_PROB, TAP_N_ACCEPT, TAP_EXTRA_TOKEN, TAP_N_EMITTED, TAP_STATUS) = range(13)
+ TAP_LOGITS_P, TAP_ACCEPT_PROB, TAP_N_ACCEPT, TAP_EXTRA_TOKEN, TAP_N_EMITTED, TAP_STATUS, TAP_EVALS) = range(14)
 
 PROF_NAMES = ["gemm_drafter", "gemm_target", "head_drafter", "head_target", "attn_drafter", "attn_target",
               "layernorm", "glue", "sample", "row_stats", "accept", "commit"]
@@ -32,7 +32,7 @@ EXPORTS = [
     "sdd_workspace_bytes", "sdd_create", "sdd_reset", "sdd_draft_begin", "sdd_draft_step", "sdd_draft",
     "sdd_verify_accept", "sdd_step", "sdd_ar_step", "sdd_sps_workspace_bytes", "sdd_sps_attach", "sdd_sps_step",
     "sdd_progress", "sdd_accept_scratch_bytes", "sdd_accept_logits",
-    "sdd_accept_logits_static", "sdd_debug_gemm_bf16", "sdd_debug_attention_bf16",
+    "sdd_accept_logits_static", "sdd_debug_gemm_bf16", "sdd_debug_attention_bf16", "sdd_debug_wait_timeout",
     "sdd_tap", "sdd_counters", "sdd_profile_begin", "sdd_profile_end", "sdd_sync_status", "sdd_destroy", "sdd_strerror", "sdd_last_cuda_error",
 ]
 
@@ -88,6 +88,7 @@ def lib() -> C.CDLL:
         L.sdd_debug_gemm_bf16.argtypes = [vp, C.c_int64, vp, vp, i32, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp]
         L.sdd_debug_attention_bf16.argtypes = [vp, C.c_int64, i32, i32, vp, C.c_int64, i32, i32, i32, vp, i32, vp, i32, vp,
                                                i32, i32, i32, i32, i32, vp, vp]
+        L.sdd_debug_wait_timeout.argtypes = [C.c_int64, vp, vp]
         L.sdd_tap.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(u64)]
         L.sdd_counters.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
         L.sdd_profile_begin.argtypes = [vp]
@@ -193,6 +194,8 @@ def sdd_accept_logits_static(logits_p, logits_q, draft_ids, n_accept, out_ids, a
     assert n_accept.shape == (rows,) and out_ids.shape == (rows, gamma + 1) and accept_prob.shape == (rows, gamma)
     for t in (logits_p, logits_q, draft_ids, n_accept, out_ids, accept_prob):
         assert t.is_cuda and t.is_contiguous()
+    assert logits_p.dtype == torch.float32 and logits_q.dtype == torch.float32 and accept_prob.dtype == torch.float32
+    assert draft_ids.dtype == torch.int32 and n_accept.dtype == torch.int32 and out_ids.dtype == torch.int32
     st = stream if stream is not None else torch.cuda.current_stream(logits_p.device)
     _check(lib().sdd_accept_logits_static(logits_p.data_ptr(), logits_q.data_ptr(), draft_ids.data_ptr(), rows, gamma,
                                           V, float(temp_p), float(temp_q), int(seed), int(rnd), n_accept.data_ptr(),
@@ -226,6 +229,14 @@ def sdd_debug_attention_bf16(q, q_col0, k, k_col0, k_rows_per_seq, vt, out, ctx_
                                           out.data_ptr(), out.stride(0), ctx_len.data_ptr(), batch, n_head, gamma, mode,
                                           q_rows_per_seq, status.data_ptr() if status is not None else None,
                                           st.cuda_stream), "sdd_debug_attention_bf16")
+
+
+def sdd_debug_wait_timeout(limit_cycles: int, status, stream=None):
+    """Runs the library's one-CTA probe whose bounded waits run out after `limit_cycles` SM clocks; `status` (int32
+    CUDA tensor holding 0) then holds 1."""
+    torch = _torch()
+    st = stream if stream is not None else torch.cuda.current_stream(status.device)
+    _check(lib().sdd_debug_wait_timeout(int(limit_cycles), status.data_ptr(), st.cuda_stream), "sdd_debug_wait_timeout")
 
 
 _TAP_DTYPES = {TAP_STEP_LOGITS: "f", TAP_Q_LOGITS: "f", TAP_LOGQ: "f", TAP_LOGITS_P: "f", TAP_ACCEPT_PROB: "f"}

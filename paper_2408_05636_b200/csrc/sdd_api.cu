@@ -1,5 +1,6 @@
 // C ABI of the SpecDiff round: argument checking, workspace layout, and the host-side schedule
 // that enqueues the kernels of Algorithm 1 on the caller's stream.  See include/sdd.h.
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -92,7 +93,7 @@ static int parse_model(const sdd_model* m, int want_causal, Net* net) {
 struct Buffers {
   RoundState* rs;
   int *tokens, *ctx_len, *n_emitted, *slot_ids, *reveal_step, *n_accept, *extra_token;
-  float *logq, *accept_prob;
+  float *logq, *lse_q, *accept_prob;   // lse_q: log-sum-exp of every stored q row
   float *step_logits, *q_logits, *logits_p;
   float2* partial_p;
   float* h;                    // residual stream, fp32
@@ -129,6 +130,7 @@ static size_t carve(const Dims& D, const Net& P, const Net& Q, uint8_t* base, Bu
   b.n_accept = (int*)take(Bn * 4);
   b.extra_token = (int*)take(Bn * 4);
   b.logq = (float*)take(Bn * G * 4);
+  b.lse_q = (float*)take(Bn * G * 4);
   b.accept_prob = (float*)take(Bn * G * 4);
   b.step_logits = (float*)take(Bn * G * V * 4);
   b.q_logits = (float*)take(Bn * G * V * 4);
@@ -342,7 +344,7 @@ static int forward_drafter(sdd_ctx* c) {
   const bool prune = c->slot_prune == 1 || (c->slot_prune < 0 && rows >= 2048);
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_drafter<T>((const T*)Q.wte, (const T*)Q.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
                                         D.batch, D.gamma, lcap, Q.d, B.h, c->st, skip, Q.layers[0].ln1_g, Q.layers[0].ln1_b,
-                                        (T*)B.xn));
+                                        (T*)B.xn, Q.vocab, &B.rs->status));
   const bool tc = use_tc<T>(c, Q);
   SDD_TRY((run_blocks<T>(c, Q, rows, CAT_GEMM_Q, false, skip,
     [&](int, QkvDst* qd) -> bool {
@@ -438,7 +440,7 @@ static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) 
   // a verification forward carries the round's own draft length (gamma + 1 rows); slot_ids is [batch][that length]
   const int slot_stride = mode == TARGET_VERIFY ? rows_per_seq - 1 : D.gamma;
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_target<T>((const T*)P.wte, (const T*)P.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
-                                       D.batch, slot_stride, rows_per_seq, mode, P.d, B.h, c->st));
+                                       D.batch, slot_stride, rows_per_seq, mode, P.d, B.h, c->st, P.vocab, &B.rs->status));
   return forward_causal<T>(c, P, B.kv, B.ctx_len, mode, rows_per_seq, lm_head, B.logits_p, c->hilo, CAT_GEMM_P, CAT_HEAD_P,
                            CAT_ATTN_P);
 }
@@ -456,11 +458,11 @@ static int forward_ar_drafter(sdd_ctx* c, int gamma, int j) {
   const Dims& D = c->D;
   const int rows = j == 0 ? 2 : 1, off = j == 0 ? -1 : j;
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_ar<T>((const T*)A.wte, (const T*)A.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
-                                             D.batch, gamma, rows, off, A.d, B.h, c->ar_eff, c->st));
+                                             D.batch, gamma, rows, off, A.d, B.h, c->ar_eff, c->st, A.vocab, &B.rs->status));
   SDD_TRY(forward_causal<T>(c, A, c->ar_kv, c->ar_eff, TARGET_VERIFY, rows, true, B.logits_p, false, CAT_GEMM_Q, CAT_HEAD_Q,
                             CAT_ATTN_Q));
-  SDD_LAUNCH(c, CAT_SAMPLE, launch_ar_sample(B.logits_p, rows, B.slot_ids, B.q_logits, B.logq, B.reveal_step, D.batch, gamma, j,
-                                             D.V, c->inv_tau_q, c->key, B.rs, c->st));
+  SDD_LAUNCH(c, CAT_SAMPLE, launch_ar_sample(B.logits_p, rows, B.slot_ids, B.q_logits, B.logq, B.lse_q, B.reveal_step, D.batch,
+                                             gamma, j, D.V, c->inv_tau_q, c->key, B.rs, c->st));
   return SDD_OK;
 }
 
@@ -468,11 +470,15 @@ static int forward_ar_drafter(sdd_ctx* c, int gamma, int j) {
 // padded row count of this round's drafter forwards
 static void choose_lcap(sdd_ctx* c) {
   const int Bn = c->D.batch;
+  // the commit kernel writes head stamp, body, tail stamp; a reader therefore takes the tail first and the head
+  // last: equal stamps then bracket a body that no writer touched in between
   volatile int* m = c->mirror;
-  const int s0 = m[0];
+  const int s1 = m[1 + 2 * Bn];
+  std::atomic_thread_fence(std::memory_order_acquire);
   std::vector<int> seen(Bn);
   for (int b = 0; b < Bn; ++b) seen[b] = m[1 + b];
-  const int s1 = m[1 + 2 * Bn];
+  std::atomic_thread_fence(std::memory_order_acquire);
+  const int s0 = m[0];
   const int per_round = c->D.gamma + 1;
   if (s0 == s1 && s1 > 0 && (uint64_t)s1 <= c->rounds) {
     const long long behind = (long long)c->rounds - s1;
@@ -498,8 +504,8 @@ static int draft_step_t(sdd_ctx* c) {
   const Dims& D = c->D;
   const int k = D.T - c->steps_done;
   SDD_TRY(forward_drafter<T>(c));
-  SDD_LAUNCH(c, CAT_SAMPLE, launch_unmask_sample(B.step_logits, B.slot_ids, B.q_logits, B.logq, B.reveal_step, D.batch, D.gamma, D.V, k,
-                                     c->inv_tau_q, c->key, B.rs, c->cache_skip ? 1 : 0, c->st));
+  SDD_LAUNCH(c, CAT_SAMPLE, launch_unmask_sample(B.step_logits, B.slot_ids, B.q_logits, B.logq, B.lse_q, B.reveal_step, D.batch,
+                                     D.gamma, D.V, k, c->inv_tau_q, c->key, B.rs, c->cache_skip ? 1 : 0, c->st));
   c->steps_done++;
   return SDD_OK;
 }
@@ -513,7 +519,7 @@ static int verify_accept_t(sdd_ctx* c, int gamma, int32_t* out_ids, int32_t* n_o
   SDD_TRY(forward_target<T>(c, TARGET_VERIFY, gamma + 1, true));
   SDD_LAUNCH(c, CAT_STATS, launch_row_stats(B.logits_p, (long long)D.batch * (gamma + 1), nullptr, 0, D.V, c->inv_tau_p, 0.f,
                                  B.partial_p, c->st));
-  SDD_LAUNCH(c, CAT_ACCEPT, launch_accept(B.logits_p, B.q_logits, B.slot_ids, B.logq, B.partial_p, nullptr, D.batch, gamma, D.V,
+  SDD_LAUNCH(c, CAT_ACCEPT, launch_accept(B.logits_p, B.q_logits, B.slot_ids, B.logq, B.lse_q, B.partial_p, nullptr, D.batch, gamma, D.V,
                               c->inv_tau_p, c->inv_tau_p == 0.f ? 0.f : 1.f, c->key, 0u, B.rs, B.accept_prob, B.n_accept,
                               B.extra_token, nullptr, c->st));
   SDD_LAUNCH(c, CAT_COMMIT, launch_commit(B.tokens, D.tok_stride, B.ctx_len, B.n_emitted, B.slot_ids, B.n_accept, B.extra_token,
@@ -851,13 +857,13 @@ static int prefill_ar_drafter(sdd_ctx* c) {
   if (A.dtype == SDD_BF16) {
     SDD_LAUNCH(c, CAT_GLUE, launch_embed_target<__nv_bfloat16>((const __nv_bfloat16*)A.wte, (const __nv_bfloat16*)A.wpe, B.tokens,
                                                                c->D.tok_stride, B.ctx_len, B.slot_ids, c->D.batch, c->D.gamma,
-                                                               rows, TARGET_PREFILL, A.d, B.h, c->st));
+                                                               rows, TARGET_PREFILL, A.d, B.h, c->st, A.vocab, &B.rs->status));
     s = forward_causal<__nv_bfloat16>(c, A, c->ar_kv, B.ctx_len, TARGET_PREFILL, rows, false, nullptr, false, CAT_GEMM_Q,
                                       CAT_HEAD_Q, CAT_ATTN_Q);
   } else {
     SDD_LAUNCH(c, CAT_GLUE, launch_embed_target<float>((const float*)A.wte, (const float*)A.wpe, B.tokens, c->D.tok_stride,
                                                        B.ctx_len, B.slot_ids, c->D.batch, c->D.gamma, rows, TARGET_PREFILL, A.d,
-                                                       B.h, c->st));
+                                                       B.h, c->st, A.vocab, &B.rs->status));
     s = forward_causal<float>(c, A, c->ar_kv, B.ctx_len, TARGET_PREFILL, rows, false, nullptr, false, CAT_GEMM_Q, CAT_HEAD_Q,
                               CAT_ATTN_Q);
   }
@@ -912,10 +918,13 @@ int32_t sdd_progress(sdd_ctx* c, uint64_t* rounds_done, int32_t* min_emitted) {
   const int Bn = c->D.batch;
   volatile int* m = c->mirror;
   for (int attempt = 0; attempt < 64; ++attempt) {
-    const int s0 = m[0];
+    // tail stamp, body, head stamp: the reverse of the commit kernel's write order (see choose_lcap)
+    const int s1 = m[1 + 2 * Bn];
+    std::atomic_thread_fence(std::memory_order_acquire);
     int mn = 0x7fffffff;
     for (int b = 0; b < Bn; ++b) { const int e = m[1 + Bn + b]; if (e < mn) mn = e; }
-    const int s1 = m[1 + 2 * Bn];
+    std::atomic_thread_fence(std::memory_order_acquire);
+    const int s0 = m[0];
     if (s0 == s1) {
       if (rounds_done) *rounds_done = (uint64_t)s1;
       if (min_emitted) *min_emitted = s1 == 0 ? 0 : mn;
@@ -946,7 +955,7 @@ int32_t sdd_accept_logits(const float* logits_p, const float* logits_q, const in
   const long long rows_p = (long long)rows * (gamma + 1), rows_q = (long long)rows * gamma;
   const int chunks = stats_chunks_for(V);
   SDD_CUDA(launch_row_stats(logits_p, rows_p, logits_q, itp == 0.f ? 0 : rows_q, V, itp, itq, partial, st));
-  SDD_CUDA(launch_accept(logits_p, logits_q, draft_ids, nullptr, partial, partial + rows_p * chunks, rows, gamma, V, itp, itq,
+  SDD_CUDA(launch_accept(logits_p, logits_q, draft_ids, nullptr, nullptr, partial, partial + rows_p * chunks, rows, gamma, V, itp, itq,
                          make_key(seed), (uint32_t)round, nullptr, accept_prob, n_accept, nullptr, out_ids, st));
   return SDD_OK;
 }
@@ -980,6 +989,12 @@ int32_t sdd_debug_attention_bf16(const void* q, int64_t q_rows_total, int32_t q_
   return SDD_OK;
 }
 
+int32_t sdd_debug_wait_timeout(int64_t limit_cycles, int32_t* status_word, void* stream) {
+  if (status_word == nullptr || limit_cycles < 1 || limit_cycles > 2000000000ll) return SDD_E_ARG;
+  SDD_CUDA(launch_wait_timeout_probe((long long)limit_cycles, status_word, (cudaStream_t)stream));
+  return SDD_OK;
+}
+
 int32_t sdd_tap(sdd_ctx* c, int32_t what, const void** dev_ptr, uint64_t* bytes) {
   if (c == nullptr || dev_ptr == nullptr || bytes == nullptr) return SDD_E_ARG;
   const Buffers& B = c->B;
@@ -998,6 +1013,7 @@ int32_t sdd_tap(sdd_ctx* c, int32_t what, const void** dev_ptr, uint64_t* bytes)
     case SDD_TAP_EXTRA_TOKEN: *dev_ptr = B.extra_token; *bytes = Bn * 4; break;
     case SDD_TAP_N_EMITTED: *dev_ptr = B.n_emitted; *bytes = Bn * 4; break;
     case SDD_TAP_STATUS: *dev_ptr = &B.rs->status; *bytes = 4; break;
+    case SDD_TAP_EVALS: *dev_ptr = &B.rs->evals_run; *bytes = 8; break;
     default: return SDD_E_ARG;
   }
   return SDD_OK;
@@ -1016,7 +1032,8 @@ int32_t sdd_sync_status(sdd_ctx* c) {
   int status = 0;
   SDD_CUDA(cudaMemcpy(&status, &c->B.rs->status, 4, cudaMemcpyDeviceToHost));
   if (status == DEV_OK) return SDD_OK;
-  return status == DEV_TIMEOUT ? SDD_E_TIMEOUT : SDD_E_CTX_FULL;
+  if (status == DEV_TIMEOUT) return SDD_E_TIMEOUT;
+  return status == DEV_BAD_TOKEN ? SDD_E_INDEX : SDD_E_CTX_FULL;
 }
 
 int32_t sdd_profile_begin(sdd_ctx* c) {
@@ -1085,6 +1102,7 @@ const char* sdd_strerror(int32_t s) {
     case SDD_E_TIMEOUT: return "bounded device-side wait expired";
     case SDD_E_UNIMPL: return "not implemented";
     case SDD_E_STATE: return "call order violated";
+    case SDD_E_INDEX: return "a token id or position outside its table was met on the device";
     default: return "unknown status";
   }
 }

@@ -198,6 +198,7 @@ __device__ __forceinline__ float gelu_tanh_fast(float x) {
 }
 
 // device status word values (first error wins)
-enum : int { DEV_OK = 0, DEV_TIMEOUT = 1, DEV_BAD_INDEX = 2 };
+enum : int { DEV_OK = 0, DEV_TIMEOUT = 1, DEV_BAD_INDEX = 2 /* a commit past the token buffer */,
+             DEV_BAD_TOKEN = 3 /* a token id outside the vocabulary */ };
 
 }  // namespace sdd

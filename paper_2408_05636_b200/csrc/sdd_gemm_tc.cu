@@ -894,6 +894,52 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 }
 
 // ---------------------------------------------------------------------------------------------
+// The error path of the kernels above, run on purpose: one CTA with their role layout in which nothing ever fills
+// the first ring stage.  The MMA role's bounded wait on full[0] runs out after `limit` clocks; it raises the abort
+// flag and the status word; the epilogue warps, which wait for the accumulator, see the flag and leave; the producer
+// finds the flag, has no copy in flight to wait for, and leaves; TMEM is freed; the CTA returns.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(THREADS) wait_timeout_probe_kernel(long long limit, int* status) {
+  __shared__ __align__(8) unsigned long long bars[3];   // full[0], empty[0], tmem_full
+  __shared__ uint32_t tmem_slot_s;
+  __shared__ int abort_s;
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[1]), tmem_full = smem_u32(&bars[2]);
+  volatile int* abort_flag = &abort_s;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    mbar_init(full0, 1); mbar_init(empty0, 1); mbar_init(tmem_full, 1);
+    abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(&tmem_slot_s, 32);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = tmem_slot_s;
+  pdl_wait();
+  pdl_launch_dependents();
+  if (warp == 0) {
+    // the producer, at the point where it wants to refill a stage: it waits for the MMA that would free it, which
+    // never comes; it leaves on the abort flag or on its own limit, with no copy in flight
+    if (lane == 0) mbar_wait(empty0, 0u, abort_flag, status, limit);
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const bool ok = mbar_wait(full0, 0u, abort_flag, status, limit);   // nothing arrives: runs out
+      if (ok) umma_commit(tmem_full);
+    }
+  } else {
+    const bool ready = named_bar_and(1, 128, mbar_wait(tmem_full, 0u, abort_flag, status, limit));
+    (void)ready;                                                         // never true here: no accumulator to drain
+  }
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    fence_after_sync();
+    tmem_dealloc(tmem_base, 32);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side: tensor maps (cached per pointer / shape / box) and launch
 // ---------------------------------------------------------------------------------------------
 template <int BN, bool SWAP, bool HILO, bool DEEP>
@@ -1022,6 +1068,11 @@ cudaError_t get_tensor_map(const void* ptr, long long rows, long long cols, long
   g_maps[key] = m;
   *out = m;
   return cudaSuccess;
+}
+
+cudaError_t launch_wait_timeout_probe(long long limit_cycles, int* status, cudaStream_t st) {
+  launch_k(tc::wait_timeout_probe_kernel, dim3(1), dim3(tc::THREADS), 0, st, limit_cycles, status);
+  return cudaGetLastError();
 }
 
 // A: activations [M rows used, capacity a_cap rows, K], W: weights [N, K]; both dense bf16.

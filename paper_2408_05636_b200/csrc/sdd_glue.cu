@@ -50,7 +50,8 @@ __global__ void __launch_bounds__(EMB_THREADS)
 embed_drafter_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
                      int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
                      int gamma, int L_cap, int d, float* __restrict__ h, const int* __restrict__ skip,
-                     const float* __restrict__ ln_g, const float* __restrict__ ln_b, T* __restrict__ xn) {
+                     const float* __restrict__ ln_g, const float* __restrict__ ln_b, T* __restrict__ xn, int vocab,
+                     int* __restrict__ status) {
   pdl_wait();
   pdl_launch_dependents();
   if (skip != nullptr && *skip) return;
@@ -59,11 +60,19 @@ embed_drafter_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const
   const long long row = (long long)b * L_cap + i;
   float* __restrict__ dst = h + row * d;
   float x[EMB_MAX_PER_THREAD];
-  if (i >= c + gamma) {                      // padding row: zeros (its LayerNorm is the LayerNorm bias)
+  // ids come from the caller's prompt: one outside [0, vocab] (vocab = [MASK]) must not index the table
+  int tok = 0;
+  if (i < c + gamma) {
+    tok = i < c ? tokens[(long long)b * tok_stride + i] : slot_ids[(long long)b * gamma + (i - c)];
+    if ((unsigned)tok > (unsigned)vocab) {
+      if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, DEV_OK, DEV_BAD_TOKEN);
+      tok = -1;
+    }
+  }
+  if (i >= c + gamma || tok < 0) {           // padding row (or a bad id): zeros (its LayerNorm is the LayerNorm bias)
 #pragma unroll
     for (int k = 0; k < EMB_MAX_PER_THREAD; ++k) x[k] = 0.f;
   } else {
-    const int tok = i < c ? tokens[(long long)b * tok_stride + i] : slot_ids[(long long)b * gamma + (i - c)];
     const T* __restrict__ te = wte + (long long)tok * d;
     const T* __restrict__ pe = wpe + (long long)i * d;
 #pragma unroll
@@ -85,21 +94,28 @@ embed_drafter_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const
 template <typename T>
 __global__ void embed_target_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
                                     int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
-                                    int gamma, int rows_per_seq, int mode, int d, float* __restrict__ h) {
+                                    int gamma, int rows_per_seq, int mode, int d, float* __restrict__ h, int vocab,
+                                    int* __restrict__ status) {
   pdl_wait();
   pdl_launch_dependents();
   const int j = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
   float* __restrict__ dst = h + ((long long)b * rows_per_seq + j) * d;
   int tok, pos;
+  bool pad = false;
   if (mode == TARGET_VERIFY) {
     pos = c - 1 + j;
     tok = j == 0 ? tokens[(long long)b * tok_stride + c - 1] : slot_ids[(long long)b * gamma + j - 1];
   } else {
     pos = j;
-    tok = j < c - 1 ? tokens[(long long)b * tok_stride + j] : -1;
+    pad = j >= c - 1;
+    tok = pad ? 0 : tokens[(long long)b * tok_stride + j];
   }
-  if (tok < 0) {
+  if (!pad && (unsigned)tok >= (unsigned)vocab) {   // a caller's id outside the table: zero row, reported through the status word
+    if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, DEV_OK, DEV_BAD_TOKEN);
+    pad = true;
+  }
+  if (pad) {
     for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = 0.f;
     return;
   }
@@ -116,7 +132,7 @@ template <typename T>
 __global__ void embed_ar_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const int* __restrict__ tokens,
                                 int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
                                 int gamma, int rows_per_seq, int off, int d, float* __restrict__ h,
-                                int* __restrict__ eff_len) {
+                                int* __restrict__ eff_len, int vocab, int* __restrict__ status) {
   pdl_wait();
   pdl_launch_dependents();
   const int i = blockIdx.x, b = blockIdx.y;
@@ -129,6 +145,11 @@ __global__ void embed_ar_kernel(const T* __restrict__ wte, const T* __restrict__
     return;
   }
   const int tok = pos < c ? tokens[(long long)b * tok_stride + pos] : slot_ids[(long long)b * gamma + pos - c];
+  if ((unsigned)tok >= (unsigned)vocab) {    // an id outside the table: zero row, reported through the status word
+    if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, DEV_OK, DEV_BAD_TOKEN);
+    for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = 0.f;
+    return;
+  }
   const T* __restrict__ te = wte + (long long)tok * d;
   const T* __restrict__ pe = wpe + (long long)pos * d;
   for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = to_f32(te[e]) + to_f32(pe[e]);
@@ -312,27 +333,27 @@ __global__ void kv_append_kernel(const T* __restrict__ qkv, T* __restrict__ cach
 template <typename T>
 cudaError_t launch_embed_drafter(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                  const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st,
-                                 const int* skip, const float* ln_g, const float* ln_b, T* xn) {
+                                 const int* skip, const float* ln_g, const float* ln_b, T* xn, int vocab, int* status) {
   if (d > EMB_THREADS * EMB_MAX_PER_THREAD) return cudaErrorInvalidValue;
   launch_k(embed_drafter_kernel<T>, dim3(L_cap, batch), dim3(EMB_THREADS), 0, st, wte, wpe, tokens, tok_stride, ctx_len, slot_ids,
-           gamma, L_cap, d, h, skip, ln_g, ln_b, xn);
+           gamma, L_cap, d, h, skip, ln_g, ln_b, xn, vocab, status);
   return cudaGetLastError();
 }
 template <typename T>
 cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                 const int* slot_ids, int batch, int gamma, int rows_per_seq, int mode, int d, float* h,
-                                cudaStream_t st) {
+                                cudaStream_t st, int vocab, int* status) {
   if (rows_per_seq <= 0) return cudaSuccess;
   launch_k(embed_target_kernel<T>, dim3(dim3(rows_per_seq, batch)), dim3(128), 0, st, wte, wpe, tokens, tok_stride, ctx_len, slot_ids, gamma,
-                                                                    rows_per_seq, mode, d, h);
+                                                                    rows_per_seq, mode, d, h, vocab, status);
   return cudaGetLastError();
 }
 template <typename T>
 cudaError_t launch_embed_ar(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                             const int* slot_ids, int batch, int gamma, int rows_per_seq, int off, int d, float* h,
-                            int* eff_len, cudaStream_t st) {
+                            int* eff_len, cudaStream_t st, int vocab, int* status) {
   launch_k(embed_ar_kernel<T>, dim3(rows_per_seq, batch), dim3(128), 0, st, wte, wpe, tokens, tok_stride, ctx_len, slot_ids,
-           gamma, rows_per_seq, off, d, h, eff_len);
+           gamma, rows_per_seq, off, d, h, eff_len, vocab, status);
   return cudaGetLastError();
 }
 template <typename T>
@@ -375,11 +396,11 @@ cudaError_t launch_kv_append(const T* qkv, T* cache, const int* ctx_len, int bat
 #define SDD_INSTANTIATE_GLUE(T)                                                                                          \
   template cudaError_t launch_embed_drafter<T>(const T*, const T*, const int*, int, const int*, const int*, int, int,   \
                                                int, int, float*, cudaStream_t, const int*, const float*, const float*,  \
-                                               T*);                                                                     \
+                                               T*, int, int*);                                                          \
   template cudaError_t launch_embed_target<T>(const T*, const T*, const int*, int, const int*, const int*, int, int,    \
-                                              int, int, int, float*, cudaStream_t);                                     \
+                                              int, int, int, float*, cudaStream_t, int, int*);                          \
   template cudaError_t launch_embed_ar<T>(const T*, const T*, const int*, int, const int*, const int*, int, int, int,   \
-                                          int, int, float*, int*, cudaStream_t);                                        \
+                                          int, int, float*, int*, cudaStream_t, int, int*);                             \
   template cudaError_t launch_layernorm<T>(const float*, const float*, const float*, T*, long long, int, cudaStream_t, \
                                            T*, const int*);                                                                         \
   template cudaError_t launch_layernorm_slots<T>(const float*, const float*, const float*, T*, const int*, int, int,    \

@@ -13,7 +13,9 @@ struct RoundState {
   uint32_t ticket;     // CTAs of that step's sampling kernel that have finished
   int skip_forward;    // 1: the last step revealed nothing, so the next drafter evaluation would reproduce the
                        //    logits it already has ("cache" strategy): its kernels return at once
-  int pad[3];
+  int evals_run;       // drafter evaluations of this generation that ran ...
+  int evals_skipped;   // ... and that were skipped on skip_forward (counted by the sampling kernel's last CTA)
+  int pad[1];
 };
 
 // How a target forward maps its rows to sequence positions.
@@ -47,18 +49,20 @@ struct QkvDst {
 int stats_chunks_for(int V);
 cudaError_t launch_row_stats(const float* a, long long rows_a, const float* b, long long rows_b, int V, float inv_tau_a,
                              float inv_tau_b, float2* partial, cudaStream_t st);
-cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float* q_logits, float* logq, int* reveal_step,
-                                 int batch, int gamma, int V, int k, float inv_tau_q, PhiloxKey key,
+// lseq [batch, gamma] receives the log-sum-exp of every stored q row (the acceptance step's residual draw reads it)
+cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float* q_logits, float* logq, float* lseq,
+                                 int* reveal_step, int batch, int gamma, int V, int k, float inv_tau_q, PhiloxKey key,
                                  RoundState* rs, int cache_skip, cudaStream_t st);
+// round pipeline: logq_in / lseq_in from the draws, partial_q null; stand-alone: logq_in / lseq_in null, partial_q given
 cudaError_t launch_accept(const float* logits_p, const float* q_rows, const int* draft_ids, const float* logq_in,
-                          const float2* partial_p, const float2* partial_q, int rows, int gamma, int V, float inv_tau_p,
-                          float inv_tau_q_rows, PhiloxKey key, uint32_t rnd, const RoundState* rs, float* accept_prob,
+                          const float* lseq_in, const float2* partial_p, const float2* partial_q, int rows, int gamma, int V,
+                          float inv_tau_p, float inv_tau_q_rows, PhiloxKey key, uint32_t rnd, RoundState* rs, float* accept_prob,
                           int* n_accept, int* extra_token, int* out_ids, cudaStream_t st);
 cudaError_t launch_commit(int* tokens, int tok_stride, int* ctx_len, int* n_emitted, const int* slot_ids,
                           const int* n_accept, const int* extra_token, int batch, int gamma, int max_new, RoundState* rs,
                           int* out_ids, int* n_out, volatile int* host_mirror, cudaStream_t st);
 // draw of slot j from the last of the rows_per_seq logit rows per sequence (autoregressive drafter)
-cudaError_t launch_ar_sample(const float* logits, int rows_per_seq, int* slot_ids, float* q_logits, float* logq,
+cudaError_t launch_ar_sample(const float* logits, int rows_per_seq, int* slot_ids, float* q_logits, float* logq, float* lseq,
                              int* reveal_step, int batch, int gamma, int j, int V, float inv_tau_q, PhiloxKey key,
                              const RoundState* rs, cudaStream_t st);
 cudaError_t launch_reset_slots(int* slot_ids, int* reveal_step, int n, int mask_id, RoundState* rs, cudaStream_t st);
@@ -68,16 +72,19 @@ template <typename T>
 cudaError_t launch_embed_drafter(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                  const int* slot_ids, int batch, int gamma, int L_cap, int d, float* h, cudaStream_t st,
                                  const int* skip = nullptr, const float* ln_g = nullptr, const float* ln_b = nullptr,
-                                 T* xn = nullptr);   // xn != null: also xn = LayerNorm(h; ln_g, ln_b), the first block's
+                                 T* xn = nullptr,    // xn != null: also xn = LayerNorm(h; ln_g, ln_b), the first block's
+                                 int vocab = 0x7fffffff, int* status = nullptr);
+// Token ids index the embedding tables, so every embedding kernel checks them: an id outside [0, vocab) (the drafter
+// also takes vocab, its [MASK] row) gives a zero embedding row and raises DEV_BAD_TOKEN in *status (if non-null).
 template <typename T>
 cudaError_t launch_embed_target(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                                 const int* slot_ids, int batch, int gamma, int rows_per_seq, int mode, int d, float* h,
-                                cudaStream_t st);
+                                cudaStream_t st, int vocab = 0x7fffffff, int* status = nullptr);
 // rows of an autoregressive drafter's evaluation: positions ctx_len[b] + off - 1 + i; writes eff_len[b] = ctx_len[b] + off
 template <typename T>
 cudaError_t launch_embed_ar(const T* wte, const T* wpe, const int* tokens, int tok_stride, const int* ctx_len,
                             const int* slot_ids, int batch, int gamma, int rows_per_seq, int off, int d, float* h,
-                            int* eff_len, cudaStream_t st);
+                            int* eff_len, cudaStream_t st, int vocab = 0x7fffffff, int* status = nullptr);
 // LayerNorm of `rows` rows of h (fp32, row stride d) into out (activation type); out_lo (optional) receives the
 // rounding remainder y - out so that (out, out_lo) carries y to about 16 significant bits
 template <typename T>
@@ -110,6 +117,9 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
                            int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st,
                            const QkvDst* qkv = nullptr, const __nv_bfloat16* A_lo = nullptr, void* out_lo = nullptr,
                            const int* skip = nullptr);
+
+// one CTA whose bounded waits run out after limit_cycles (see sdd_debug_wait_timeout)
+cudaError_t launch_wait_timeout_probe(long long limit_cycles, int* status, cudaStream_t st);
 
 // one-time set-up of the tensor-core kernels (dynamic shared-memory limits); also done lazily on first launch
 cudaError_t tc_prepare_gemm();

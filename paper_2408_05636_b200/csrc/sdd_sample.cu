@@ -250,10 +250,12 @@ constexpr int SAMPLE_THREADS = 512;
 
 // returns true in every CTA of a cluster whose slot was revealed by this step
 // Gumbel-max draw of one slot by the cluster that owns it: x = argmax_v (z_v + G_v), z = src * inv_tau_q (arg-max of
-// src when greedy); the row z is stored to dst and log q(x) = z_x - logsumexp(z) to *logq_out.  `mark` goes to
+// src when greedy); the row z is stored to dst, log q(x) = z_x - logsumexp(z) to *logq_out and logsumexp(z) to
+// *lseq_out.  `mark` goes to
 // *reveal_out (the denoising step, or the evaluation index of an autoregressive drafter).
 __device__ __forceinline__ void draw_slot(const float* __restrict__ src, float* __restrict__ dst, int* __restrict__ slot_out,
-                                          float* __restrict__ logq_out, int* __restrict__ reveal_out, int j, int b, int V,
+                                          float* __restrict__ logq_out, float* __restrict__ lseq_out,
+                                          int* __restrict__ reveal_out, int j, int b, int V,
                                           int mark, float inv_tau_q, PhiloxKey key, uint32_t rnd) {
   cg::cluster_group cl = cg::this_cluster();
   const int rank = (int)cl.block_rank();
@@ -301,6 +303,7 @@ __device__ __forceinline__ void draw_slot(const float* __restrict__ src, float* 
     const float lse = greedy ? 0.f : cluster_merge_lse(cl, &part);
     *slot_out = win.i;
     *logq_out = greedy ? 0.f : src[win.i] * inv_tau_q - lse;
+    *lseq_out = lse;               // the stored row's log-sum-exp: the residual draw of the acceptance step needs it
     *reveal_out = mark;
   }
   cl.sync();   // partials stay alive until rank 0 has read them
@@ -310,6 +313,7 @@ __device__ __forceinline__ bool unmask_sample_row(const float* __restrict__ step
                      int* __restrict__ slot_ids,             // [B, gamma]  (V = masked)
                      float* __restrict__ q_logits,           // [B, gamma, V]
                      float* __restrict__ logq,               // [B, gamma]
+                     float* __restrict__ lseq,               // [B, gamma]
                      int* __restrict__ reveal_step,          // [B, gamma]
                      int gamma, int V, int k, float inv_tau_q, PhiloxKey key, const RoundState* __restrict__ rs) {
   const int j = blockIdx.x / VC, b = blockIdx.y;
@@ -321,8 +325,8 @@ __device__ __forceinline__ bool unmask_sample_row(const float* __restrict__ step
   const uint32_t wu = philox4x32_10(0u, (uint32_t)j, rnd, rng_c3(RNG_UNMASK, (uint32_t)k, (uint32_t)b), key).x;
   const uint32_t m_odd = ((wu >> 9) << 1) | 1u;
   if (!(m_odd * (uint32_t)k < (1u << 24))) return false;
-  draw_slot(step_logits + row * V, q_logits + row * V, slot_ids + row, logq + row, reveal_step + row, j, b, V, k, inv_tau_q,
-            key, rnd);
+  draw_slot(step_logits + row * V, q_logits + row * V, slot_ids + row, logq + row, lseq + row, reveal_step + row, j, b, V, k,
+            inv_tau_q, key, rnd);
   return true;
 }
 
@@ -332,11 +336,11 @@ __device__ __forceinline__ bool unmask_sample_row(const float* __restrict__ step
 // at once (the paper's "ddpm cache" strategy: a step without change costs no network evaluation).
 __global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(SAMPLE_THREADS)
 unmask_sample_kernel(const float* __restrict__ step_logits, int* __restrict__ slot_ids, float* __restrict__ q_logits,
-                     float* __restrict__ logq, int* __restrict__ reveal_step, int gamma, int V, int k, float inv_tau_q,
-                     PhiloxKey key, RoundState* __restrict__ rs, int cache_skip) {
+                     float* __restrict__ logq, float* __restrict__ lseq, int* __restrict__ reveal_step, int gamma, int V, int k,
+                     float inv_tau_q, PhiloxKey key, RoundState* __restrict__ rs, int cache_skip) {
   pdl_wait();
   pdl_launch_dependents();
-  const bool revealed = unmask_sample_row(step_logits, slot_ids, q_logits, logq, reveal_step, gamma, V, k, inv_tau_q, key, rs);
+  const bool revealed = unmask_sample_row(step_logits, slot_ids, q_logits, logq, lseq, reveal_step, gamma, V, k, inv_tau_q, key, rs);
   if (threadIdx.x == 0) {
     if (revealed && (blockIdx.x % VC) == 0) atomicAdd(&rs->revealed, 1u);
     __threadfence();
@@ -344,6 +348,8 @@ unmask_sample_kernel(const float* __restrict__ step_logits, int* __restrict__ sl
     if (t == gridDim.x * gridDim.y - 1) {
       __threadfence();
       const uint32_t n = atomicExch(&rs->revealed, 0u);
+      // the flag as it stood during this step tells whether the step's drafter evaluation ran
+      if (rs->skip_forward) rs->evals_skipped += 1; else rs->evals_run += 1;
       rs->skip_forward = (cache_skip && n == 0u) ? 1 : 0;
       rs->ticket = 0u;
     }
@@ -354,30 +360,32 @@ unmask_sample_kernel(const float* __restrict__ step_logits, int* __restrict__ sl
 // `rows_per_seq` rows the evaluation produced for each sequence; the slot is always written.  grid = (VC, batch).
 __global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(SAMPLE_THREADS)
 ar_sample_kernel(const float* __restrict__ logits, int rows_per_seq, int* __restrict__ slot_ids, float* __restrict__ q_logits,
-                 float* __restrict__ logq, int* __restrict__ reveal_step, int gamma, int j, int V, float inv_tau_q,
-                 PhiloxKey key, const RoundState* __restrict__ rs) {
+                 float* __restrict__ logq, float* __restrict__ lseq, int* __restrict__ reveal_step, int gamma, int j, int V,
+                 float inv_tau_q, PhiloxKey key, const RoundState* __restrict__ rs) {
   pdl_wait();
   pdl_launch_dependents();
   const int b = blockIdx.y;
   const long long row = (long long)b * gamma + j;
   draw_slot(logits + ((long long)b * rows_per_seq + rows_per_seq - 1) * V, q_logits + row * V, slot_ids + row, logq + row,
-            reveal_step + row, j, b, V, gamma - j, inv_tau_q, key, rs->round);
+            lseq + row, reveal_step + row, j, b, V, gamma - j, inv_tau_q, key, rs->round);
 }
 
 // ---------------------------------------------------------------------------------------------
 // acceptance scan + extra token                                  grid = (VC * rows), cluster VC per row
 //
 // logits_p [rows, gamma+1, V]; q rows [rows, gamma, V] hold z_q = l * inv_tau_q_rows (inv_tau_q_rows
-// = 1 when the rows were stored already divided by the temperature).  log q(x) comes either from
-// `logq_in` (round pipeline) or from the q-row partial statistics (stand-alone call).
+// = 1 when the rows were stored already divided by the temperature).  log q(x) and the q rows' log-sum-exp come
+// either from `logq_in` / `lseq_in` (round pipeline: stored by the draw) or from the q-row partial statistics
+// (stand-alone call).  A draft id outside [0, V) is never used as an index: its row counts as rejected, the
+// sequence's n_accept becomes -1 (out_ids all -1) and, in the round pipeline, the status word DEV_BAD_TOKEN.
 // ---------------------------------------------------------------------------------------------
 constexpr int ACCEPT_THREADS = 256;
 
 __global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(ACCEPT_THREADS)
 accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_rows, const int* __restrict__ draft_ids,
-              const float* __restrict__ logq_in, const float2* __restrict__ partial_p,
+              const float* __restrict__ logq_in, const float* __restrict__ lseq_in, const float2* __restrict__ partial_p,
               const float2* __restrict__ partial_q, int chunks, int gamma, int V, float inv_tau_p,
-              float inv_tau_q_rows, PhiloxKey key, uint32_t rnd_arg, const RoundState* __restrict__ rs,
+              float inv_tau_q_rows, PhiloxKey key, uint32_t rnd_arg, RoundState* __restrict__ rs,
               float* __restrict__ accept_prob, int* __restrict__ n_accept, int* __restrict__ extra_token,
               int* __restrict__ out_ids) {
   pdl_wait();
@@ -390,14 +398,13 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
   extern __shared__ float s_dyn[];           // [gamma+1] lse_p (or arg-max bits), [gamma] lse_q
   float* s_lsep = s_dyn;
   float* s_lseq = s_dyn + gamma + 1;
-  __shared__ int s_n;
+  __shared__ int s_n, s_bad;
   __shared__ int s_rej[ACCEPT_THREADS / 32];
   __shared__ float s_val[ACCEPT_THREADS / 32];
   __shared__ int s_idx[ACCEPT_THREADS / 32];
-  __shared__ float s_m2[ACCEPT_THREADS / 32], s_s2[ACCEPT_THREADS / 32];
-  __shared__ float s_lse2;
   __shared__ RowPartial part;
 
+  if (threadIdx.x == 0) s_bad = 0;
   const float2* pp = partial_p + (long long)b * (gamma + 1) * chunks;
   for (int j = threadIdx.x; j <= gamma; j += ACCEPT_THREADS) {
     if (greedy) s_lsep[j] = __int_as_float(merge_partials_argmax(pp + (long long)j * chunks, chunks));
@@ -415,7 +422,10 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
     const int j = threadIdx.x;
     const int x = draft_ids[(long long)b * gamma + j];
     float ratio;
-    if (greedy) {
+    if ((unsigned)x >= (unsigned)V) {
+      ratio = 0.f;
+      s_bad = 1;
+    } else if (greedy) {
       ratio = (x == __float_as_int(s_lsep[j])) ? 1.f : 0.f;
     } else {
       const float logp = logits_p[((long long)b * (gamma + 1) + j) * V + x] * inv_tau_p - s_lsep[j];
@@ -451,21 +461,8 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
     const float lsep = s_lsep[n];
     float lseq = 0.f;
     if (resid) {
-      if (partial_q != nullptr) lseq = s_lseq[n];
-      else {
-        // round pipeline: q row statistics are not kept; the cluster recomputes the row's log-sum-exp
-        MaxSum ms;
-        ms.m = -INFINITY;
-        ms.s = 0.f;
-        for (int v = rank * ACCEPT_THREADS + threadIdx.x; v < V; v += VC * ACCEPT_THREADS)
-          maxsum_push(ms, qrow[v] * inv_tau_q_rows);
-        ms = block_maxsum<ACCEPT_THREADS>(ms, s_m2, s_s2);
-        if (threadIdx.x == 0) { part.m = ms.m; part.s = ms.s; }
-        cl.sync();
-        if (threadIdx.x == 0) s_lse2 = cluster_merge_lse(cl, &part);
-        __syncthreads();
-        lseq = s_lse2;
-      }
+      // stand-alone call: from the q rows' chunk statistics; round pipeline: stored by the draw of slot n
+      lseq = partial_q != nullptr ? s_lseq[n] : lseq_in[(long long)b * gamma + n];
     }
     const uint32_t c3 = rng_c3(resid ? RNG_RESID : RNG_BONUS, 0u, (uint32_t)b);
     const int nblk = (V + 3) >> 2;
@@ -531,11 +528,13 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
       if (win.i == 0x7fffffff) win = cluster_merge_argmax(cl, &part, true);
       t = win.i;
     }
-    n_accept[b] = n;
+    const bool bad = s_bad != 0;
+    if (bad && rs != nullptr) atomicCAS(&rs->status, DEV_OK, DEV_BAD_TOKEN);
+    n_accept[b] = bad ? -1 : n;
     if (extra_token != nullptr) extra_token[b] = t;
     if (out_ids != nullptr) {
       for (int j = 0; j <= gamma; ++j)
-        out_ids[(long long)b * (gamma + 1) + j] = j < n ? draft_ids[(long long)b * gamma + j] : (j == n ? t : -1);
+        out_ids[(long long)b * (gamma + 1) + j] = bad ? -1 : (j < n ? draft_ids[(long long)b * gamma + j] : (j == n ? t : -1));
     }
   }
   cl.sync();   // partials stay alive until rank 0 has read them
@@ -625,29 +624,29 @@ cudaError_t launch_row_stats(const float* a, long long rows_a, const float* b, l
   return cudaGetLastError();
 }
 
-cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float* q_logits, float* logq, int* reveal_step,
-                                 int batch, int gamma, int V, int k, float inv_tau_q, PhiloxKey key,
+cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float* q_logits, float* logq, float* lseq,
+                                 int* reveal_step, int batch, int gamma, int V, int k, float inv_tau_q, PhiloxKey key,
                                  RoundState* rs, int cache_skip, cudaStream_t st) {
   dim3 grid(VC * gamma, batch);
-  launch_k(unmask_sample_kernel, dim3(grid), dim3(SAMPLE_THREADS), 0, st, step_logits, slot_ids, q_logits, logq, reveal_step, gamma, V, k,
-                                                       inv_tau_q, key, rs, cache_skip);
+  launch_k(unmask_sample_kernel, dim3(grid), dim3(SAMPLE_THREADS), 0, st, step_logits, slot_ids, q_logits, logq, lseq, reveal_step, gamma,
+           V, k, inv_tau_q, key, rs, cache_skip);
   return cudaGetLastError();
 }
 
-cudaError_t launch_ar_sample(const float* logits, int rows_per_seq, int* slot_ids, float* q_logits, float* logq,
+cudaError_t launch_ar_sample(const float* logits, int rows_per_seq, int* slot_ids, float* q_logits, float* logq, float* lseq,
                              int* reveal_step, int batch, int gamma, int j, int V, float inv_tau_q, PhiloxKey key,
                              const RoundState* rs, cudaStream_t st) {
-  launch_k(ar_sample_kernel, dim3(VC, batch), dim3(SAMPLE_THREADS), 0, st, logits, rows_per_seq, slot_ids, q_logits, logq,
+  launch_k(ar_sample_kernel, dim3(VC, batch), dim3(SAMPLE_THREADS), 0, st, logits, rows_per_seq, slot_ids, q_logits, logq, lseq,
            reveal_step, gamma, j, V, inv_tau_q, key, rs);
   return cudaGetLastError();
 }
 
 cudaError_t launch_accept(const float* logits_p, const float* q_rows, const int* draft_ids, const float* logq_in,
-                          const float2* partial_p, const float2* partial_q, int rows, int gamma, int V, float inv_tau_p,
-                          float inv_tau_q_rows, PhiloxKey key, uint32_t rnd, const RoundState* rs, float* accept_prob,
+                          const float* lseq_in, const float2* partial_p, const float2* partial_q, int rows, int gamma, int V,
+                          float inv_tau_p, float inv_tau_q_rows, PhiloxKey key, uint32_t rnd, RoundState* rs, float* accept_prob,
                           int* n_accept, int* extra_token, int* out_ids, cudaStream_t st) {
   const size_t smem = (size_t)(2 * gamma + 1) * sizeof(float);
-  launch_k(accept_kernel, dim3(VC * rows), dim3(ACCEPT_THREADS), smem, st, logits_p, q_rows, draft_ids, logq_in, partial_p, partial_q,
+  launch_k(accept_kernel, dim3(VC * rows), dim3(ACCEPT_THREADS), smem, st, logits_p, q_rows, draft_ids, logq_in, lseq_in, partial_p, partial_q,
                                                     stats_chunks(V), gamma, V, inv_tau_p, inv_tau_q_rows, key, rnd, rs,
                                                     accept_prob, n_accept, extra_token, out_ids);
   return cudaGetLastError();

@@ -5,7 +5,8 @@
     python -m paper_2408_05636_b200.microbench accept --rows 64 --gamma 32 [--vocab 50257]
 
 Each prints one JSON line with the time per launch and the achieved rate.  `--iters` launches are timed
-after `--warmup`; inputs are seeded random tensors created on the device.
+after `--warmup`; inputs are seeded random tensors created on the device (bench.py times the acceptance step on the
+host-generated cases of synth.accept_case instead, see accept_case_timed).
 """
 from __future__ import annotations
 
@@ -78,6 +79,35 @@ def accept(rows, gamma, vocab=50257, sigma=0.5, iters=20, warmup=3, seed=31):
 
     def call():
         res["n"] = sdd.sdd_accept_logits(lp, lq, ids, 1.0, 1.0, seed, 7, scratch, st)[0]
+
+    ms = time_launches(call, iters, warmup, st)
+    nbytes = rows * (2 * gamma + 1) * vocab * 4.0
+    return {"kernel": "accept", "rows": rows, "gamma": gamma, "vocab": vocab, "us": ms * 1e3,
+            "gbs": nbytes / (ms * 1e-3) / 1e9, "bytes": nbytes, "mean_accepted": float(res["n"].float().mean().item())}
+
+
+def accept_case_timed(base, gamma, iters=20, warmup=3, seed=31, rnd=7):
+    """Times sdd_accept_logits on a seeded case of the input generator (synth.AcceptCase: host arrays), re-indexed to
+    draft length `gamma` with the generator's own row index (synth.accept_row_index), so that the timed inputs are
+    exactly the ones the parity tests replay through the oracle."""
+    import synth
+    rows, g0 = base.draft_ids.shape
+    vocab = base.logits_p.shape[2]
+    p_idx, q_idx = synth.accept_row_index(g0, gamma)
+    lp0 = torch.from_numpy(base.logits_p).cuda()
+    lq0 = torch.from_numpy(base.logits_q).cuda()
+    ids0 = torch.from_numpy(base.draft_ids).cuda()
+    lp = lp0[:, torch.from_numpy(p_idx).cuda()].contiguous()
+    del lp0
+    lq = lq0[:, torch.from_numpy(q_idx).cuda()].contiguous()
+    del lq0
+    ids = ids0[:, torch.from_numpy(q_idx).cuda()].contiguous()
+    scratch = torch.empty(sdd.sdd_accept_scratch_bytes(rows, gamma, vocab), dtype=torch.uint8, device="cuda")
+    st = torch.cuda.Stream()
+    res = {}
+
+    def call():
+        res["n"] = sdd.sdd_accept_logits(lp, lq, ids, 1.0, 1.0, seed, rnd, scratch, st)[0]
 
     ms = time_launches(call, iters, warmup, st)
     nbytes = rows * (2 * gamma + 1) * vocab * 4.0

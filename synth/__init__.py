@@ -78,6 +78,8 @@ def _wl(name, dtype, V, tl, td, th, ql, qd, qh, n_ctx, prompt, gamma, T, batch, 
 WORKLOADS: Dict[str, Workload] = {
     # tiny fp32 case the oracle finishes in well under a second per round
     "tiny_fp32": _wl("tiny_fp32", "fp32", 512, 2, 256, 4, 2, 128, 4, 128, 32, 8, 4, 1, 36, (1, 2, 3)),
+    # the smallest pair that runs on the bf16 tensor-core path (d_head must be 64 there): two layers, two heads
+    "tiny_bf16": _wl("tiny_bf16", "bf16", 512, 2, 128, 2, 2, 128, 2, 128, 32, 8, 2, 1, 36, (5, 6, 7)),
     # GPT-2-small-shaped pair (the paper's 110M-class drafter size), 256 new tokens
     "small_bf16": _wl("small_bf16", "bf16", 50257, 12, 768, 12, 12, 768, 12, 1024, 256, 16, 8, 1, 256, (11, 12, 13)),
     # GPT-2-XL-shaped target with a 24-layer d=1024 drafter
@@ -209,3 +211,20 @@ def accept_case(rows: int, gamma: int, vocab: int, sigma: float, seed: int,
     else:
         ids[:] = rng.integers(0, vocab, size=(rows, gamma), dtype=np.int32)
     return AcceptCase(np.ascontiguousarray(lp), np.ascontiguousarray(lq), ids, float(sigma))
+
+
+def accept_row_index(gamma_base: int, gamma: int):
+    """Row indices that turn a case of draft length gamma_base into one of length gamma by cutting or repeating
+    rows: target row j and draft row j of the new case are rows j % gamma_base of the old one (so a target row stays
+    paired with the draft row it shares its common component with), the last target row (the one that follows a fully
+    accepted draft) stays the last.  Returns (target row index [gamma + 1], draft row index [gamma])."""
+    q_idx = np.arange(gamma, dtype=np.int64) % gamma_base
+    p_idx = np.concatenate([q_idx, np.array([gamma_base], dtype=np.int64)])
+    return p_idx, q_idx
+
+
+def resize_accept_case(case: AcceptCase, gamma: int) -> AcceptCase:
+    """The same rows with another draft length (see accept_row_index); pure re-indexing of `case`."""
+    p_idx, q_idx = accept_row_index(case.draft_ids.shape[1], gamma)
+    return AcceptCase(np.ascontiguousarray(case.logits_p[:, p_idx]), np.ascontiguousarray(case.logits_q[:, q_idx]),
+                      np.ascontiguousarray(case.draft_ids[:, q_idx]), case.sigma, dict(case.meta))

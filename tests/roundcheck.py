@@ -138,7 +138,7 @@ def check_whole_rounds(sess, mp, mq, wl, n_rounds, tol, seqs, n_sampled_steps=2,
                     x, gap = sd.argmax_with_gap(z + px.vocab_gumbels(wl.philox_seed, px.DRAFT, rnd, 0, int(j), b, V))
                     if x != slots[j]:
                         assert gap < parity.GAP_BAND
-                        log.append(("draft-near-tie", rnd, b, int(j), int(slots[j]), int(x), float(gap)))
+                        log.append(("draft", "gap", rnd, b, int(j), int(slots[j]), int(x), float(gap)))
                     assert abs(logq[j] - (z[slots[j]] - sd.logsumexp(z))) < 1e-5
                     # the reveal test of this slot: failed at every step before k, passed at k
                     for kk in range(T, k - 1, -1):

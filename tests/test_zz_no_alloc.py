@@ -40,6 +40,32 @@ def test_static_scratch_variant_matches_regular_entry_point_twice():
         assert int(n.min()) >= 0 and int(n.max()) <= gamma
 
 
+def test_static_scratch_variant_greedy_and_allocates_nothing():
+    """Temperature 0 (arg-max statistics in the scratch instead of soft-max sums), and the point of the entry point:
+    a call leaves the device's free memory and torch's own allocation count where they were."""
+    import paper_2408_05636_b200 as sdd
+    dev = "cuda:0"
+    rows, gamma, V = 4, 5, 3001
+    case = synth.accept_case(rows, gamma, V, 0.5, seed=72, draw_drafts=False)
+    top = case.logits_p[:, :-1].argmax(-1).astype(np.int32)
+    case.draft_ids[:, :2] = top[:, :2]                    # two accepted tokens per row
+    lp = torch.from_numpy(case.logits_p).to(dev)
+    lq = torch.from_numpy(case.logits_q).to(dev)
+    ids = torch.from_numpy(case.draft_ids).to(dev)
+    n_ref, out_ref, prob_ref = sdd.sdd_accept_logits(lp, lq, ids, 0.0, 0.0, 5, 1)
+    n, out, prob = _outputs(rows, gamma, dev)
+    sdd.sdd_accept_logits_static(lp, lq, ids, n, out, prob, 0.0, 0.0, 5, 1)     # first call: address look-up done
+    torch.cuda.synchronize()
+    free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+    sdd.sdd_accept_logits_static(lp, lq, ids, n, out, prob, 0.0, 0.0, 5, 1)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
+    assert torch.equal(n, n_ref) and torch.equal(out, out_ref) and torch.equal(prob, prob_ref)
+    assert int(n.min()) >= 2
+    with pytest.raises(AssertionError):                   # the binding refuses tensors of another element type
+        sdd.sdd_accept_logits_static(lp.to(torch.bfloat16), lq, ids, n, out, prob, 0.0, 0.0, 5, 1)
+
+
 def test_static_scratch_variant_rejects_oversize_problem():
     import paper_2408_05636_b200 as sdd
     dev = "cuda:0"
