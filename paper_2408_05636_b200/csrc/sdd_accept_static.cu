@@ -58,7 +58,7 @@ extern "C" int32_t sdd_accept_logits_static(const float* logits_p, const float* 
   // so nothing in the shared array has to be cleared between calls
   if (launch_row_stats(logits_p, rows_p, logits_q, itp == 0.f ? 0 : rows_q, V, itp, itq, partial, st) != cudaSuccess)
     return SDD_E_CUDA;
-  if (launch_accept(logits_p, logits_q, draft_ids, nullptr, nullptr, partial, partial + rows_p * chunks, rows, gamma, V, itp, itq,
+  if (launch_accept(logits_p, logits_q, draft_ids, nullptr, nullptr, partial, chunks, partial + rows_p * chunks, chunks, rows, gamma, V, itp, itq,
                     make_key(seed), (uint32_t)round, nullptr, accept_prob, n_accept, nullptr, out_ids, st) != cudaSuccess)
     return SDD_E_CUDA;
   return SDD_OK;

@@ -106,6 +106,7 @@ struct Buffers {
 
 struct Dims {
   int batch, gamma, T, max_new, V, tok_stride, chunks;
+  int chunks_cap;              // pairs per row that partial_p has room for (the LM head's fused statistics need more than row_stats)
   int lcap_max;                // padded rows per sequence of the largest drafter forward
   long long rows_q, rows_p;    // largest row counts of a drafter / target forward
   int max_prompt;
@@ -135,7 +136,7 @@ static size_t carve(const Dims& D, const Net& P, const Net& Q, uint8_t* base, Bu
   b.step_logits = (float*)take(Bn * G * V * 4);
   b.q_logits = (float*)take(Bn * G * V * 4);
   b.logits_p = (float*)take(Bn * (G + 1) * V * 4);
-  b.partial_p = (float2*)take(Bn * (G + 1) * D.chunks * sizeof(float2));
+  b.partial_p = (float2*)take(Bn * (G + 1) * D.chunks_cap * sizeof(float2));
   const size_t rq = (size_t)D.rows_q, rp = (size_t)D.rows_p;
   auto mx = [](size_t a, size_t c) { return a > c ? a : c; };
   b.h = (float*)take(mx(rq * Q.d, rp * P.d) * 4);
@@ -188,6 +189,7 @@ struct sdd_ctx {
   bool hilo;                   // SDD_HILO != 0 (default): hi/lo activation pairs in the target's MLP and LM head
   bool force_simt;             // SDD_GEMM=simt: run bf16 GEMMs on the CUDA-core kernel (cross-check)
   int bn_hint;                 // SDD_GEMM_BN: N tile of the tensor-core GEMM (0 = choose)
+  bool head_stats;             // SDD_HEAD_STATS != 0 (default): soft-max statistics from the target LM head's epilogue
   bool use_graph;              // SDD_GRAPH != 0: sdd_step replays a captured graph per row-count bucket
   struct GraphEntry { cudaGraphExec_t exec; uint64_t launches; };
   std::map<std::tuple<int, void*, void*>, GraphEntry> graphs;
@@ -246,6 +248,7 @@ static void fill_dims(const Net& P, const Net& Q, const sdd_params* p, int max_p
   D->batch = p->batch; D->gamma = p->gamma; D->T = p->T; D->max_new = p->max_new; D->V = P.vocab;
   D->tok_stride = P.n_ctx < Q.n_ctx ? P.n_ctx : Q.n_ctx;
   D->chunks = stats_chunks_for(P.vocab);
+  D->chunks_cap = head_stats_chunks_max(P.vocab) > D->chunks ? head_stats_chunks_max(P.vocab) : D->chunks;
   int lmax = max_prompt + p->max_new + p->gamma;
   if (lmax > D->tok_stride) lmax = D->tok_stride;
   D->lcap_max = (int)align_up((size_t)lmax, ROW_TILE);
@@ -261,13 +264,15 @@ static void fill_dims(const Net& P, const Net& Q, const sdd_params* p, int max_p
 template <typename T>
 static int gemm(sdd_ctx* c, int cat, const void* A, size_t a_elems, const void* W, const float* bias, long long M, int N,
                 int K, int epi, void* out, int ldc, const QkvDst* qd = nullptr, const void* A_lo = nullptr,
-                void* out_lo = nullptr, const int* skip = nullptr) {
+                void* out_lo = nullptr, const int* skip = nullptr, const HeadStats* stats = nullptr, int* stats_chunks = nullptr) {
+  if (stats_chunks != nullptr) *stats_chunks = 0;
   if (M <= 0) return SDD_OK;
   ProfScope prof(c, cat);
   c->launches++;
   if (std::is_same<T, __nv_bfloat16>::value && !c->force_simt) {
     SDD_CUDA(launch_gemm_tc((const __nv_bfloat16*)A, (long long)(a_elems / (size_t)K), (const __nv_bfloat16*)W, bias, (int)M,
-                            N, K, epi, out, ldc, c->bn_hint, &c->B.rs->status, c->st, qd, (const __nv_bfloat16*)A_lo, out_lo, skip));
+                            N, K, epi, out, ldc, c->bn_hint, &c->B.rs->status, c->st, qd, (const __nv_bfloat16*)A_lo, out_lo, skip,
+                            c->head_stats ? stats : nullptr, stats_chunks));
   } else {
     SDD_CUDA(launch_gemm_simt<T>((const T*)A, K, (const T*)W, bias, (int)M, N, K, epi, out, ldc, c->st, skip));
   }
@@ -387,7 +392,8 @@ static int forward_drafter(sdd_ctx* c) {
 // per-sequence length that fixes the rows' positions (see TargetMode); the caller has written the embeddings to B.h.
 template <typename T>
 static int forward_causal(sdd_ctx* c, const Net& N, void* kv, const int* len, int mode, int rows_per_seq, bool lm_head,
-                          float* logits_out, bool hilo, int gcat, int hcat, int acat) {
+                          float* logits_out, bool hilo, int gcat, int hcat, int acat, const HeadStats* stats = nullptr,
+                          int* stats_chunks = nullptr) {
   const Buffers& B = c->B;
   const Dims& D = c->D;
   const long long rows = (long long)D.batch * rows_per_seq;
@@ -425,14 +431,15 @@ static int forward_causal(sdd_ctx* c, const Net& N, void* kv, const int* len, in
     T* xf_lo = hilo ? (T*)B.xf_lo : nullptr;
     SDD_LAUNCH(c, CAT_LAYERNORM, launch_layernorm<T>(B.h, N.lnf_g, N.lnf_b, (T*)B.xf, rows, N.d, c->st, xf_lo));
     SDD_TRY(gemm<T>(c, hcat, B.xf, c->xf_elems, N.wte, nullptr, rows, D.V, N.d, EPI_STORE_F32, logits_out, D.V, nullptr,
-                    xf_lo));
+                    xf_lo, nullptr, nullptr, stats, stats_chunks));
   }
   return SDD_OK;
 }
 
 // target forward over rows_per_seq new tokens per sequence against the KV cache
 template <typename T>
-static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) {
+static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head, const HeadStats* stats = nullptr,
+                          int* stats_chunks = nullptr) {
   const Net& P = c->P;
   const Buffers& B = c->B;
   const Dims& D = c->D;
@@ -442,7 +449,7 @@ static int forward_target(sdd_ctx* c, int mode, int rows_per_seq, bool lm_head) 
   SDD_LAUNCH(c, CAT_GLUE, launch_embed_target<T>((const T*)P.wte, (const T*)P.wpe, B.tokens, D.tok_stride, B.ctx_len, B.slot_ids,
                                        D.batch, slot_stride, rows_per_seq, mode, P.d, B.h, c->st, P.vocab, &B.rs->status));
   return forward_causal<T>(c, P, B.kv, B.ctx_len, mode, rows_per_seq, lm_head, B.logits_p, c->hilo, CAT_GEMM_P, CAT_HEAD_P,
-                           CAT_ATTN_P);
+                           CAT_ATTN_P, stats, stats_chunks);
 }
 
 // One evaluation of the autoregressive drafter of a speculative-decoding round, producing the logits of slot j
@@ -516,10 +523,17 @@ static int verify_accept_t(sdd_ctx* c, int gamma, int32_t* out_ids, int32_t* n_o
   // nothing is tested, and the extra token is the draw from p (Algorithm 1 with an empty draft)
   const Buffers& B = c->B;
   const Dims& D = c->D;
-  SDD_TRY(forward_target<T>(c, TARGET_VERIFY, gamma + 1, true));
-  SDD_LAUNCH(c, CAT_STATS, launch_row_stats(B.logits_p, (long long)D.batch * (gamma + 1), nullptr, 0, D.V, c->inv_tau_p, 0.f,
-                                 B.partial_p, c->st));
-  SDD_LAUNCH(c, CAT_ACCEPT, launch_accept(B.logits_p, B.q_logits, B.slot_ids, B.logq, B.lse_q, B.partial_p, nullptr, D.batch, gamma, D.V,
+  // the rows' soft-max statistics come out of the LM head's epilogue where that runs on a persistent tensor-core
+  // kernel (chunks > 0); otherwise a pass over the logits produces them
+  const HeadStats hs = {c->inv_tau_p, B.partial_p, D.chunks_cap};
+  int chunks = 0;
+  SDD_TRY(forward_target<T>(c, TARGET_VERIFY, gamma + 1, true, &hs, &chunks));
+  if (chunks == 0) {
+    SDD_LAUNCH(c, CAT_STATS, launch_row_stats(B.logits_p, (long long)D.batch * (gamma + 1), nullptr, 0, D.V, c->inv_tau_p, 0.f,
+                                   B.partial_p, c->st));
+    chunks = D.chunks;
+  }
+  SDD_LAUNCH(c, CAT_ACCEPT, launch_accept(B.logits_p, B.q_logits, B.slot_ids, B.logq, B.lse_q, B.partial_p, chunks, nullptr, 0, D.batch, gamma, D.V,
                               c->inv_tau_p, c->inv_tau_p == 0.f ? 0.f : 1.f, c->key, 0u, B.rs, B.accept_prob, B.n_accept,
                               B.extra_token, nullptr, c->st));
   SDD_LAUNCH(c, CAT_COMMIT, launch_commit(B.tokens, D.tok_stride, B.ctx_len, B.n_emitted, B.slot_ids, B.n_accept, B.extra_token,
@@ -598,6 +612,8 @@ int32_t sdd_create(const sdd_model* target, const sdd_model* drafter, const sdd_
     c->hilo = hl == nullptr || atoi(hl) != 0;
     const char* bn = getenv("SDD_GEMM_BN");
     c->bn_hint = bn ? atoi(bn) : 0;
+    const char* hs = getenv("SDD_HEAD_STATS");
+    c->head_stats = hs == nullptr || atoi(hs) != 0;
     const char* gr = getenv("SDD_GRAPH");
     // the legacy default stream cannot be captured: rounds are then enqueued kernel by kernel
     c->use_graph = (gr == nullptr || atoi(gr) != 0) && c->st != nullptr && c->st != cudaStreamLegacy;
@@ -955,7 +971,7 @@ int32_t sdd_accept_logits(const float* logits_p, const float* logits_q, const in
   const long long rows_p = (long long)rows * (gamma + 1), rows_q = (long long)rows * gamma;
   const int chunks = stats_chunks_for(V);
   SDD_CUDA(launch_row_stats(logits_p, rows_p, logits_q, itp == 0.f ? 0 : rows_q, V, itp, itq, partial, st));
-  SDD_CUDA(launch_accept(logits_p, logits_q, draft_ids, nullptr, nullptr, partial, partial + rows_p * chunks, rows, gamma, V, itp, itq,
+  SDD_CUDA(launch_accept(logits_p, logits_q, draft_ids, nullptr, nullptr, partial, chunks, partial + rows_p * chunks, chunks, rows, gamma, V, itp, itq,
                          make_key(seed), (uint32_t)round, nullptr, accept_prob, n_accept, nullptr, out_ids, st));
   return SDD_OK;
 }

@@ -14,6 +14,10 @@
 // Shared memory: the K tile of a stage is dead once S = Q K^T has completed and stays unused until P V has
 // completed (only then is the stage handed back to the producer), so the first half of P (keys 0..63) is written
 // over it; with that the CTA needs 96 KB and two CTAs share an SM, one's soft-max overlapping the other's MMAs.
+// PIPE variant (grids of at most one CTA per SM, where a CTA's chain of key tiles is what bounds the launch): S is
+// double-buffered in TMEM (512 columns, one CTA per SM) and the K / V^T ring has three stages, so S(t+1) = Q K(t+1)^T is
+// issued before the MMA thread waits for P(t) and is complete when the soft-max warps get to it; a tile's chain is then
+// soft-max -> next soft-max instead of S -> soft-max -> P V -> S.
 // Waits are bounded exactly as in the GEMM kernel.
 #include <cstdlib>
 #include <mutex>
@@ -32,14 +36,17 @@ constexpr int AT_P_BYTES = 128 * 64 * 2;            // P k-block 1 (keys 64..127
 constexpr int AT_K_BYTES = 128 * 64 * 2;            // 16 KB
 constexpr int AT_VT_BYTES = 2 * 64 * 64 * 2;        // two boxes [64 d_head rows x 64 keys]: 16 KB
 constexpr int AT_STAGE_BYTES = AT_K_BYTES + AT_VT_BYTES;
-constexpr int AT_KV_STAGES = 2;
-constexpr int AT_BAR_OFF = AT_Q_BYTES + AT_P_BYTES + AT_KV_STAGES * AT_STAGE_BYTES;   // 96 KB: two CTAs per SM
-constexpr int AT_SMEM = AT_BAR_OFF + 1024 + 128 + 3 * 1024;   // barriers, then the soft-max exchange arrays
-constexpr uint32_t AT_TMEM_COLS = 256;              // S: columns 0..127, PV accumulators: 128..191 and 192..255
+// PIPE = false: two K / V^T stages, 96 KB, two CTAs per SM; TMEM: S in columns 0..127, PV accumulators 128..191 and 192..255
+// PIPE = true : three stages, 128 KB, one CTA per SM; TMEM: S buffers 0..127 and 128..255, PV accumulators 256..319 and 320..383
+template <bool PIPE> constexpr int at_stages() { return PIPE ? 3 : 2; }
+template <bool PIPE> constexpr int at_bar_off() { return AT_Q_BYTES + AT_P_BYTES + at_stages<PIPE>() * AT_STAGE_BYTES; }
+template <bool PIPE> constexpr int at_smem() { return at_bar_off<PIPE>() + 1024 + 128 + 3 * 1024; }   // barriers, then the soft-max exchange arrays
+template <bool PIPE> constexpr uint32_t at_tmem_cols() { return PIPE ? 512u : 256u; }
+template <bool PIPE> constexpr uint32_t at_acc_col() { return PIPE ? 256u : 128u; }
 // key-split launches add a receive area for the other CTAs' partial states (it must not lie over tiles that this CTA
 // may still be using when a faster CTA sends): at most 136 rows of 64 floats plus their m and l
-constexpr int AT_RECV_OFF = AT_BAR_OFF + 3328;
-constexpr int AT_SMEM_SPLIT = AT_RECV_OFF + 36 * 1024 + 1024;
+template <bool PIPE> constexpr int at_recv_off() { return at_bar_off<PIPE>() + 3328; }
+template <bool PIPE> constexpr int at_smem_split() { return at_recv_off<PIPE>() + 36 * 1024 + 1024; }
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -73,9 +80,15 @@ __device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, float a, fl
   asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
-__global__ void __launch_bounds__(AT_THREADS, 2)
+template <bool PIPE>
+__global__ void __launch_bounds__(AT_THREADS, PIPE ? 1 : 2)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_vt, const AttnParams prm) {
+  constexpr int AT_KV_STAGES = at_stages<PIPE>();
+  constexpr int AT_BAR_OFF = at_bar_off<PIPE>();
+  constexpr int AT_RECV_OFF = at_recv_off<PIPE>();
+  constexpr uint32_t AT_TMEM_COLS = at_tmem_cols<PIPE>();
+  constexpr uint32_t ACC_COL = at_acc_col<PIPE>();
   const int kv_split = prm.kv_split, kv_rank = (int)blockIdx.x % kv_split;   // cluster = kv_split consecutive CTAs in x
   const int qt = (int)blockIdx.x / kv_split, h = blockIdx.y, b = blockIdx.z;
   pdl_wait();   // ctx_len and Q / K / V^T come from earlier kernels
@@ -105,15 +118,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   auto sK = [&](int s) { return base + AT_Q_BYTES + AT_P_BYTES + s * AT_STAGE_BYTES; };
   auto sVT = [&](int s) { return sK(s) + AT_K_BYTES; };
   const uint32_t bars = base + AT_BAR_OFF;
-  const uint32_t q_full = bars, s_full = bars + 8, p_ready = bars + 16, pv_full = bars + 24;
-  auto kv_full = [&](int s) { return bars + 32 + 8u * s; };
-  auto kv_empty = [&](int s) { return bars + 48 + 8u * s; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + AT_BAR_OFF + 64);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + AT_BAR_OFF + 72);
+  const uint32_t q_full = bars, p_ready = bars + 8, pv_full = bars + 16;
+  auto s_full = [&](int b) { return bars + 24 + 8u * b; };            // one per S buffer (PIPE: two, else only [0])
+  auto kv_full = [&](int s) { return bars + 40 + 8u * s; };
+  auto kv_empty = [&](int s) { return bars + 64 + 8u * s; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + AT_BAR_OFF + 96);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + AT_BAR_OFF + 104);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    mbar_init(q_full, 1); mbar_init(s_full, 1); mbar_init(p_ready, 256); mbar_init(pv_full, 1);
+    mbar_init(q_full, 1); mbar_init(s_full(0), 1); mbar_init(s_full(1), 1); mbar_init(p_ready, 256); mbar_init(pv_full, 1);
     for (int s = 0; s < AT_KV_STAGES; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -131,8 +145,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       int issued = 0;
       for (int it = 0; it < my_kt; ++it) {
         const int t = kv_rank + it * kv_split;      // key tile; `it` counts this CTA's iterations (stages, phases)
-        const int s = it & 1;
-        if (!mbar_wait(kv_empty(s), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag, prm.status)) break;
+        const int s = it % AT_KV_STAGES;
+        if (!mbar_wait(kv_empty(s), ((uint32_t)(it / AT_KV_STAGES) & 1u) ^ 1u, abort_flag, prm.status)) break;
         mbar_expect_tx(kv_full(s), AT_STAGE_BYTES);
         tma_load_2d(sK(s), &map_k, kv_full(s), prm.k_col0 + h * AT_DH, b * prm.k_rows_per_seq + t * 128);
         tma_load_2d(sVT(s), &map_vt, kv_full(s), t * 128, b * prm.d + h * AT_DH);
@@ -144,7 +158,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         while (!mbar_try(q_full, 0u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
         for (int t = issued > AT_KV_STAGES ? issued - AT_KV_STAGES : 0; t < issued; ++t) {
           t0 = clock64();
-          while (!mbar_try(kv_full(t & 1), (uint32_t)(t >> 1) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+          while (!mbar_try(kv_full(t % AT_KV_STAGES), (uint32_t)(t / AT_KV_STAGES) & 1u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
         }
       }
     }
@@ -155,27 +169,41 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       constexpr uint32_t idesc_pv = make_idesc<64>();
       bool ok = mbar_wait(q_full, 0u, abort_flag, prm.status);
       const uint64_t dq = make_smem_desc(sQ);
-      for (int t = 0; t < my_kt && ok; ++t) {        // t: this CTA's iteration (the key tile does not matter here)
-        const int s = t & 1;
-        ok = mbar_wait(kv_full(s), (uint32_t)(t >> 1) & 1u, abort_flag, prm.status);
-        if (!ok) break;
+      // S(t) = Q K(t)^T into S buffer t & 1 (PIPE) or the one S buffer; t counts this CTA's iterations
+      auto issue_s = [&](int t) -> bool {
+        const int s = t % AT_KV_STAGES;
+        if (!mbar_wait(kv_full(s), (uint32_t)(t / AT_KV_STAGES) & 1u, abort_flag, prm.status)) return false;
         fence_after_sync();
         const uint64_t dk = make_smem_desc(sK(s));
+        const uint32_t sc = PIPE ? (uint32_t)(t & 1) * 128u : 0u;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) umma(tmem_base, dq + 2u * k, dk + 2u * k, idesc_s, k > 0 ? 1u : 0u);
-        umma_commit(s_full);
+        for (int k = 0; k < 4; ++k) umma(tmem_base + sc, dq + 2u * k, dk + 2u * k, idesc_s, k > 0 ? 1u : 0u);
+        umma_commit(s_full(PIPE ? (t & 1) : 0));
+        return true;
+      };
+      if (PIPE && ok) ok = issue_s(0);
+      for (int t = 0; t < my_kt && ok; ++t) {        // t: this CTA's iteration (the key tile does not matter here)
+        const int s = t % AT_KV_STAGES;
+        if (PIPE) {
+          // the next tile's scores are issued before the wait for this tile's probabilities: the soft-max warps are done
+          // with S buffer (t + 1) & 1 since p_ready(t - 1), which this thread has seen
+          if (t + 1 < my_kt) ok = issue_s(t + 1);
+        } else {
+          ok = issue_s(t);
+        }
+        if (!ok) break;
         ok = mbar_wait(p_ready, (uint32_t)t & 1u, abort_flag, prm.status);
         if (!ok) break;
         fence_after_sync();
-        // one accumulator per half of the key tile (columns 128..191: keys 0..63, 192..255: keys 64..127); both add up
-        // over the CTA's tiles in TMEM
+        // one accumulator per half of the key tile (keys 0..63 and keys 64..127 of the tile); both add up over the
+        // CTA's tiles in TMEM
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb) {
           const uint64_t dp = make_smem_desc(kb == 0 ? sK(s) : sP);
           const uint64_t dv = make_smem_desc(sVT(s) + kb * (64 * 64 * 2));
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            umma(tmem_base + 128u + (uint32_t)(kb * 64), dp + 2u * k, dv + 2u * k, idesc_pv, (t | k) ? 1u : 0u);
+            umma(tmem_base + ACC_COL + (uint32_t)(kb * 64), dp + 2u * k, dv + 2u * k, idesc_pv, (t | k) ? 1u : 0u);
         }
         umma_commit(pv_full);
         umma_commit(kv_empty(s));
@@ -207,31 +235,44 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // when the thread's maximum has grown by more than 2^8 since its reference was set (the probabilities are then
     // bounded by 256, exact arithmetic otherwise unchanged), so the common tile has no fold, no exchange between the
     // halves and no barrier among the warps.  The halves are combined once, after the last tile.
-    const uint32_t t_acc = t_lane + 128u + (uint32_t)(hf * 64);
+    const uint32_t t_acc = t_lane + ACC_COL + (uint32_t)(hf * 64);
     uint32_t v[32];
     for (int it = 0; it < my_kt; ++it) {
       const int t = kv_rank + it * kv_split;           // key tile; `it` counts this CTA's iterations (stages, phases)
-      ok = __all_sync(0xffffffffu, mbar_wait(s_full, (uint32_t)it & 1u, abort_flag, prm.status));
+      ok = __all_sync(0xffffffffu, mbar_wait(s_full(PIPE ? (it & 1) : 0), (uint32_t)(PIPE ? (it >> 1) : it) & 1u, abort_flag,
+                                             prm.status));
       if (!ok) break;
       fence_after_sync();
       const int key0 = t * 128 + hf * 64;
+      const uint32_t t_s = t_lane + (PIPE ? (uint32_t)(it & 1) * 128u : 0u);    // this tile's S buffer
       // this thread's 64 probabilities are one row of a P k-block: block 0 lies over the stage's (consumed) K tile
-      uint8_t* p_row = gbase + (hf == 0 ? AT_Q_BYTES + AT_P_BYTES + (it & 1) * AT_STAGE_BYTES : AT_Q_BYTES) + r * 128;
+      uint8_t* p_row = gbase + (hf == 0 ? AT_Q_BYTES + AT_P_BYTES + (it % AT_KV_STAGES) * AT_STAGE_BYTES : AT_Q_BYTES) + r * 128;
       // tcgen05.ld / st are warp-collective: every branch around them is taken by whole warps
       const bool full_w = __all_sync(0xffffffffu, key0 + 64 <= key_limit);
-      // the 64 scores are read twice from TMEM (once for the maximum, once for the exponentials) instead of being kept
-      // in 64 registers: two CTAs per SM need the kernel to stay below 100 registers
+      // !PIPE: the 64 scores are read twice from TMEM (once for the maximum, once for the exponentials) instead of being
+      // kept in 64 registers: two CTAs per SM need the kernel to stay below 100 registers.  PIPE (one CTA per SM) keeps them.
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
-#pragma unroll 1
-      for (int cc = 0; cc < 2; ++cc) {
-        tmem_ld32(t_lane + (uint32_t)(hf * 64 + cc * 32), v);
+      auto max_chunk = [&](const uint32_t (&x)[32], int cc) {
         if (full_w) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(v[j]));
+          for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(x[j]));
         } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (key0 + cc * 32 + j < key_limit) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(v[j]));
+            if (key0 + cc * 32 + j < key_limit) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(x[j]));
+        }
+      };
+      uint32_t sc[PIPE ? 2 : 1][32];
+      if constexpr (PIPE) {
+        tmem_ld32(t_s + (uint32_t)(hf * 64), sc[0]);
+        max_chunk(sc[0], 0);
+        tmem_ld32(t_s + (uint32_t)(hf * 64 + 32), sc[1]);
+        max_chunk(sc[1], 1);
+      } else {
+#pragma unroll 1
+        for (int cc = 0; cc < 2; ++cc) {
+          tmem_ld32(t_s + (uint32_t)(hf * 64 + cc * 32), v);
+          max_chunk(v, cc);
         }
       }
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale;     // -inf: no visible key
@@ -261,10 +302,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       const float m_use = m == -INFINITY ? 0.f : m;
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-      auto exp_chunk = [&](auto full_tag, int cc) {
+      auto exp_chunk = [&](auto full_tag, auto cc_tag) {
         constexpr bool FULL = decltype(full_tag)::value;
-        tmem_ld32(t_lane + (uint32_t)(hf * 64 + cc * 32), v);
-        const uint32_t (&x)[32] = v;
+        constexpr int cc = decltype(cc_tag)::value;
+        if constexpr (!PIPE) tmem_ld32(t_s + (uint32_t)(hf * 64 + cc * 32), v);
+        const uint32_t (&x)[32] = PIPE ? sc[PIPE ? cc : 0] : v;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           uint32_t pk[4];
@@ -286,8 +328,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       };
       // two copies, chosen by a real (warp-uniform) branch: the visibility tests cost a third of the issue slots when
       // they are predicated into the common unmasked path
-      if (full_w) { exp_chunk(std::true_type{}, 0); exp_chunk(std::true_type{}, 1); }
-      else { exp_chunk(std::false_type{}, 0); exp_chunk(std::false_type{}, 1); }
+      using C0 = std::integral_constant<int, 0>;
+      using C1 = std::integral_constant<int, 1>;
+      if (full_w) { exp_chunk(std::true_type{}, C0{}); exp_chunk(std::true_type{}, C1{}); }
+      else { exp_chunk(std::false_type{}, C0{}); exp_chunk(std::false_type{}, C1{}); }
       l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       fence_before_sync();          // accumulator reads / writes above are ordered before the MMA that follows the arrive
       fence_async_smem();
@@ -312,10 +356,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       l = l * w_me + l_o * w_o;
       m = mm;
       if (my_kt > 0) {
-        tmem_ld32(t_lane + 128u + (uint32_t)(hf * 64 + hf * 32), v);           // own half's accumulator
+        tmem_ld32(t_lane + ACC_COL + (uint32_t)(hf * 64 + hf * 32), v);        // own half's accumulator
 #pragma unroll
         for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(v[j]) * w_me;
-        tmem_ld32(t_lane + 128u + (uint32_t)((hf ^ 1) * 64 + hf * 32), v);     // the other half's
+        tmem_ld32(t_lane + ACC_COL + (uint32_t)((hf ^ 1) * 64 + hf * 32), v);  // the other half's
 #pragma unroll
         for (int j = 0; j < 32; ++j) o[j] = fmaf(__uint_as_float(v[j]), w_o, o[j]);
       }
@@ -398,7 +442,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 }  // namespace tc
 
 cudaError_t tc_prepare_attn() {
-  return cudaFuncSetAttribute(tc::attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AT_SMEM_SPLIT);
+  cudaError_t e = cudaFuncSetAttribute(tc::attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::at_smem_split<false>());
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(tc::attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::at_smem_split<true>());
 }
 
 cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q_ld, int q_col0, const __nv_bfloat16* k,
@@ -422,6 +468,10 @@ cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q
   p.q_rows_per_seq = q_rows_per_seq; p.k_rows_per_seq = k_rows_per_seq; p.q_col0 = q_col0; p.k_col0 = k_col0;
   p.d = d; p.status = status; p.skip = skip; p.kv_split = 1;
   dim3 grid((q_rows_per_seq + 127) / 128, n_head, batch);
+  // at most one CTA per SM: the launch is bound by each CTA's chain of key tiles, not by throughput -> PIPE variant
+  // (SDD_ATTN_PIPE=0 switches it off)
+  static const bool pipe_on = [] { const char* e = getenv("SDD_ATTN_PIPE"); return e == nullptr || atoi(e) != 0; }();
+  const bool pipe = pipe_on && (long long)grid.x * grid.y * grid.z <= 148;
   // Unmasked attention on a grid that leaves most SMs idle (one sequence): the key tiles of a query tile are shared out
   // over a cluster of CTAs, which shortens the chain of dependent tiles per CTA; CTA 0 merges the partial states.
   // SDD_ATTN_SPLIT=0 switches it off.
@@ -437,11 +487,12 @@ cudaError_t launch_attn_tc(const __nv_bfloat16* q, long long q_rows_total, int q
     if ((e == nullptr || atoi(e) != 0) && split > 1) {
       p.kv_split = split;
       grid.x *= split;
-      launch_k_cluster(attn_tc_kernel, grid, dim3(AT_THREADS), AT_SMEM_SPLIT, st, (unsigned)split, mq, mk, mv, p);
+      launch_k_cluster(attn_tc_kernel<false>, grid, dim3(AT_THREADS), at_smem_split<false>(), st, (unsigned)split, mq, mk, mv, p);
       return cudaGetLastError();
     }
   }
-  launch_k(attn_tc_kernel, dim3(grid), dim3(AT_THREADS), AT_SMEM, st, mq, mk, mv, p);
+  if (pipe) launch_k(attn_tc_kernel<true>, dim3(grid), dim3(AT_THREADS), at_smem<true>(), st, mq, mk, mv, p);
+  else launch_k(attn_tc_kernel<false>, dim3(grid), dim3(AT_THREADS), at_smem<false>(), st, mq, mk, mv, p);
   return cudaGetLastError();
 }
 

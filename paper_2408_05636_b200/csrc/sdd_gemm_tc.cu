@@ -354,10 +354,156 @@ __device__ __forceinline__ void epilogue_manual(uint32_t tmem_acc, int m0, int n
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// LM-head epilogues that also produce the rows' soft-max statistics (HeadStats): the logits are stored as by
+// EPI_STORE_F32, and every (token row, slice of the vocabulary) gets one pair (max z, sum exp(z - max)), z = logit *
+// inv_tau -- or (max logit, index of its first occurrence) when inv_tau == 0 -- so that the acceptance step never
+// reads the logit matrix for its statistics.
+// ---------------------------------------------------------------------------------------------
+// Reduction of 32 values per lane across the warp in 31 shuffles: on return a[0] of lane L holds op over all lanes of
+// their a[L] (each step halves the values a lane keeps and exchanges the other half with the lane `o` away).
+template <typename Op>
+__device__ __forceinline__ void warp_reduce_scatter(float (&a)[32], int lane, Op op) {
+#pragma unroll
+  for (int st = 0; st < 5; ++st) {
+    const int o = 16 >> st;            // partner distance = number of values kept
+    const bool upper = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      if (i < o) {
+        const float send = upper ? a[i] : a[i + o];
+        const float keep = upper ? a[i + o] : a[i];
+        a[i] = op(keep, __shfl_xor_sync(0xffffffffu, send, o));
+      }
+    }
+  }
+}
+// the same for (value, index) pairs under the arg-max order (ties: lowest index)
+__device__ __forceinline__ void warp_reduce_scatter_argmax(float (&a)[32], int (&ix)[32], int lane) {
+#pragma unroll
+  for (int st = 0; st < 5; ++st) {
+    const int o = 16 >> st;
+    const bool upper = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      if (i < o) {
+        const float send = upper ? a[i] : a[i + o];
+        const int send_i = upper ? ix[i] : ix[i + o];
+        ArgMax keep;
+        keep.s = upper ? a[i + o] : a[i];
+        keep.i = upper ? ix[i + o] : ix[i];
+        ArgMax got;
+        got.s = __shfl_xor_sync(0xffffffffu, send, o);
+        got.i = __shfl_xor_sync(0xffffffffu, send_i, o);
+        keep = argmax_better(keep, got);
+        a[i] = keep.s;
+        ix[i] = keep.i;
+      }
+    }
+  }
+}
+
+// SWAP orientation (tile = 128 vocabulary rows x up to BN tokens; a thread owns one vocabulary row r): out[token][r]
+// = logit, and per warp one pair per token over the warp's 32 vocabulary rows: slice index = tile * 4 + q.
+template <int BN>
+__device__ __forceinline__ void epilogue_head_swap(uint32_t tmem_acc, int m0, int q, int lane, int V, int tokens,
+                                                   float* __restrict__ out, int ldc, const HeadStats& hs, int chunks,
+                                                   int tile) {
+  const int r = m0 + q * 32 + lane;
+  const bool r_ok = r < V;
+  const bool greedy = hs.inv_tau == 0.f;
+  const float k = hs.inv_tau * 1.4426950408889634f;
+#pragma unroll 1
+  for (int cc = 0; cc < BN / 32; ++cc) {
+    const int c0 = cc * 32;
+    if (c0 >= tokens) break;
+    uint32_t v[32];
+    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+    float x[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const float acc = __uint_as_float(v[j]);
+      if (r_ok && c0 + j < tokens) out[(long long)(c0 + j) * ldc + r] = acc;
+      x[j] = r_ok ? acc : -INFINITY;
+    }
+    float2 pair;
+    if (greedy) {
+      int ix[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) ix[j] = r_ok ? r : 0x7fffffff;
+      warp_reduce_scatter_argmax(x, ix, lane);
+      pair = make_float2(x[0], __int_as_float(ix[0]));
+    } else {
+      float mx[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) mx[j] = x[j];
+      warp_reduce_scatter(mx, lane, [](float a, float b) { return fmaxf(a, b); });
+      const float m_mine = mx[0];                      // maximum of token c0 + lane over the warp's rows
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float mj = __shfl_sync(0xffffffffu, m_mine, j);
+        x[j] = (r_ok && mj > -INFINITY) ? exp2f((x[j] - mj) * k) : 0.f;
+      }
+      warp_reduce_scatter(x, lane, [](float a, float b) { return a + b; });
+      pair = make_float2(m_mine * hs.inv_tau, x[0]);
+    }
+    if (c0 + lane < tokens) hs.partial[(long long)(c0 + lane) * chunks + tile * 4 + q] = pair;
+  }
+}
+
+// NORMAL orientation (tile = 128 token rows x BN vocabulary columns; a thread owns one token row): out[r][column] =
+// logit, and one pair per (token row, tile): slice index = the tile's index along the vocabulary.
+template <int BN>
+__device__ __forceinline__ void epilogue_head_normal(uint32_t tmem_acc, int m0, int n0, int q, int lane, int rows, int V,
+                                                     float* __restrict__ out, int ldc, const HeadStats& hs, int chunks,
+                                                     int n_tile) {
+  const int r = m0 + q * 32 + lane;
+  const bool r_ok = r < rows;
+  const bool greedy = hs.inv_tau == 0.f;
+  const float k = hs.inv_tau * 1.4426950408889634f;
+  float m = -INFINITY, sum = 0.f;
+  int arg = 0x7fffffff;
+#pragma unroll 1
+  for (int cc = 0; cc < BN / 32; ++cc) {
+    const int c0 = n0 + cc * 32;
+    if (c0 >= V) break;
+    uint32_t v[32];
+    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
+    float* o = out + (long long)r * ldc + c0;
+    float cm = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const float x = __uint_as_float(v[j]);
+      if (c0 + j < V) {
+        if (r_ok) o[j] = x;
+        if (greedy) { if (x > cm) { cm = x; if (x > m) arg = c0 + j; } }
+        else cm = fmaxf(cm, x);
+      }
+    }
+    if (greedy) {
+      m = fmaxf(m, cm);
+    } else if (cm > -INFINITY) {
+      const float m_new = fmaxf(m, cm);
+      sum = m == -INFINITY ? 0.f : sum * exp2f((m - m_new) * k);
+      m = m_new;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (c0 + j < V) sum += exp2f((__uint_as_float(v[j]) - m) * k);
+    }
+  }
+  if (r_ok) hs.partial[(long long)r * chunks + n_tile] = greedy ? make_float2(m, __int_as_float(arg)) : make_float2(m * hs.inv_tau, sum);
+}
+
 // grid = (N tiles, M tiles, K splits).  With more than one K split every CTA accumulates its share of the K
 // range and adds it to the fp32 output with atomics (EPI_RESIDUAL only; the bias is added by split 0).
+// Tiles of 128 columns or more (NORMAL orientation) are drained by two groups of four epilogue warps, each with half of
+// the tile's columns, staging buffers and named barriers of its own: the one-tile kernel cannot overlap its epilogue
+// with anything, and a 128 x 256 tile costs four warps several microseconds (one wave of such CTAs is the whole launch).
+template <int BN, bool SWAP>
+constexpr int one_tile_threads() { return (!SWAP && BN >= 128) ? 320 : THREADS; }
+
 template <int BN, bool SWAP, bool HILO, bool DEEP>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(one_tile_threads<BN, SWAP>())
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ OutMaps maps_out, int tma_out,
                int rows_a, int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out,
@@ -488,10 +634,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (ok) umma_commit(tmem_full_bar);
     }
   } else {
-    // epilogue warps 2..5 own TMEM lane quarters (warp id % 4)
+    // epilogue warps own TMEM lane quarters (warp id % 4); with two groups, group g = (warp - 2) / 4 takes the chunks
+    // [g * BN / 64, (g + 1) * BN / 64) and the staging buffers at 32 KB * g of the (now idle) operand ring
     const int q = warp & 3;
+    constexpr bool TWO = one_tile_threads<BN, SWAP>() == 320;
+    const int grp = TWO ? (warp - 2) >> 2 : 0;
+    const EpiGroup eg = TWO ? EpiGroup{grp * (BN / 64), (grp + 1) * (BN / 64), 2, 2 + grp, 64 + grp * 128} : whole_tile_group<BN>();
+    uint8_t* stage_g = generic_base + grp * (2 * 128 * 128);
+    const uint32_t stage_u = base + grp * (2 * 128 * 128);
     // every lane waits; the outcome is made warp-uniform because tcgen05.ld is a warp-wide instruction
-    // (and uniform over the four epilogue warps, which meet at named barriers in the TMA-store path)
+    // (and uniform over the four warps of a group, which meet at named barriers in the TMA-store path)
     float* bias_s = reinterpret_cast<float*>(generic_base + STAGES * STAGE_BYTES + 256);
     // tma_out == 2 (fused QKV): only tiles that lie wholly in the columns kept in place (Q, and K without a cache)
     // are plain row-major stores; the others scatter into the K cache / V^T and take the manual path
@@ -499,22 +651,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // straddle sequences there)
     const bool use_tma = !SWAP && (tma_out == 1 || (tma_out >= 2 && n0 + BN <= (qd.k_dst != nullptr ? qd.d : 2 * qd.d)));
     const bool vt_tma = !SWAP && tma_out == 3 && n0 >= 2 * qd.d && n0 + BN <= rows_b;
-    if (use_tma || vt_tma) stage_bias<BN>(bias_s, bias, n0, rows_b);     // while the main loop runs
-    const bool ready = named_bar_and(1, 128, mbar_wait(tmem_full_bar, 0u, abort_flag, status));
+    if (use_tma || vt_tma) stage_bias(bias_s, bias, n0, rows_b, eg);     // while the main loop runs
+    const bool ready = named_bar_and(TWO ? 4 + grp : 1, 128, mbar_wait(tmem_full_bar, 0u, abort_flag, status));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ready && use_tma) {
       int n_store = 0;
-      epilogue_tma<BN>(tmem_base, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &maps_out.out, generic_base, base,
-                       n_store);
-      if (threadIdx.x == 64) tma_wait_group_read<0>();      // shared memory stays valid until the copies have read it
+      epilogue_tma<BN>(tmem_base, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &maps_out.out, stage_g, stage_u,
+                       n_store, eg);
+      if ((int)threadIdx.x == eg.first_tid) tma_wait_group_read<0>();      // shared memory stays valid until the copies have read it
     } else if (ready && vt_tma) {
       int n_store = 0;
       const int sb = m0 / qd.rows_per_seq;
-      epilogue_vt<BN>(tmem_base, q, lane, bias_s, &maps_out.vt, generic_base, base, n_store, sb * qd.d + (n0 - 2 * qd.d),
-                      m0 - sb * qd.rows_per_seq);
-      if (threadIdx.x == 64) tma_wait_group_read<0>();
+      epilogue_vt<BN>(tmem_base, q, lane, bias_s, &maps_out.vt, stage_g, stage_u, n_store, sb * qd.d + (n0 - 2 * qd.d),
+                      m0 - sb * qd.rows_per_seq, eg);
+      if ((int)threadIdx.x == eg.first_tid) tma_wait_group_read<0>();
     } else if (ready) {
-      epilogue_manual<BN, SWAP, SWAP>(tmem_base, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, split, qd);
+      epilogue_manual<BN, SWAP, SWAP>(tmem_base, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, split, qd, eg.c_begin,
+                                      eg.c_end);
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -550,7 +703,7 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                        const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ OutMaps maps_out, int tma_out,
                        int rows_a, int rows_b, int K, int epi, const float* __restrict__ bias, void* __restrict__ out,
                        void* __restrict__ out_lo, int ldc, int* status, const QkvDst qd, const int* __restrict__ skip,
-                       int tiles_m, int tiles_n, int n_fastest) {
+                       int tiles_m, int tiles_n, int n_fastest, const HeadStats hs, int hs_chunks) {
   constexpr int STAGES = persist_stages<BN, HILO, SWAP>();
   constexpr int STAGE_BYTES = stage_bytes<BN, SWAP, HILO>();
   constexpr int LO_OFF = BM * BK * 2 + BN * BK * 2;
@@ -693,8 +846,12 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       if (!ready) break;
       fence_after_sync();
       const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
-      if (SWAP)
+      if (SWAP && hs.partial != nullptr)        // LM head: logits + their soft-max statistics
+        epilogue_head_swap<BN>(acc, m0, q, lane, rows_a, rows_b, reinterpret_cast<float*>(out), ldc, hs, hs_chunks, m0 / BM);
+      else if (SWAP)
         epilogue_manual<BN, true>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, false, qd);
+      else if (hs.partial != nullptr)
+        epilogue_head_normal<BN>(acc, m0, n0, q, lane, rows_a, rows_b, reinterpret_cast<float*>(out), ldc, hs, hs_chunks, n0 / BN);
       else if (use_tma)
         epilogue_tma<BN>(acc, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &maps_out.out,
                          generic_base + STAGING_OFF, base + STAGING_OFF, n_store);
@@ -947,7 +1104,7 @@ static cudaError_t launch_cfg2(const CUtensorMap& ma, const CUtensorMap& mb, con
                               int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias, void* out, void* out_lo,
                               int ldc, int* status, cudaStream_t st, const QkvDst& qd, int splits, const int* skip) {
   dim3 grid((rows_b + BN - 1) / BN, (rows_a + BM - 1) / BM, splits);
-  launch_k(gemm_tc_kernel<BN, SWAP, HILO, DEEP>, grid, dim3(THREADS), smem_bytes<BN, SWAP, HILO, DEEP>(), st, ma, mb, ml, mo, tma_out,
+  launch_k(gemm_tc_kernel<BN, SWAP, HILO, DEEP>, grid, dim3(one_tile_threads<BN, SWAP>()), smem_bytes<BN, SWAP, HILO, DEEP>(), st, ma, mb, ml, mo, tma_out,
            rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip);
   return cudaGetLastError();
 }
@@ -966,25 +1123,27 @@ static cudaError_t launch_cfg(const CUtensorMap& ma, const CUtensorMap& mb, cons
 template <int BN, bool HILO>
 static cudaError_t launch_persist(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const OutMaps& mo,
                                   int tma_out, int rows_a, int rows_b, int K, int epi, const float* bias, void* out,
-                                  void* out_lo, int ldc, int* status, cudaStream_t st, const QkvDst& qd, const int* skip) {
+                                  void* out_lo, int ldc, int* status, cudaStream_t st, const QkvDst& qd, const int* skip,
+                                  const HeadStats& hs = HeadStats{}) {
   const int tiles_m = (rows_a + BM - 1) / BM, tiles_n = (rows_b + BN - 1) / BN;
   const long long tiles = (long long)tiles_m * tiles_n;
   const unsigned grid = (unsigned)(tiles < 148 ? tiles : 148);
   launch_k(gemm_tc_persist_kernel<BN, HILO>, dim3(grid), dim3(THREADS), persist_smem_bytes<BN, HILO>(), st, ma, mb, ml, mo,
            tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n,
-           (long long)rows_b * K * 2 <= (48ll << 20) ? 1 : 0);
+           (long long)rows_b * K * 2 <= (48ll << 20) ? 1 : 0, hs, tiles_n);
   return cudaGetLastError();
 }
 
 template <int BN, bool HILO>
 static cudaError_t launch_persist_swap(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& ml, const OutMaps& mo,
                                        int rows_a, int rows_b, int K, int epi, const float* bias, void* out, void* out_lo,
-                                       int ldc, int* status, cudaStream_t st, const QkvDst& qd, const int* skip) {
+                                       int ldc, int* status, cudaStream_t st, const QkvDst& qd, const int* skip,
+                                       const HeadStats& hs) {
   const int tiles_m = (rows_a + BM - 1) / BM, tiles_n = (rows_b + BN - 1) / BN;
   const long long tiles = (long long)tiles_m * tiles_n;
   const unsigned grid = (unsigned)(tiles < 148 ? tiles : 148);
   launch_k(gemm_tc_persist_kernel<BN, HILO, true>, dim3(grid), dim3(THREADS), persist_smem_bytes<BN, HILO, true>(), st, ma, mb, ml,
-           mo, 0, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n, 0);
+           mo, 0, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n, 0, hs, 4 * tiles_m);
   return cudaGetLastError();
 }
 
@@ -1070,6 +1229,8 @@ cudaError_t get_tensor_map(const void* ptr, long long rows, long long cols, long
   return cudaSuccess;
 }
 
+int head_stats_chunks_max(int V) { return 4 * ((V + tc::BM - 1) / tc::BM); }
+
 cudaError_t launch_wait_timeout_probe(long long limit_cycles, int* status, cudaStream_t st) {
   launch_k(tc::wait_timeout_probe_kernel, dim3(1), dim3(tc::THREADS), 0, st, limit_cycles, status);
   return cudaGetLastError();
@@ -1078,9 +1239,18 @@ cudaError_t launch_wait_timeout_probe(long long limit_cycles, int* status, cudaS
 // A: activations [M rows used, capacity a_cap rows, K], W: weights [N, K]; both dense bf16.
 cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_bfloat16* W, const float* bias, int M, int N,
                            int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st, const QkvDst* qkv,
-                           const __nv_bfloat16* A_lo, void* out_lo, const int* skip) {
+                           const __nv_bfloat16* A_lo, void* out_lo, const int* skip, const HeadStats* stats, int* stats_chunks) {
   using namespace tc;
+  if (stats_chunks != nullptr) *stats_chunks = 0;
   if (M <= 0 || N <= 0) return cudaSuccess;
+  // soft-max statistics from the epilogue: fp32 logit stores on a persistent kernel, if the caller's buffer has room
+  auto stats_for = [&](int chunks) -> HeadStats {
+    HeadStats none = {};
+    if (stats == nullptr || stats->partial == nullptr || epi != EPI_STORE_F32 || bias != nullptr || chunks > stats->chunks_capacity)
+      return none;
+    if (stats_chunks != nullptr) *stats_chunks = chunks;
+    return *stats;
+  };
   static std::once_flag once;
   static cudaError_t prep = cudaSuccess;
   std::call_once(once, [] { prep = tc_prepare_gemm(); });
@@ -1121,11 +1291,12 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     {
       const char* pe = getenv("SDD_GEMM_PERSIST");
       if ((pe == nullptr || atoi(pe) != 0) && splits == 1 && (N + BM - 1) / BM > 2 * SMS) {
+        const HeadStats hs = stats_for(4 * ((N + BM - 1) / BM));
         if (bn == 32)
-          return hilo ? launch_persist_swap<32, true>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip)
-                      : launch_persist_swap<32, false>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip);
-        return hilo ? launch_persist_swap<64, true>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip)
-                    : launch_persist_swap<64, false>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip);
+          return hilo ? launch_persist_swap<32, true>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip, hs)
+                      : launch_persist_swap<32, false>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip, hs);
+        return hilo ? launch_persist_swap<64, true>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip, hs)
+                    : launch_persist_swap<64, false>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip, hs);
       }
     }
     if (bn == 32) return launch_hl<32, true>(hilo, ma, mb, ml, none, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
@@ -1199,9 +1370,10 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
   // many 256-wide tiles and no K split: the persistent kernel (SDD_GEMM_PERSIST=0 switches it off)
   static const bool persist_on = [] { const char* e = getenv("SDD_GEMM_PERSIST"); return e == nullptr || atoi(e) != 0; }();
   if (persist_on && bn == 256 && splits == 1 && mt * ((N + 255) / 256) > 2 * SMS) {
+    const HeadStats hs = stats_for((N + 255) / 256);
     if (hilo)
-      return launch_persist<256, true>(ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, skip);
-    return launch_persist<256, false>(ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, skip);
+      return launch_persist<256, true>(ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, skip, hs);
+    return launch_persist<256, false>(ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, skip, hs);
   }
   switch (bn) {
     case 256: return launch_hl<256, false>(hilo, ma, mb, ml, mo, tma_out, M, N, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);

@@ -43,6 +43,17 @@ struct QkvDst {
   int rows_per_seq, mode, d, k_seq_rows, vt_ld;
 };
 
+// Soft-max statistics of the logit rows computed in the epilogue of the tensor-core LM head (persistent kernels), so
+// that no kernel has to read the (gamma + 1) x V logits again for them: per (token row, slice of the vocabulary) one
+// pair (max z, sum exp(z - max)) with z = logit * inv_tau -- greedy (inv_tau == 0): (max logit, index of the first
+// maximum as int bits) -- at partial[row * chunks + slice], the layout the acceptance kernel merges.
+struct HeadStats {
+  float inv_tau;
+  float2* partial;        // null: no statistics
+  int chunks_capacity;    // pairs per row that `partial` has room for
+};
+int head_stats_chunks_max(int V);   // pairs per row the fused statistics may need for a vocabulary of V
+
 // Every kernel of a drafter evaluation takes `skip` (may be null): when *skip != 0 the kernel returns at once.
 
 // ---- vocabulary kernels (sdd_sample.cu) -----------------------------------------------------
@@ -54,8 +65,10 @@ cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float*
                                  int* reveal_step, int batch, int gamma, int V, int k, float inv_tau_q, PhiloxKey key,
                                  RoundState* rs, int cache_skip, cudaStream_t st);
 // round pipeline: logq_in / lseq_in from the draws, partial_q null; stand-alone: logq_in / lseq_in null, partial_q given
+// chunks_p / chunks_q: pairs per row in partial_p / partial_q
 cudaError_t launch_accept(const float* logits_p, const float* q_rows, const int* draft_ids, const float* logq_in,
-                          const float* lseq_in, const float2* partial_p, const float2* partial_q, int rows, int gamma, int V,
+                          const float* lseq_in, const float2* partial_p, int chunks_p, const float2* partial_q, int chunks_q,
+                          int rows, int gamma, int V,
                           float inv_tau_p, float inv_tau_q_rows, PhiloxKey key, uint32_t rnd, RoundState* rs, float* accept_prob,
                           int* n_accept, int* extra_token, int* out_ids, cudaStream_t st);
 cudaError_t launch_commit(int* tokens, int tok_stride, int* ctx_len, int* n_emitted, const int* slot_ids,
@@ -116,7 +129,9 @@ cudaError_t launch_gemm_simt(const T* A, int lda, const T* W, const float* bias,
 cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_bfloat16* W, const float* bias, int M, int N,
                            int K, int epi, void* out, int ldc, int bn_hint, int* status, cudaStream_t st,
                            const QkvDst* qkv = nullptr, const __nv_bfloat16* A_lo = nullptr, void* out_lo = nullptr,
-                           const int* skip = nullptr);
+                           const int* skip = nullptr, const HeadStats* stats = nullptr, int* stats_chunks = nullptr);
+// stats (EPI_STORE_F32 only): where the launch runs on a persistent kernel the epilogue also writes the rows' soft-max
+// statistics and *stats_chunks receives the number of pairs per row (0: not written, the caller runs row_stats)
 
 // one CTA whose bounded waits run out after limit_cycles (see sdd_debug_wait_timeout)
 cudaError_t launch_wait_timeout_probe(long long limit_cycles, int* status, cudaStream_t st);

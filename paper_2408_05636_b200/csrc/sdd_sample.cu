@@ -122,26 +122,33 @@ row_stats_kernel(const float* __restrict__ buf_a, long long rows_a, const float*
   }
 }
 
-// merge the per-chunk pairs of one row: returns the log-sum-exp of z
+// merge the per-chunk pairs of one row, by one warp (lanes stride over the chunks): the log-sum-exp of z, valid in
+// every lane
 __device__ __forceinline__ float merge_partials(const float2* __restrict__ p, int chunks) {
+  const int lane = threadIdx.x & 31;
   float m = -INFINITY;
-  for (int c = 0; c < chunks; ++c) m = fmaxf(m, p[c].x);
+  for (int c = lane; c < chunks; c += 32) m = fmaxf(m, p[c].x);
+  m = warp_max(m);
   float s = 0.f;
-  for (int c = 0; c < chunks; ++c)
-    if (p[c].x > -INFINITY) s += p[c].y * expf(p[c].x - m);
+  for (int c = lane; c < chunks; c += 32) {
+    const float2 v = p[c];
+    if (v.x > -INFINITY) s += v.y * expf(v.x - m);
+  }
+  s = warp_sum(s);
   return m + logf(s);
 }
 __device__ __forceinline__ int merge_partials_argmax(const float2* __restrict__ p, int chunks) {
+  const int lane = threadIdx.x & 31;
   ArgMax a;
   a.s = -INFINITY;
   a.i = 0x7fffffff;
-  for (int c = 0; c < chunks; ++c) {
+  for (int c = lane; c < chunks; c += 32) {
     ArgMax b;
     b.s = p[c].x;
     b.i = __float_as_int(p[c].y);
     if (b.s > -INFINITY) a = argmax_better(a, b);
   }
-  return a.i;
+  return warp_argmax(a).i;
 }
 
 // block-wide arg-max; result valid in thread 0
@@ -384,7 +391,7 @@ constexpr int ACCEPT_THREADS = 256;
 __global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(ACCEPT_THREADS)
 accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_rows, const int* __restrict__ draft_ids,
               const float* __restrict__ logq_in, const float* __restrict__ lseq_in, const float2* __restrict__ partial_p,
-              const float2* __restrict__ partial_q, int chunks, int gamma, int V, float inv_tau_p,
+              int chunks, const float2* __restrict__ partial_q, int chunks_q, int gamma, int V, float inv_tau_p,
               float inv_tau_q_rows, PhiloxKey key, uint32_t rnd_arg, RoundState* __restrict__ rs,
               float* __restrict__ accept_prob, int* __restrict__ n_accept, int* __restrict__ extra_token,
               int* __restrict__ out_ids) {
@@ -406,13 +413,18 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
 
   if (threadIdx.x == 0) s_bad = 0;
   const float2* pp = partial_p + (long long)b * (gamma + 1) * chunks;
-  for (int j = threadIdx.x; j <= gamma; j += ACCEPT_THREADS) {
-    if (greedy) s_lsep[j] = __int_as_float(merge_partials_argmax(pp + (long long)j * chunks, chunks));
-    else s_lsep[j] = merge_partials(pp + (long long)j * chunks, chunks);
+  // one warp per row merges the row's pairs (a few from row_stats_kernel, over a thousand from the LM head's epilogue)
+  for (int j = threadIdx.x >> 5; j <= gamma; j += ACCEPT_THREADS / 32) {
+    const float v = greedy ? __int_as_float(merge_partials_argmax(pp + (long long)j * chunks, chunks))
+                           : merge_partials(pp + (long long)j * chunks, chunks);
+    if ((threadIdx.x & 31) == 0) s_lsep[j] = v;
   }
   if (partial_q != nullptr && !greedy) {
-    const float2* pq = partial_q + (long long)b * gamma * chunks;
-    for (int j = threadIdx.x; j < gamma; j += ACCEPT_THREADS) s_lseq[j] = merge_partials(pq + (long long)j * chunks, chunks);
+    const float2* pq = partial_q + (long long)b * gamma * chunks_q;
+    for (int j = threadIdx.x >> 5; j < gamma; j += ACCEPT_THREADS / 32) {
+      const float v = merge_partials(pq + (long long)j * chunks_q, chunks_q);
+      if ((threadIdx.x & 31) == 0) s_lseq[j] = v;
+    }
   }
   __syncthreads();
 
@@ -642,12 +654,13 @@ cudaError_t launch_ar_sample(const float* logits, int rows_per_seq, int* slot_id
 }
 
 cudaError_t launch_accept(const float* logits_p, const float* q_rows, const int* draft_ids, const float* logq_in,
-                          const float* lseq_in, const float2* partial_p, const float2* partial_q, int rows, int gamma, int V,
+                          const float* lseq_in, const float2* partial_p, int chunks_p, const float2* partial_q, int chunks_q,
+                          int rows, int gamma, int V,
                           float inv_tau_p, float inv_tau_q_rows, PhiloxKey key, uint32_t rnd, RoundState* rs, float* accept_prob,
                           int* n_accept, int* extra_token, int* out_ids, cudaStream_t st) {
   const size_t smem = (size_t)(2 * gamma + 1) * sizeof(float);
-  launch_k(accept_kernel, dim3(VC * rows), dim3(ACCEPT_THREADS), smem, st, logits_p, q_rows, draft_ids, logq_in, lseq_in, partial_p, partial_q,
-                                                    stats_chunks(V), gamma, V, inv_tau_p, inv_tau_q_rows, key, rnd, rs,
+  launch_k(accept_kernel, dim3(VC * rows), dim3(ACCEPT_THREADS), smem, st, logits_p, q_rows, draft_ids, logq_in, lseq_in, partial_p,
+                                                    chunks_p, partial_q, chunks_q, gamma, V, inv_tau_p, inv_tau_q_rows, key, rnd, rs,
                                                     accept_prob, n_accept, extra_token, out_ids);
   return cudaGetLastError();
 }
