@@ -577,6 +577,15 @@ def run_ours(args):
                  "peak_source": f"of {peaks['source']} (burst)"}
     roofline["accept"] = accept_roof
     roofline["gemm"] = gemm_roof
+    # what the acceptance step of a round reads, next to the size of the target's logit matrix: the soft-max statistics
+    # come out of the LM head's epilogue (one pair per row and 32-row slice of the vocabulary), so the acceptance kernel
+    # reads those pairs, gamma target logits at the draft ids, and the target and draft rows of the first rejection twice
+    pairs = 4 * ((V + 127) // 128)
+    roofline["accept_path_in_round"] = {
+        "bytes_read_per_round": (wl.gamma + 1) * pairs * 8 + 4 * V * 4 + wl.gamma * 4,
+        "logit_matrix_bytes": (wl.gamma + 1) * V * 4,
+        "row_stats_launches_per_round": round(kernels["row_stats"]["launches"] / prof_rounds, 2) if "row_stats" in kernels else 0,
+        "note": "the logit matrix is written once by the LM head and never read in full"}
 
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -17,7 +17,8 @@
 // PIPE variant (grids of at most one CTA per SM, where a CTA's chain of key tiles is what bounds the launch): S is
 // double-buffered in TMEM (512 columns, one CTA per SM) and the K / V^T ring has three stages, so S(t+1) = Q K(t+1)^T is
 // issued before the MMA thread waits for P(t) and is complete when the soft-max warps get to it; a tile's chain is then
-// soft-max -> next soft-max instead of S -> soft-max -> P V -> S.
+// soft-max -> next soft-max instead of S -> soft-max -> P V -> S.  The second half of P has two buffers there (the
+// first half lies over the tile's own K stage), so P(t+1) is written while P(t) V(t) may still be running.
 // Waits are bounded exactly as in the GEMM kernel.
 #include <cstdlib>
 #include <mutex>
@@ -37,9 +38,11 @@ constexpr int AT_K_BYTES = 128 * 64 * 2;            // 16 KB
 constexpr int AT_VT_BYTES = 2 * 64 * 64 * 2;        // two boxes [64 d_head rows x 64 keys]: 16 KB
 constexpr int AT_STAGE_BYTES = AT_K_BYTES + AT_VT_BYTES;
 // PIPE = false: two K / V^T stages, 96 KB, two CTAs per SM; TMEM: S in columns 0..127, PV accumulators 128..191 and 192..255
-// PIPE = true : three stages, 128 KB, one CTA per SM; TMEM: S buffers 0..127 and 128..255, PV accumulators 256..319 and 320..383
+// PIPE = true : three stages and two buffers for the second half of P, 144 KB, one CTA per SM; TMEM: S buffers 0..127 and
+//               128..255, PV accumulators 256..319 and 320..383
 template <bool PIPE> constexpr int at_stages() { return PIPE ? 3 : 2; }
-template <bool PIPE> constexpr int at_bar_off() { return AT_Q_BYTES + AT_P_BYTES + at_stages<PIPE>() * AT_STAGE_BYTES; }
+template <bool PIPE> constexpr int at_p_bytes() { return (PIPE ? 2 : 1) * AT_P_BYTES; }   // PIPE: P k-block 1 double-buffered
+template <bool PIPE> constexpr int at_bar_off() { return AT_Q_BYTES + at_p_bytes<PIPE>() + at_stages<PIPE>() * AT_STAGE_BYTES; }
 template <bool PIPE> constexpr int at_smem() { return at_bar_off<PIPE>() + 1024 + 128 + 3 * 1024; }   // barriers, then the soft-max exchange arrays
 template <bool PIPE> constexpr uint32_t at_tmem_cols() { return PIPE ? 512u : 256u; }
 template <bool PIPE> constexpr uint32_t at_acc_col() { return PIPE ? 256u : 128u; }
@@ -89,45 +92,35 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   constexpr int AT_RECV_OFF = at_recv_off<PIPE>();
   constexpr uint32_t AT_TMEM_COLS = at_tmem_cols<PIPE>();
   constexpr uint32_t ACC_COL = at_acc_col<PIPE>();
+  constexpr int P_TOTAL = at_p_bytes<PIPE>();
   const int kv_split = prm.kv_split, kv_rank = (int)blockIdx.x % kv_split;   // cluster = kv_split consecutive CTAs in x
   const int qt = (int)blockIdx.x / kv_split, h = blockIdx.y, b = blockIdx.z;
-  pdl_wait();   // ctx_len and Q / K / V^T come from earlier kernels
-  pdl_launch_dependents();
-  if (prm.skip != nullptr && *prm.skip) return;
-  const int c = prm.ctx_len[b];
-  const int q0 = qt * 128;
-  int n_valid_q;
-  if (prm.mode == 0) n_valid_q = c + prm.gamma;
-  else if (prm.mode == 1) n_valid_q = prm.q_rows_per_seq;
-  else n_valid_q = c - 1;
-  if (n_valid_q > prm.q_rows_per_seq) n_valid_q = prm.q_rows_per_seq;
-  if (q0 >= n_valid_q) return;                       // padding tile (uniform for the CTA)
-  const int last_valid = (n_valid_q < q0 + 128 ? n_valid_q : q0 + 128) - 1;
-  int n_keys_cta;
-  if (prm.mode == 0) n_keys_cta = c + prm.gamma;
-  else if (prm.mode == 1) n_keys_cta = c - 1 + last_valid + 1;
-  else n_keys_cta = last_valid + 1;
-  if (n_keys_cta > prm.k_rows_per_seq) n_keys_cta = prm.k_rows_per_seq;
-  const int num_kt = (n_keys_cta + 127) / 128;
-  const int my_kt = kv_rank < num_kt ? (num_kt - kv_rank + kv_split - 1) / kv_split : 0;   // key tiles of this CTA
 
+  // set-up that touches only shared and tensor memory comes first: it runs under the tail of the kernel ahead
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t sQ = base, sP = base + AT_Q_BYTES;
-  auto sK = [&](int s) { return base + AT_Q_BYTES + AT_P_BYTES + s * AT_STAGE_BYTES; };
+  const uint32_t sQ = base;
+  auto sP = [&](int t) { return base + AT_Q_BYTES + (PIPE ? (uint32_t)(t & 1) * AT_P_BYTES : 0u); };   // P k-block 1 of tile t
+  auto sK = [&](int s) { return base + AT_Q_BYTES + P_TOTAL + s * AT_STAGE_BYTES; };
   auto sVT = [&](int s) { return sK(s) + AT_K_BYTES; };
   const uint32_t bars = base + AT_BAR_OFF;
-  const uint32_t q_full = bars, p_ready = bars + 8, pv_full = bars + 16;
-  auto s_full = [&](int b) { return bars + 24 + 8u * b; };            // one per S buffer (PIPE: two, else only [0])
-  auto kv_full = [&](int s) { return bars + 40 + 8u * s; };
-  auto kv_empty = [&](int s) { return bars + 64 + 8u * s; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + AT_BAR_OFF + 96);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + AT_BAR_OFF + 104);
+  // PIPE keeps one barrier per parity of the tile for "P written", "P V done" and "S done": a soft-max warp may be one
+  // tile ahead of the slowest one there (S(t+1) is complete before the last warp has finished tile t), so its arrivals
+  // for tile t + 1 must not be counted with those still missing for tile t; !PIPE uses only the barriers [0]
+  const uint32_t q_full = bars;
+  auto p_ready = [&](int i) { return bars + 8 + 8u * i; };
+  auto pv_full = [&](int i) { return bars + 24 + 8u * i; };
+  auto s_full = [&](int i) { return bars + 40 + 8u * i; };
+  auto kv_full = [&](int s) { return bars + 56 + 8u * s; };
+  auto kv_empty = [&](int s) { return bars + 80 + 8u * s; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + AT_BAR_OFF + 104);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + AT_BAR_OFF + 112);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    mbar_init(q_full, 1); mbar_init(s_full(0), 1); mbar_init(s_full(1), 1); mbar_init(p_ready, 256); mbar_init(pv_full, 1);
+    mbar_init(q_full, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(p_ready(i), 256); mbar_init(pv_full(i), 1); mbar_init(s_full(i), 1); }
     for (int s = 0; s < AT_KV_STAGES; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -138,7 +131,34 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0) {
+  pdl_wait();   // ctx_len and Q / K / V^T come from earlier kernels
+  pdl_launch_dependents();
+  // a skipped drafter evaluation, or a tile of padding rows only: nothing to do (uniform over the CTA and its cluster)
+  bool active = !(prm.skip != nullptr && *prm.skip);
+  const int c = active ? prm.ctx_len[b] : 1;
+  const int q0 = qt * 128;
+  int n_valid_q;
+  if (prm.mode == 0) n_valid_q = c + prm.gamma;
+  else if (prm.mode == 1) n_valid_q = prm.q_rows_per_seq;
+  else n_valid_q = c - 1;
+  if (n_valid_q > prm.q_rows_per_seq) n_valid_q = prm.q_rows_per_seq;
+  if (q0 >= n_valid_q) active = false;
+  const int last_valid = (n_valid_q < q0 + 128 ? n_valid_q : q0 + 128) - 1;
+  int n_keys_cta;
+  if (prm.mode == 0) n_keys_cta = c + prm.gamma;
+  else if (prm.mode == 1) n_keys_cta = c - 1 + last_valid + 1;
+  else n_keys_cta = last_valid + 1;
+  if (n_keys_cta > prm.k_rows_per_seq) n_keys_cta = prm.k_rows_per_seq;
+  const int num_kt = active ? (n_keys_cta + 127) / 128 : 0;
+  const int my_kt = kv_rank < num_kt ? (num_kt - kv_rank + kv_split - 1) / kv_split : 0;   // key tiles of this CTA
+  // completion of P(t) V(t): PIPE keeps one barrier per parity of t, so that a wait for tile t - 2 cannot be taken for
+  // one on a phase still to come
+  auto wait_pv = [&](int t) {
+    return mbar_wait(pv_full(PIPE ? (t & 1) : 0), (uint32_t)(PIPE ? (t >> 1) : t) & 1u, abort_flag, prm.status);
+  };
+
+  if (!active) {
+  } else if (warp == 0) {
     if (lane == 0 && my_kt > 0) {
       mbar_expect_tx(q_full, AT_Q_BYTES);
       tma_load_2d(sQ, &map_q, q_full, prm.q_col0 + h * AT_DH, b * prm.q_rows_per_seq + q0);
@@ -192,20 +212,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           ok = issue_s(t);
         }
         if (!ok) break;
-        ok = mbar_wait(p_ready, (uint32_t)t & 1u, abort_flag, prm.status);
+        ok = mbar_wait(p_ready(PIPE ? (t & 1) : 0), (uint32_t)(PIPE ? (t >> 1) : t) & 1u, abort_flag, prm.status);
         if (!ok) break;
         fence_after_sync();
         // one accumulator per half of the key tile (keys 0..63 and keys 64..127 of the tile); both add up over the
         // CTA's tiles in TMEM
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb) {
-          const uint64_t dp = make_smem_desc(kb == 0 ? sK(s) : sP);
+          const uint64_t dp = make_smem_desc(kb == 0 ? sK(s) : sP(t));
           const uint64_t dv = make_smem_desc(sVT(s) + kb * (64 * 64 * 2));
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             umma(tmem_base + ACC_COL + (uint32_t)(kb * 64), dp + 2u * k, dv + 2u * k, idesc_pv, (t | k) ? 1u : 0u);
         }
-        umma_commit(pv_full);
+        umma_commit(pv_full(PIPE ? (t & 1) : 0));
         umma_commit(kv_empty(s));
       }
     }
@@ -246,7 +266,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const int key0 = t * 128 + hf * 64;
       const uint32_t t_s = t_lane + (PIPE ? (uint32_t)(it & 1) * 128u : 0u);    // this tile's S buffer
       // this thread's 64 probabilities are one row of a P k-block: block 0 lies over the stage's (consumed) K tile
-      uint8_t* p_row = gbase + (hf == 0 ? AT_Q_BYTES + AT_P_BYTES + (it % AT_KV_STAGES) * AT_STAGE_BYTES : AT_Q_BYTES) + r * 128;
+      uint8_t* p_row = gbase + (hf == 0 ? AT_Q_BYTES + P_TOTAL + (it % AT_KV_STAGES) * AT_STAGE_BYTES
+                                        : AT_Q_BYTES + (PIPE ? (it & 1) * AT_P_BYTES : 0)) + r * 128;
       // tcgen05.ld / st are warp-collective: every branch around them is taken by whole warps
       const bool full_w = __all_sync(0xffffffffu, key0 + 64 <= key_limit);
       // !PIPE: the 64 scores are read twice from TMEM (once for the maximum, once for the exponentials) instead of being
@@ -281,7 +302,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const float m_new = fmaxf(m, mx);
         const float corr = (m == -INFINITY || m_new == -INFINITY) ? 0.f : ex2(m - m_new);
         if (it > 0) {
-          ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)(it - 1) & 1u, abort_flag, prm.status));
+          ok = __all_sync(0xffffffffu, wait_pv(it - 1));
           if (!ok) break;
           fence_after_sync();
 #pragma unroll
@@ -295,9 +316,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         l *= corr;
         m = m_new;
       }
-      // P(t) may overwrite P(t-1) once PV(t-1) has read it (long done by now)
-      if (it > 0) {
-        ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)(it - 1) & 1u, abort_flag, prm.status));
+      // P(t) overwrites the buffer of P(t-1) (PIPE: of P(t-2)) once that tile's P V has read it
+      if (it >= (PIPE ? 2 : 1)) {
+        ok = __all_sync(0xffffffffu, wait_pv(it - (PIPE ? 2 : 1)));
         if (!ok) break;
       }
       const float m_use = m == -INFINITY ? 0.f : m;
@@ -335,9 +356,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       fence_before_sync();          // accumulator reads / writes above are ordered before the MMA that follows the arrive
       fence_async_smem();
-      mbar_arrive(p_ready);
+      mbar_arrive(p_ready(PIPE ? (it & 1) : 0));
     }
-    if (ok && my_kt > 0) ok = __all_sync(0xffffffffu, mbar_wait(pv_full, (uint32_t)(my_kt - 1) & 1u, abort_flag, prm.status));
+    if (ok && my_kt > 0) ok = __all_sync(0xffffffffu, wait_pv(my_kt - 1));
     ok = named_bar_and(1, 256, ok);
     float o[AT_DH / 2];                                // this thread's 32 output columns (unnormalised)
 #pragma unroll

@@ -77,7 +77,7 @@ cudaError_t launch_commit(int* tokens, int tok_stride, int* ctx_len, int* n_emit
 // draw of slot j from the last of the rows_per_seq logit rows per sequence (autoregressive drafter)
 cudaError_t launch_ar_sample(const float* logits, int rows_per_seq, int* slot_ids, float* q_logits, float* logq, float* lseq,
                              int* reveal_step, int batch, int gamma, int j, int V, float inv_tau_q, PhiloxKey key,
-                             const RoundState* rs, cudaStream_t st);
+                             RoundState* rs, cudaStream_t st);
 cudaError_t launch_reset_slots(int* slot_ids, int* reveal_step, int n, int mask_id, RoundState* rs, cudaStream_t st);
 
 // ---- glue (sdd_glue.cu) ---------------------------------------------------------------------

@@ -263,7 +263,7 @@ constexpr int SAMPLE_THREADS = 512;
 __device__ __forceinline__ void draw_slot(const float* __restrict__ src, float* __restrict__ dst, int* __restrict__ slot_out,
                                           float* __restrict__ logq_out, float* __restrict__ lseq_out,
                                           int* __restrict__ reveal_out, int j, int b, int V,
-                                          int mark, float inv_tau_q, PhiloxKey key, uint32_t rnd) {
+                                          int mark, float inv_tau_q, PhiloxKey key, uint32_t rnd, int* __restrict__ status) {
   cg::cluster_group cl = cg::this_cluster();
   const int rank = (int)cl.block_rank();
   const bool greedy = inv_tau_q == 0.f;
@@ -306,8 +306,12 @@ __device__ __forceinline__ void draw_slot(const float* __restrict__ src, float* 
   }
   cl.sync();
   if (rank == 0 && threadIdx.x == 0) {
-    const ArgMax win = cluster_merge_argmax(cl, &part, false);
+    ArgMax win = cluster_merge_argmax(cl, &part, false);
     const float lse = greedy ? 0.f : cluster_merge_lse(cl, &part);
+    if ((unsigned)win.i >= (unsigned)V) {   // no entry compared greater than -inf: the logits are not numbers
+      win.i = 0;
+      if (status != nullptr) atomicCAS(status, DEV_OK, DEV_BAD_TOKEN);
+    }
     *slot_out = win.i;
     *logq_out = greedy ? 0.f : src[win.i] * inv_tau_q - lse;
     *lseq_out = lse;               // the stored row's log-sum-exp: the residual draw of the acceptance step needs it
@@ -322,7 +326,7 @@ __device__ __forceinline__ bool unmask_sample_row(const float* __restrict__ step
                      float* __restrict__ logq,               // [B, gamma]
                      float* __restrict__ lseq,               // [B, gamma]
                      int* __restrict__ reveal_step,          // [B, gamma]
-                     int gamma, int V, int k, float inv_tau_q, PhiloxKey key, const RoundState* __restrict__ rs) {
+                     int gamma, int V, int k, float inv_tau_q, PhiloxKey key, RoundState* __restrict__ rs) {
   const int j = blockIdx.x / VC, b = blockIdx.y;
   const uint32_t rnd = rs->round;
   const long long row = (long long)b * gamma + j;
@@ -333,7 +337,7 @@ __device__ __forceinline__ bool unmask_sample_row(const float* __restrict__ step
   const uint32_t m_odd = ((wu >> 9) << 1) | 1u;
   if (!(m_odd * (uint32_t)k < (1u << 24))) return false;
   draw_slot(step_logits + row * V, q_logits + row * V, slot_ids + row, logq + row, lseq + row, reveal_step + row, j, b, V, k,
-            inv_tau_q, key, rnd);
+            inv_tau_q, key, rnd, &rs->status);
   return true;
 }
 
@@ -368,13 +372,13 @@ unmask_sample_kernel(const float* __restrict__ step_logits, int* __restrict__ sl
 __global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(SAMPLE_THREADS)
 ar_sample_kernel(const float* __restrict__ logits, int rows_per_seq, int* __restrict__ slot_ids, float* __restrict__ q_logits,
                  float* __restrict__ logq, float* __restrict__ lseq, int* __restrict__ reveal_step, int gamma, int j, int V,
-                 float inv_tau_q, PhiloxKey key, const RoundState* __restrict__ rs) {
+                 float inv_tau_q, PhiloxKey key, RoundState* __restrict__ rs) {
   pdl_wait();
   pdl_launch_dependents();
   const int b = blockIdx.y;
   const long long row = (long long)b * gamma + j;
   draw_slot(logits + ((long long)b * rows_per_seq + rows_per_seq - 1) * V, q_logits + row * V, slot_ids + row, logq + row,
-            lseq + row, reveal_step + row, j, b, V, gamma - j, inv_tau_q, key, rs->round);
+            lseq + row, reveal_step + row, j, b, V, gamma - j, inv_tau_q, key, rs->round, &rs->status);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -540,7 +544,11 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
       if (win.i == 0x7fffffff) win = cluster_merge_argmax(cl, &part, true);
       t = win.i;
     }
-    const bool bad = s_bad != 0;
+    bool bad = s_bad != 0;
+    if ((unsigned)t >= (unsigned)V) {   // no entry compared greater than -inf: the logits are not numbers
+      t = 0;
+      bad = true;
+    }
     if (bad && rs != nullptr) atomicCAS(&rs->status, DEV_OK, DEV_BAD_TOKEN);
     n_accept[b] = bad ? -1 : n;
     if (extra_token != nullptr) extra_token[b] = t;
@@ -647,7 +655,7 @@ cudaError_t launch_unmask_sample(const float* step_logits, int* slot_ids, float*
 
 cudaError_t launch_ar_sample(const float* logits, int rows_per_seq, int* slot_ids, float* q_logits, float* logq, float* lseq,
                              int* reveal_step, int batch, int gamma, int j, int V, float inv_tau_q, PhiloxKey key,
-                             const RoundState* rs, cudaStream_t st) {
+                             RoundState* rs, cudaStream_t st) {
   launch_k(ar_sample_kernel, dim3(VC, batch), dim3(SAMPLE_THREADS), 0, st, logits, rows_per_seq, slot_ids, q_logits, logq, lseq,
            reveal_step, gamma, j, V, inv_tau_q, key, rs);
   return cudaGetLastError();

@@ -18,9 +18,11 @@ def _ref(q, k, v, causal_from=None):
     return o.transpose(0, 1)
 
 
-# the last case: many CTAs (several waves), sequences whose last key tile is full or ragged
+# the fourth case: many CTAs (several waves), sequences whose last key tile is full or ragged; the last two: grids of at
+# most one CTA per SM with long chains of key tiles (the pipelined variant: 8, 9 and 7 tiles per CTA)
 @pytest.mark.parametrize("H,lens,gamma,lcap", [(2, [100], 16, 128), (3, [250, 37, 511], 16, 640), (12, [300], 32, 384),
-                                                (16, [700, 130, 250, 1000, 496, 129], 16, 1024)])
+                                                (16, [700, 130, 250, 1000, 496, 129], 16, 1024),
+                                                (4, [1000, 1100], 32, 1152), (16, [850], 32, 896)])
 def test_drafter_mode(H, lens, gamma, lcap):
     import paper_2408_05636_b200 as sdd
     B, d = len(lens), H * 64
@@ -45,10 +47,11 @@ def test_drafter_mode(H, lens, gamma, lcap):
         assert torch.all(out[b * lcap + L: (b + 1) * lcap] == 9.0)      # padding rows untouched
 
 
-@pytest.mark.parametrize("mode,lens,rows", [(1, [40, 300], 17), (1, [1, 129], 33), (2, [200, 50], 199), (2, [2], 1)])
+@pytest.mark.parametrize("mode,lens,rows", [(1, [40, 300], 17), (1, [1, 129], 33), (2, [200, 50], 199), (2, [2], 1),
+                                            (1, [1000, 650], 33), (2, [1100], 1099)])
 def test_target_modes(mode, lens, rows):
     import paper_2408_05636_b200 as sdd
-    H, n_ctx, gamma = 4, 512, rows - 1
+    H, n_ctx, gamma = 4, (512 if max(lens) + rows <= 512 else 1280), rows - 1
     B, d = len(lens), H * 64
     g = torch.Generator(device="cuda").manual_seed(17 * mode + rows)
     qkv = torch.randn(B * rows + 200, 3 * d, device="cuda", generator=g).to(torch.bfloat16)

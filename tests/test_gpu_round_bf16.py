@@ -191,3 +191,18 @@ def test_tiny_bf16_rounds_every_stage():
     print("near-ties:", log, "max logit err q/p:", stats["max_q_err"], stats["max_p_err"])
     parity.assert_few(log)
     s.close()
+
+
+def test_small_bf16_batch8_greedy_round():
+    """Temperature 0 with 136 target rows: the LM head then runs in the token-major orientation on the persistent kernel,
+    whose epilogue hands the acceptance step each row's arg-max (statistics fused into the LM head).  One round, T = 2,
+    two of the eight sequences followed by the oracle."""
+    import paper_2408_05636_b200 as sdd
+    wl = synth.scaled_workload(synth.WORKLOADS["small_bf16"], batch=8, T=2)
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 8, 150, wl.prompt_seed)
+    plen = [150, 64, 131, 77, 150, 99, 140, 128]
+    s = sdd.Session(dp, dq, prompts, plen, wl.gamma, 2, 40, 0.0, 0.0, wl.philox_seed)
+    log, stats = roundcheck.check_rounds(s, mp, mq, wl, 1, 0.0, 0.0, TOL, seqs=[0, 7])
+    assert not log
+    s.close()
