@@ -578,9 +578,9 @@ def run_ours(args):
     roofline["accept"] = accept_roof
     roofline["gemm"] = gemm_roof
     # what the acceptance step of a round reads, next to the size of the target's logit matrix: the soft-max statistics
-    # come out of the LM head's epilogue (one pair per row and 32-row slice of the vocabulary), so the acceptance kernel
+    # come out of the LM head's epilogue (one pair per row and 128-row slice of the vocabulary), so the acceptance kernel
     # reads those pairs, gamma target logits at the draft ids, and the target and draft rows of the first rejection twice
-    pairs = 4 * ((V + 127) // 128)
+    pairs = (V + 127) // 128
     roofline["accept_path_in_round"] = {
         "bytes_read_per_round": (wl.gamma + 1) * pairs * 8 + 4 * V * 4 + wl.gamma * 4,
         "logit_matrix_bytes": (wl.gamma + 1) * V * 4,

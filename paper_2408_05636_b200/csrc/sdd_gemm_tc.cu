@@ -404,19 +404,21 @@ __device__ __forceinline__ void warp_reduce_scatter_argmax(float (&a)[32], int (
 }
 
 // SWAP orientation (tile = 128 vocabulary rows x up to BN tokens; a thread owns one vocabulary row r): out[token][r]
-// = logit, and per warp one pair per token over the warp's 32 vocabulary rows: slice index = tile * 4 + q.
+// = logit.  Each warp reduces its 32 vocabulary rows per token with shuffles; the four warps' pairs meet in shared
+// memory (`ex`: [BN / 32][4][32] float2, free between two tiles' epilogues because the four warps pass a common
+// barrier before every tile) and warp 0 writes one pair per (token, tile): slice index = tile.
 template <int BN>
 __device__ __forceinline__ void epilogue_head_swap(uint32_t tmem_acc, int m0, int q, int lane, int V, int tokens,
                                                    float* __restrict__ out, int ldc, const HeadStats& hs, int chunks,
-                                                   int tile) {
+                                                   int tile, float2* ex) {
   const int r = m0 + q * 32 + lane;
   const bool r_ok = r < V;
   const bool greedy = hs.inv_tau == 0.f;
   const float k = hs.inv_tau * 1.4426950408889634f;
+  const int n_cc = (tokens + 31) / 32 < BN / 32 ? (tokens + 31) / 32 : BN / 32;
 #pragma unroll 1
-  for (int cc = 0; cc < BN / 32; ++cc) {
+  for (int cc = 0; cc < n_cc; ++cc) {
     const int c0 = cc * 32;
-    if (c0 >= tokens) break;
     uint32_t v[32];
     tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
     float x[32];
@@ -445,9 +447,41 @@ __device__ __forceinline__ void epilogue_head_swap(uint32_t tmem_acc, int m0, in
         x[j] = (r_ok && mj > -INFINITY) ? exp2f((x[j] - mj) * k) : 0.f;
       }
       warp_reduce_scatter(x, lane, [](float a, float b) { return a + b; });
-      pair = make_float2(m_mine * hs.inv_tau, x[0]);
+      pair = make_float2(m_mine, x[0]);                // (max logit, sum exp((logit - max) * inv_tau))
     }
-    if (c0 + lane < tokens) hs.partial[(long long)(c0 + lane) * chunks + tile * 4 + q] = pair;
+    ex[(cc * 4 + q) * 32 + lane] = pair;
+  }
+  named_bar_sync(2, 128);
+  if (q == 0) {
+    for (int cc = 0; cc < n_cc; ++cc) {
+      const int tok = cc * 32 + lane;
+      if (tok >= tokens) break;
+      float2 a = ex[(cc * 4 + 0) * 32 + lane];
+      if (greedy) {
+        ArgMax best;
+        best.s = a.x; best.i = __float_as_int(a.y);
+#pragma unroll
+        for (int w = 1; w < 4; ++w) {
+          const float2 b = ex[(cc * 4 + w) * 32 + lane];
+          ArgMax o;
+          o.s = b.x; o.i = __float_as_int(b.y);
+          best = argmax_better(best, o);
+        }
+        a = make_float2(best.s, __int_as_float(best.i));
+      } else {
+        float m = a.x;
+#pragma unroll
+        for (int w = 1; w < 4; ++w) m = fmaxf(m, ex[(cc * 4 + w) * 32 + lane].x);
+        float sum = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const float2 b = ex[(cc * 4 + w) * 32 + lane];
+          if (b.x > -INFINITY) sum += b.y * exp2f((b.x - m) * k);
+        }
+        a = make_float2(m * hs.inv_tau, sum);
+      }
+      hs.partial[(long long)tok * chunks + tile] = a;
+    }
   }
 }
 
@@ -697,7 +731,9 @@ constexpr int persist_smem_bytes() {
   return persist_stages<BN, HILO, SWAP>() * stage_bytes<BN, SWAP, HILO>() + 2 * 128 * 128 + 1024 + 512 + 2048;
 }
 
-template <int BN, bool HILO, bool SWAP = false>
+// STATS: the LM-head instantiations whose epilogue also writes the rows' soft-max statistics (HeadStats); kept apart so
+// that the other launches do not carry that code
+template <int BN, bool HILO, bool SWAP = false, bool STATS = false>
 __global__ void __launch_bounds__(THREADS)
 gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                        const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ OutMaps maps_out, int tma_out,
@@ -846,12 +882,13 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       if (!ready) break;
       fence_after_sync();
       const uint32_t acc = tmem_base + (uint32_t)(buf * BN);
-      if (SWAP && hs.partial != nullptr)        // LM head: logits + their soft-max statistics
-        epilogue_head_swap<BN>(acc, m0, q, lane, rows_a, rows_b, reinterpret_cast<float*>(out), ldc, hs, hs_chunks, m0 / BM);
+      if constexpr (STATS && SWAP)       // LM head: logits + their soft-max statistics (the staging buffers are free here)
+        epilogue_head_swap<BN>(acc, m0, q, lane, rows_a, rows_b, reinterpret_cast<float*>(out), ldc, hs, hs_chunks, m0 / BM,
+                               reinterpret_cast<float2*>(generic_base + STAGING_OFF));
+      else if constexpr (STATS)
+        epilogue_head_normal<BN>(acc, m0, n0, q, lane, rows_a, rows_b, reinterpret_cast<float*>(out), ldc, hs, hs_chunks, n0 / BN);
       else if (SWAP)
         epilogue_manual<BN, true>(acc, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, false, qd);
-      else if (hs.partial != nullptr)
-        epilogue_head_normal<BN>(acc, m0, n0, q, lane, rows_a, rows_b, reinterpret_cast<float*>(out), ldc, hs, hs_chunks, n0 / BN);
       else if (use_tma)
         epilogue_tma<BN>(acc, m0, n0, q, lane, epi == EPI_QKV ? (int)EPI_STORE : epi, bias_s, &maps_out.out,
                          generic_base + STAGING_OFF, base + STAGING_OFF, n_store);
@@ -1128,9 +1165,13 @@ static cudaError_t launch_persist(const CUtensorMap& ma, const CUtensorMap& mb, 
   const int tiles_m = (rows_a + BM - 1) / BM, tiles_n = (rows_b + BN - 1) / BN;
   const long long tiles = (long long)tiles_m * tiles_n;
   const unsigned grid = (unsigned)(tiles < 148 ? tiles : 148);
-  launch_k(gemm_tc_persist_kernel<BN, HILO>, dim3(grid), dim3(THREADS), persist_smem_bytes<BN, HILO>(), st, ma, mb, ml, mo,
-           tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n,
-           (long long)rows_b * K * 2 <= (48ll << 20) ? 1 : 0, hs, tiles_n);
+  const int n_fastest = (long long)rows_b * K * 2 <= (48ll << 20) ? 1 : 0;
+  if (hs.partial != nullptr)
+    launch_k(gemm_tc_persist_kernel<BN, HILO, false, true>, dim3(grid), dim3(THREADS), persist_smem_bytes<BN, HILO>(), st, ma, mb, ml, mo,
+             tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n, n_fastest, hs, tiles_n);
+  else
+    launch_k(gemm_tc_persist_kernel<BN, HILO>, dim3(grid), dim3(THREADS), persist_smem_bytes<BN, HILO>(), st, ma, mb, ml, mo,
+             tma_out, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n, n_fastest, hs, tiles_n);
   return cudaGetLastError();
 }
 
@@ -1142,8 +1183,12 @@ static cudaError_t launch_persist_swap(const CUtensorMap& ma, const CUtensorMap&
   const int tiles_m = (rows_a + BM - 1) / BM, tiles_n = (rows_b + BN - 1) / BN;
   const long long tiles = (long long)tiles_m * tiles_n;
   const unsigned grid = (unsigned)(tiles < 148 ? tiles : 148);
-  launch_k(gemm_tc_persist_kernel<BN, HILO, true>, dim3(grid), dim3(THREADS), persist_smem_bytes<BN, HILO, true>(), st, ma, mb, ml,
-           mo, 0, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n, 0, hs, 4 * tiles_m);
+  if (hs.partial != nullptr)
+    launch_k(gemm_tc_persist_kernel<BN, HILO, true, true>, dim3(grid), dim3(THREADS), persist_smem_bytes<BN, HILO, true>(), st, ma, mb,
+             ml, mo, 0, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n, 0, hs, tiles_m);
+  else
+    launch_k(gemm_tc_persist_kernel<BN, HILO, true>, dim3(grid), dim3(THREADS), persist_smem_bytes<BN, HILO, true>(), st, ma, mb, ml,
+             mo, 0, rows_a, rows_b, K, epi, bias, out, out_lo, ldc, status, qd, skip, tiles_m, tiles_n, 0, hs, tiles_m);
   return cudaGetLastError();
 }
 
@@ -1185,8 +1230,14 @@ cudaError_t tc_prepare_gemm() {
                                 persist_smem_bytes<256, false>())) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(gemm_tc_persist_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 persist_smem_bytes<256, true>())) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_persist_kernel<256, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                persist_smem_bytes<256, false>())) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(gemm_tc_persist_kernel<256, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                persist_smem_bytes<256, true>())) != cudaSuccess) return e;
 #define SDD_PREP_PS(BN_, HL_)                                                                                              \
   if ((e = cudaFuncSetAttribute(gemm_tc_persist_kernel<BN_, HL_, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
+                                persist_smem_bytes<BN_, HL_, true>())) != cudaSuccess) return e;                            \
+  if ((e = cudaFuncSetAttribute(gemm_tc_persist_kernel<BN_, HL_, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
                                 persist_smem_bytes<BN_, HL_, true>())) != cudaSuccess) return e;
   SDD_PREP_PS(32, false) SDD_PREP_PS(32, true) SDD_PREP_PS(64, false) SDD_PREP_PS(64, true)
 #undef SDD_PREP_PS
@@ -1229,7 +1280,7 @@ cudaError_t get_tensor_map(const void* ptr, long long rows, long long cols, long
   return cudaSuccess;
 }
 
-int head_stats_chunks_max(int V) { return 4 * ((V + tc::BM - 1) / tc::BM); }
+int head_stats_chunks_max(int V) { return (V + tc::BM - 1) / tc::BM; }
 
 cudaError_t launch_wait_timeout_probe(long long limit_cycles, int* status, cudaStream_t st) {
   launch_k(tc::wait_timeout_probe_kernel, dim3(1), dim3(tc::THREADS), 0, st, limit_cycles, status);
@@ -1291,7 +1342,7 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     {
       const char* pe = getenv("SDD_GEMM_PERSIST");
       if ((pe == nullptr || atoi(pe) != 0) && splits == 1 && (N + BM - 1) / BM > 2 * SMS) {
-        const HeadStats hs = stats_for(4 * ((N + BM - 1) / BM));
+        const HeadStats hs = stats_for((N + BM - 1) / BM);
         if (bn == 32)
           return hilo ? launch_persist_swap<32, true>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip, hs)
                       : launch_persist_swap<32, false>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip, hs);
