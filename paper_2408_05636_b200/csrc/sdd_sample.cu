@@ -122,34 +122,46 @@ row_stats_kernel(const float* __restrict__ buf_a, long long rows_a, const float*
   }
 }
 
-// merge the per-chunk pairs of one row, by one warp (lanes stride over the chunks): the log-sum-exp of z, valid in
-// every lane
-__device__ __forceinline__ float merge_partials(const float2* __restrict__ p, int chunks) {
-  const int lane = threadIdx.x & 31;
+// Merge of the per-chunk pairs of one row by a group of `tpr` consecutive lanes (a power of two up to 32; `sub` = the
+// lane's index in its group): the log-sum-exp of z, valid in every lane of the group.  All 32 lanes of the warp call it
+// together (the shuffles are warp-wide); a group whose row does not exist passes valid = false.
+__device__ __forceinline__ float merge_partials(const float2* __restrict__ p, int chunks, int tpr, int sub, bool valid) {
   float m = -INFINITY;
-  for (int c = lane; c < chunks; c += 32) m = fmaxf(m, p[c].x);
-  m = warp_max(m);
+  if (valid)
+    for (int c = sub; c < chunks; c += tpr) m = fmaxf(m, p[c].x);
+  for (int o = tpr >> 1; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
   float s = 0.f;
-  for (int c = lane; c < chunks; c += 32) {
-    const float2 v = p[c];
-    if (v.x > -INFINITY) s += v.y * expf(v.x - m);
-  }
-  s = warp_sum(s);
+  if (valid)
+    for (int c = sub; c < chunks; c += tpr) {
+      const float2 v = p[c];
+      if (v.x > -INFINITY) s += v.y * expf(v.x - m);
+    }
+  for (int o = tpr >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
   return m + logf(s);
 }
-__device__ __forceinline__ int merge_partials_argmax(const float2* __restrict__ p, int chunks) {
-  const int lane = threadIdx.x & 31;
+__device__ __forceinline__ int merge_partials_argmax(const float2* __restrict__ p, int chunks, int tpr, int sub, bool valid) {
   ArgMax a;
   a.s = -INFINITY;
   a.i = 0x7fffffff;
-  for (int c = lane; c < chunks; c += 32) {
+  if (valid)
+    for (int c = sub; c < chunks; c += tpr) {
+      ArgMax b;
+      b.s = p[c].x;
+      b.i = __float_as_int(p[c].y);
+      if (b.s > -INFINITY) a = argmax_better(a, b);
+    }
+  for (int o = tpr >> 1; o > 0; o >>= 1) {
     ArgMax b;
-    b.s = p[c].x;
-    b.i = __float_as_int(p[c].y);
-    if (b.s > -INFINITY) a = argmax_better(a, b);
+    b.s = __shfl_xor_sync(0xffffffffu, a.s, o);
+    b.i = __shfl_xor_sync(0xffffffffu, a.i, o);
+    a = argmax_better(a, b);
   }
-  return warp_argmax(a).i;
+  return a.i;
 }
+// lanes that share a row when rows of `chunks` pairs are merged: one thread per row for the few pairs that
+// row_stats_kernel leaves (all rows of a sequence are then merged at once), a warp per row for the hundreds that the
+// LM head's epilogue leaves
+__device__ __forceinline__ int merge_group_size(int chunks) { return chunks <= 8 ? 1 : 32; }
 
 // block-wide arg-max; result valid in thread 0
 template <int THREADS>
@@ -392,7 +404,8 @@ ar_sample_kernel(const float* __restrict__ logits, int rows_per_seq, int* __rest
 // ---------------------------------------------------------------------------------------------
 constexpr int ACCEPT_THREADS = 256;
 
-__global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(ACCEPT_THREADS)
+// four CTAs per SM (64 registers): the stand-alone call's 8 x rows CTAs then fit in one wave for 64 rows
+__global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(ACCEPT_THREADS, 4)
 accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_rows, const int* __restrict__ draft_ids,
               const float* __restrict__ logq_in, const float* __restrict__ lseq_in, const float2* __restrict__ partial_p,
               int chunks, const float2* __restrict__ partial_q, int chunks_q, int gamma, int V, float inv_tau_p,
@@ -417,17 +430,27 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
 
   if (threadIdx.x == 0) s_bad = 0;
   const float2* pp = partial_p + (long long)b * (gamma + 1) * chunks;
-  // one warp per row merges the row's pairs (a few from row_stats_kernel, over a thousand from the LM head's epilogue)
-  for (int j = threadIdx.x >> 5; j <= gamma; j += ACCEPT_THREADS / 32) {
-    const float v = greedy ? __int_as_float(merge_partials_argmax(pp + (long long)j * chunks, chunks))
-                           : merge_partials(pp + (long long)j * chunks, chunks);
-    if ((threadIdx.x & 31) == 0) s_lsep[j] = v;
+  // the rows' pairs are merged by groups of lanes sized to the number of pairs (7 from row_stats_kernel: a thread per
+  // row; 393 from the LM head's epilogue: a warp per row)
+  {
+    const int tpr = merge_group_size(chunks), sub = (int)threadIdx.x % tpr, par = ACCEPT_THREADS / tpr;
+    for (int j0 = 0; j0 <= gamma; j0 += par) {
+      const int j = j0 + (int)threadIdx.x / tpr;
+      const bool valid = j <= gamma;
+      const float2* row = pp + (long long)(valid ? j : 0) * chunks;
+      const float v = greedy ? __int_as_float(merge_partials_argmax(row, chunks, tpr, sub, valid))
+                             : merge_partials(row, chunks, tpr, sub, valid);
+      if (valid && sub == 0) s_lsep[j] = v;
+    }
   }
   if (partial_q != nullptr && !greedy) {
     const float2* pq = partial_q + (long long)b * gamma * chunks_q;
-    for (int j = threadIdx.x >> 5; j < gamma; j += ACCEPT_THREADS / 32) {
-      const float v = merge_partials(pq + (long long)j * chunks_q, chunks_q);
-      if ((threadIdx.x & 31) == 0) s_lseq[j] = v;
+    const int tpr = merge_group_size(chunks_q), sub = (int)threadIdx.x % tpr, par = ACCEPT_THREADS / tpr;
+    for (int j0 = 0; j0 < gamma; j0 += par) {
+      const int j = j0 + (int)threadIdx.x / tpr;
+      const bool valid = j < gamma;
+      const float v = merge_partials(pq + (long long)(valid ? j : 0) * chunks_q, chunks_q, tpr, sub, valid);
+      if (valid && sub == 0) s_lseq[j] = v;
     }
   }
   __syncthreads();
