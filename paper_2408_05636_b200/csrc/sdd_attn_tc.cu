@@ -133,6 +133,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   pdl_wait();   // ctx_len and Q / K / V^T come from earlier kernels
   pdl_launch_dependents();
+  // The Q tile and the first K / V^T tile go out at once: their coordinates do not depend on the context length or the
+  // skip flag, whose loads would otherwise sit in front of them (with a key split the first tile of a CTA may not exist,
+  // so only unsplit launches do this).  A CTA that turns out to have nothing to do waits for the copies and drops them.
+  const bool spec = kv_split == 1;
+  if (spec && threadIdx.x == 0) {
+    mbar_expect_tx(q_full, AT_Q_BYTES);
+    tma_load_2d(sQ, &map_q, q_full, prm.q_col0 + h * AT_DH, b * prm.q_rows_per_seq + qt * 128);
+    mbar_expect_tx(kv_full(0), AT_STAGE_BYTES);
+    tma_load_2d(sK(0), &map_k, kv_full(0), prm.k_col0 + h * AT_DH, b * prm.k_rows_per_seq);
+    tma_load_2d(sVT(0), &map_vt, kv_full(0), 0, b * prm.d + h * AT_DH);
+    tma_load_2d(sVT(0) + 64 * 64 * 2, &map_vt, kv_full(0), 64, b * prm.d + h * AT_DH);
+  }
   // a skipped drafter evaluation, or a tile of padding rows only: nothing to do (uniform over the CTA and its cluster)
   bool active = !(prm.skip != nullptr && *prm.skip);
   const int c = active ? prm.ctx_len[b] : 1;
@@ -158,12 +170,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   };
 
   if (!active) {
+    if (spec && threadIdx.x == 0) {   // the copies issued ahead must have landed before the shared memory is given back
+      long long t0 = clock64();
+      while (!mbar_try(q_full, 0u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+      t0 = clock64();
+      while (!mbar_try(kv_full(0), 0u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+    }
   } else if (warp == 0) {
-    if (lane == 0 && my_kt > 0) {
-      mbar_expect_tx(q_full, AT_Q_BYTES);
-      tma_load_2d(sQ, &map_q, q_full, prm.q_col0 + h * AT_DH, b * prm.q_rows_per_seq + q0);
-      int issued = 0;
-      for (int it = 0; it < my_kt; ++it) {
+    if (lane == 0 && my_kt > 0) {   // (an unsplit launch that is active has at least one key tile)
+      if (!spec) {
+        mbar_expect_tx(q_full, AT_Q_BYTES);
+        tma_load_2d(sQ, &map_q, q_full, prm.q_col0 + h * AT_DH, b * prm.q_rows_per_seq + q0);
+      }
+      int issued = spec ? 1 : 0;
+      for (int it = issued; it < my_kt; ++it) {
         const int t = kv_rank + it * kv_split;      // key tile; `it` counts this CTA's iterations (stages, phases)
         const int s = it % AT_KV_STAGES;
         if (!mbar_wait(kv_empty(s), ((uint32_t)(it / AT_KV_STAGES) & 1u) ^ 1u, abort_flag, prm.status)) break;
@@ -285,9 +305,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       };
       uint32_t sc[PIPE ? 2 : 1][32];
       if constexpr (PIPE) {
-        tmem_ld32(t_s + (uint32_t)(hf * 64), sc[0]);
+        tmem_ld32_issue(t_s + (uint32_t)(hf * 64), sc[0]);
+        tmem_ld32_issue(t_s + (uint32_t)(hf * 64 + 32), sc[1]);
+        tmem_ld_wait(sc[0], sc[1]);
         max_chunk(sc[0], 0);
-        tmem_ld32(t_s + (uint32_t)(hf * 64 + 32), sc[1]);
         max_chunk(sc[1], 1);
       } else {
 #pragma unroll 1

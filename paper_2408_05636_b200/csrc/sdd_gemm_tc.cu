@@ -599,33 +599,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
   pdl_wait();
   pdl_launch_dependents();
+  // The activation tiles of the stages whose weight tiles are already on their way go out at once, before the skip
+  // flag has even been read (one L2 round trip that would otherwise sit in front of the first operand tile of every
+  // launch of a drafter evaluation); if the evaluation turns out to be skipped the tiles are waited for and dropped.
+  if (threadIdx.x == 0) {
+    for (int kb = 0; kb < n_pre; ++kb) {
+      const uint32_t sa = base + kb * STAGE_BYTES;
+      mbar_expect_tx(full_bar(kb), (uint32_t)STAGE_BYTES - W_BYTES);
+      if (SWAP) tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(kb), (kb0 + kb) * BK, n0);
+      else tma_load_2d(sa, &map_a, full_bar(kb), (kb0 + kb) * BK, m0);
+      if (HILO) tma_load_2d(sa + LO_OFF, &map_lo, full_bar(kb), (kb0 + kb) * BK, SWAP ? n0 : m0);
+    }
+  }
   // launches of a drafter evaluation do nothing when the evaluation is skipped (they still free their TMEM below)
   const bool active = skip == nullptr || *skip == 0;
 
   if (!active) {
-    // weight tiles fetched ahead must have landed before the CTA gives its shared memory back
+    // tiles fetched ahead must have landed before the CTA gives its shared memory back
     for (int kb = 0; kb < n_pre; ++kb) {
-      mbar_arrive(full_bar(kb));
       const long long t0 = clock64();
       while (!mbar_try(full_bar(kb), 0u) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
     }
   } else if (warp == 0) {
     if (lane == 0) {
-      int issued = 0;
-      for (int kb = 0; kb < num_kb; ++kb) {
+      int issued = n_pre;
+      for (int kb = n_pre; kb < num_kb; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
         const uint32_t sa = base + s * STAGE_BYTES;
-        if (kb < n_pre) {
-          mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES - W_BYTES);      // the weight tile is already on its way
-          if (SWAP) tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), (kb0 + kb) * BK, n0);
-          else tma_load_2d(sa, &map_a, full_bar(s), (kb0 + kb) * BK, m0);
-        } else {
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, status)) break;
-          mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES);
-          tma_load_2d(sa, &map_a, full_bar(s), (kb0 + kb) * BK, m0);
-          tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), (kb0 + kb) * BK, n0);
-        }
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, status)) break;
+        mbar_expect_tx(full_bar(s), (uint32_t)STAGE_BYTES);
+        tma_load_2d(sa, &map_a, full_bar(s), (kb0 + kb) * BK, m0);
+        tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(s), (kb0 + kb) * BK, n0);
         if (HILO) tma_load_2d(sa + LO_OFF, &map_lo, full_bar(s), (kb0 + kb) * BK, SWAP ? n0 : m0);
         issued = kb + 1;
       }

@@ -225,18 +225,20 @@ layernorm_vec_kernel(const float* __restrict__ h, const float* __restrict__ g, c
   }
   pdl_wait();
   pdl_launch_dependents();
-  if (skip != nullptr && *skip) return;
   const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
   if (row >= rows) return;
   const float* __restrict__ src = h + row * d;
+  // the row's loads are issued before the skip flag is looked at, so that the two round trips overlap
   float4 x[NV];
-  float sum = 0.f;
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
     const int e = (i * 32 + lane) * 4;
     x[i] = e < d ? *reinterpret_cast<const float4*>(src + e) : make_float4(0.f, 0.f, 0.f, 0.f);
-    sum += (x[i].x + x[i].y) + (x[i].z + x[i].w);
   }
+  if (skip != nullptr && *skip) return;
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) sum += (x[i].x + x[i].y) + (x[i].z + x[i].w);
   const float mu = warp_sum(sum) / (float)d;
   float var = 0.f;
 #pragma unroll
