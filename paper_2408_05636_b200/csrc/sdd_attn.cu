@@ -55,8 +55,8 @@ template <typename T, int DH>
 __global__ void __launch_bounds__(128)
 attn_bidir_kernel(const T* __restrict__ qkv, T* __restrict__ out, const int* __restrict__ ctx_len, int gamma, int L_cap,
                   int n_head, const int* __restrict__ skip) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   if (skip != nullptr && *skip) return;
   const int i = blockIdx.x * 4 + (threadIdx.x >> 5), h = blockIdx.y, b = blockIdx.z;
   if (i >= L_cap) return;
@@ -76,8 +76,8 @@ template <typename T, int DH>
 __global__ void __launch_bounds__(128)
 attn_cached_kernel(const T* __restrict__ qkv, const T* __restrict__ cache, T* __restrict__ out,
                    const int* __restrict__ ctx_len, int rows_per_seq, int mode, int n_ctx, int n_head) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const int j = blockIdx.x * 4 + (threadIdx.x >> 5), h = blockIdx.y, b = blockIdx.z;
   if (j >= rows_per_seq) return;
   const int d = n_head * DH;

@@ -131,8 +131,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  pdl_wait();   // ctx_len and Q / K / V^T come from earlier kernels
   pdl_launch_dependents();
+  pdl_wait();   // ctx_len and Q / K / V^T come from earlier kernels
   // The Q tile and the first K / V^T tile go out at once: their coordinates do not depend on the context length or the
   // skip flag, whose loads would otherwise sit in front of them (with a key split the first tile of a CTA may not exist,
   // so only unsplit launches do this).  A CTA that turns out to have nothing to do waits for the copies and drops them.

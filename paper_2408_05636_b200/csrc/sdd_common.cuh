@@ -146,6 +146,14 @@ __device__ __forceinline__ float gelu_tanh(float x) {
 // completed and its writes are visible.  Every kernel of the library calls pdl_wait() before its
 // first access to global memory, so stream order is preserved transitively.  Without the launch
 // attribute the instruction does nothing.
+// pdl_launch_dependents() comes BEFORE the wait: the next kernel's CTAs become resident (barriers, tensor-memory
+// allocation, descriptor and weight prefetch) while this kernel is still waiting for its own predecessor, so a chain
+// of short kernels runs two or three launches ahead.  Two rules keep that safe.  (1) A kernel that allocates tensor
+// memory triggers only after its allocation (and the block-wide barrier behind it): a later kernel's CTA on the same
+// SM can then never hold columns that this one still needs.  A dependent grid starts only when every CTA of its
+// predecessor has triggered, hence is resident, so the resident CTAs are always a contiguous window of the chain
+// and nobody waits on a CTA that cannot be scheduled.  (2) Nothing ahead of the wait reads memory that a kernel of
+// the library writes (weights, LayerNorm gains: constant), except hints whose staleness costs time only.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

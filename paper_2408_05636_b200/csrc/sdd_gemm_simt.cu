@@ -11,8 +11,8 @@ template <typename T>
 __global__ void __launch_bounds__(SG_THREADS)
 gemm_simt_kernel(const T* __restrict__ A, int lda, const T* __restrict__ W, const float* __restrict__ bias, int M, int N,
                  int K, int epi, void* __restrict__ out, int ldc, const int* __restrict__ skip) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   if (skip != nullptr && *skip) return;
   __shared__ float As[SG_BK][SG_BM + 4];
   __shared__ float Ws[SG_BK][SG_BN + 4];

@@ -597,8 +597,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       else tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(kb), (kb0 + kb) * BK, n0);
     }
   }
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   // The activation tiles of the stages whose weight tiles are already on their way go out at once, before the skip
   // flag has even been read (one L2 round trip that would otherwise sit in front of the first operand tile of every
   // launch of a drafter evaluation); if the evaluation turns out to be skipped the tiles are waited for and dropped.
@@ -793,8 +793,8 @@ gemm_tc_persist_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       else tma_load_2d(sa + BM * BK * 2, &map_b, full_bar(j), kb * BK, n0);
     }
   }
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const bool active = skip == nullptr || *skip == 0;
 
   if (!active) {
@@ -982,8 +982,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const bool active = skip == nullptr || *skip == 0;   // the same value in both CTAs (read after the producer grid)
 
   if (!active) {
@@ -1115,8 +1115,8 @@ __global__ void __launch_bounds__(THREADS) wait_timeout_probe_kernel(long long l
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_base = tmem_slot_s;
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   if (warp == 0) {
     // the producer, at the point where it wants to refill a stage: it waits for the MMA that would free it, which
     // never comes; it leaves on the abort flag or on its own limit, with no copy in flight

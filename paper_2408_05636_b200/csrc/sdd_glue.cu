@@ -52,8 +52,8 @@ embed_drafter_kernel(const T* __restrict__ wte, const T* __restrict__ wpe, const
                      int gamma, int L_cap, int d, float* __restrict__ h, const int* __restrict__ skip,
                      const float* __restrict__ ln_g, const float* __restrict__ ln_b, T* __restrict__ xn, int vocab,
                      int* __restrict__ status) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   if (skip != nullptr && *skip) return;
   const int i = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
@@ -96,8 +96,8 @@ __global__ void embed_target_kernel(const T* __restrict__ wte, const T* __restri
                                     int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
                                     int gamma, int rows_per_seq, int mode, int d, float* __restrict__ h, int vocab,
                                     int* __restrict__ status) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const int j = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
   float* __restrict__ dst = h + ((long long)b * rows_per_seq + j) * d;
@@ -133,8 +133,8 @@ __global__ void embed_ar_kernel(const T* __restrict__ wte, const T* __restrict__
                                 int tok_stride, const int* __restrict__ ctx_len, const int* __restrict__ slot_ids,
                                 int gamma, int rows_per_seq, int off, int d, float* __restrict__ h,
                                 int* __restrict__ eff_len, int vocab, int* __restrict__ status) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const int i = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
   if (i == 0 && threadIdx.x == 0) eff_len[b] = c + off;
@@ -223,8 +223,8 @@ layernorm_vec_kernel(const float* __restrict__ h, const float* __restrict__ g, c
     if (e < d) { gg[i] = *reinterpret_cast<const float4*>(g + e); bb[i] = *reinterpret_cast<const float4*>(bta + e); }
     else { gg[i] = make_float4(0.f, 0.f, 0.f, 0.f); bb[i] = gg[i]; }
   }
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
   if (row >= rows) return;
   const float* __restrict__ src = h + row * d;
@@ -269,8 +269,8 @@ template <typename T>
 __global__ void __launch_bounds__(128)
 layernorm_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
                  T* __restrict__ out, T* __restrict__ out_lo, long long rows, int d, const int* __restrict__ skip) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   if (skip != nullptr && *skip) return;
   const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -282,8 +282,8 @@ __global__ void __launch_bounds__(128)
 layernorm_slots_kernel(const float* __restrict__ h, const float* __restrict__ g, const float* __restrict__ bta,
                        T* __restrict__ out, const int* __restrict__ ctx_len, int batch, int gamma, int L_cap, int d,
                        const int* __restrict__ skip) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   if (skip != nullptr && *skip) return;
   const int r = blockIdx.x * 4 + (threadIdx.x >> 5);
   if (r >= batch * gamma) return;
@@ -299,8 +299,8 @@ template <typename T>
 __global__ void gather_slots_kernel(const T* __restrict__ att, const float* __restrict__ h, const int* __restrict__ ctx_len,
                                     int gamma, int L_cap, int d, T* __restrict__ att_s, float* __restrict__ h_s,
                                     const int* __restrict__ skip) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   if (skip != nullptr && *skip) return;
   const int j = blockIdx.x, b = blockIdx.y;
   const long long src = ((long long)b * L_cap + ctx_len[b] + j) * d, dst = ((long long)b * gamma + j) * d;
@@ -316,8 +316,8 @@ __global__ void gather_slots_kernel(const T* __restrict__ att, const float* __re
 template <typename T>
 __global__ void kv_append_kernel(const T* __restrict__ qkv, T* __restrict__ cache, const int* __restrict__ ctx_len,
                                  int rows_per_seq, int mode, int n_ctx, int d) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const int j = blockIdx.x, b = blockIdx.y;
   const int c = ctx_len[b];
   int pos;

@@ -30,8 +30,8 @@ template <bool GREEDY>
 __global__ void __launch_bounds__(STATS_THREADS)
 row_stats_kernel(const float* __restrict__ buf_a, long long rows_a, const float* __restrict__ buf_b, long long rows_b,
                  int V, int chunks, float inv_tau_a, float inv_tau_b, float2* __restrict__ partial) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const long long row = blockIdx.x / chunks;
   const int chunk = blockIdx.x - (int)(row * chunks);
   const bool is_a = row < rows_a;
@@ -361,8 +361,8 @@ __global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(SAMPLE_THREADS)
 unmask_sample_kernel(const float* __restrict__ step_logits, int* __restrict__ slot_ids, float* __restrict__ q_logits,
                      float* __restrict__ logq, float* __restrict__ lseq, int* __restrict__ reveal_step, int gamma, int V, int k,
                      float inv_tau_q, PhiloxKey key, RoundState* __restrict__ rs, int cache_skip) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const bool revealed = unmask_sample_row(step_logits, slot_ids, q_logits, logq, lseq, reveal_step, gamma, V, k, inv_tau_q, key, rs);
   if (threadIdx.x == 0) {
     if (revealed && (blockIdx.x % VC) == 0) atomicAdd(&rs->revealed, 1u);
@@ -385,8 +385,8 @@ __global__ void __cluster_dims__(VC, 1, 1) __launch_bounds__(SAMPLE_THREADS)
 ar_sample_kernel(const float* __restrict__ logits, int rows_per_seq, int* __restrict__ slot_ids, float* __restrict__ q_logits,
                  float* __restrict__ logq, float* __restrict__ lseq, int* __restrict__ reveal_step, int gamma, int j, int V,
                  float inv_tau_q, PhiloxKey key, RoundState* __restrict__ rs) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.y;
   const long long row = (long long)b * gamma + j;
   draw_slot(logits + ((long long)b * rows_per_seq + rows_per_seq - 1) * V, q_logits + row * V, slot_ids + row, logq + row,
@@ -412,8 +412,8 @@ accept_kernel(const float* __restrict__ logits_p, const float* __restrict__ q_ro
               float inv_tau_q_rows, PhiloxKey key, uint32_t rnd_arg, RoundState* __restrict__ rs,
               float* __restrict__ accept_prob, int* __restrict__ n_accept, int* __restrict__ extra_token,
               int* __restrict__ out_ids) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   cg::cluster_group cl = cg::this_cluster();
   const int rank = (int)cl.block_rank();
   const int b = blockIdx.x / VC;
@@ -592,8 +592,8 @@ __global__ void commit_kernel(int* __restrict__ tokens, int tok_stride, int* __r
                               const int* __restrict__ n_accept, const int* __restrict__ extra_token, int batch, int gamma,
                               int max_new, RoundState* rs, int* __restrict__ out_ids, int* __restrict__ n_out,
                               volatile int* host_mirror) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const uint32_t stamp = rs->round + 1u;
   if (host_mirror != nullptr && threadIdx.x == 0) {
     host_mirror[0] = (int)stamp;
@@ -638,8 +638,8 @@ __global__ void commit_kernel(int* __restrict__ tokens, int tok_stride, int* __r
 
 __global__ void reset_slots_kernel(int* __restrict__ slot_ids, int* __restrict__ reveal_step, int n, int mask_id,
                                    RoundState* __restrict__ rs) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i == 0) { rs->skip_forward = 0; rs->revealed = 0u; rs->ticket = 0u; }   // a round's first evaluation always runs
   if (i < n) {
