@@ -164,6 +164,21 @@ def test_xl_bf16_whole_round_at_its_own_T():
     s.close()
 
 
+def test_xl_bf16_whole_round_late_in_generation():
+    """The same configuration where a generation of the benchmark ends: 1000 tokens of context, so the drafter runs on
+    1152 padded rows (nine query tiles x 16 heads of pipelined attention with nine key tiles each, GEMM grids of more
+    than one wave) and the target attends over eight cached key tiles.  One round through sdd_step."""
+    import paper_2408_05636_b200 as sdd
+    wl = synth.scaled_workload(synth.WORKLOADS["xl_bf16"], prompt_len=1000, max_new=64)
+    mp, mq, dp, dq = roundcheck.build_pair(wl)
+    prompts = synth.prompt_ids(wl.target.vocab, 1, wl.prompt_len, wl.prompt_seed)
+    s = sdd.Session(dp, dq, prompts, [wl.prompt_len], wl.gamma, wl.T, wl.max_new, 1.0, 1.0, wl.philox_seed)
+    log, worst_q, worst_p = roundcheck.check_whole_rounds(s, mp, mq, wl, 1, TOL, seqs=[0], n_sampled_steps=1)
+    print("near-ties:", log, "max logit err q/p:", worst_q, worst_p)
+    parity.assert_few(log)
+    s.close()
+
+
 def test_xl_bf16_b16_sweep_corner_gamma64_T32():
     """The serving sweep's largest corner at full size: 16 sequences of 1024 tokens on the XL pair, gamma 64, T 32
     (pair GEMMs, slot-row pruning and 65 target rows per sequence in one round), through sdd_step.  One sequence of
