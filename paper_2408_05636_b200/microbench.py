@@ -2,6 +2,7 @@
 
     python -m paper_2408_05636_b200.microbench gemm  --m 8192 --n 4096 --k 4096 [--epilogue 0] [--n-tile 0]
     python -m paper_2408_05636_b200.microbench attn  --heads 16 --len 1024 [--batch 1]
+    python -m paper_2408_05636_b200.microbench attn-verify --heads 25 --len 1000 --rows 33 [--batch 1]
     python -m paper_2408_05636_b200.microbench accept --rows 64 --gamma 32 [--vocab 50257]
 
 Each prints one JSON line with the time per launch and the achieved rate.  `--iters` launches are timed
@@ -66,6 +67,23 @@ def attn(heads, length, batch=1, gamma=16, iters=50, warmup=5, seed=0):
             "tflops": flops / (ms * 1e-3) / 1e12}
 
 
+def attn_target(heads, ctx_len, rows=33, batch=1, n_ctx=2048, iters=50, warmup=5, seed=0):
+    """Verification-mode attention: `rows` new query rows per sequence over a cache of ctx_len - 1 keys plus themselves."""
+    d = heads * 64
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    qkv = torch.randn(batch * rows + 200, 3 * d, device="cuda", generator=g).to(torch.bfloat16)
+    kc = torch.randn(batch * n_ctx, d, device="cuda", generator=g).to(torch.bfloat16)
+    vt = torch.randn(batch * d, n_ctx, device="cuda", generator=g).to(torch.bfloat16)
+    out = torch.zeros(batch * rows, d, device="cuda", dtype=torch.bfloat16)
+    ctx = torch.full((batch,), ctx_len, dtype=torch.int32, device="cuda")
+    st = torch.cuda.Stream()
+    ms = time_launches(lambda: sdd.sdd_debug_attention_bf16(qkv, 0, kc, 0, n_ctx, vt, out, ctx, batch, heads, rows - 1, 1,
+                                                            rows, None, st), iters, warmup, st)
+    nbytes = batch * (2.0 * (ctx_len - 1 + rows) * d * 2 + 2.0 * rows * d * 2)
+    return {"kernel": "attn_tc_verify", "heads": heads, "ctx_len": ctx_len, "rows": rows, "batch": batch, "us": ms * 1e3,
+            "gbs": nbytes / (ms * 1e-3) / 1e9}
+
+
 def accept(rows, gamma, vocab=50257, sigma=0.5, iters=20, warmup=3, seed=31):
     g = torch.Generator(device="cuda").manual_seed(seed)
     c = torch.randn(rows, gamma + 1, vocab, device="cuda", generator=g)
@@ -117,7 +135,7 @@ def accept_case_timed(base, gamma, iters=20, warmup=3, seed=31, rnd=7):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["gemm", "attn", "accept"])
+    ap.add_argument("kernel", choices=["gemm", "attn", "attn-verify", "accept"])
     ap.add_argument("--m", type=int, default=8192)
     ap.add_argument("--n", type=int, default=4096)
     ap.add_argument("--k", type=int, default=4096)
@@ -136,6 +154,8 @@ def main():
         r = gemm(a.m, a.n, a.k, a.epilogue, a.n_tile, a.iters, a.warmup)
     elif a.kernel == "attn":
         r = attn(a.heads, a.len, a.batch, iters=a.iters, warmup=a.warmup)
+    elif a.kernel == "attn-verify":
+        r = attn_target(a.heads, a.len, a.rows, a.batch, iters=a.iters, warmup=a.warmup)
     else:
         r = accept(a.rows, a.gamma, a.vocab, iters=a.iters, warmup=a.warmup)
     print(json.dumps(r))
