@@ -354,6 +354,39 @@ __device__ __forceinline__ void epilogue_manual(uint32_t tmem_acc, int m0, int n
   }
 }
 
+// SWAP orientation, fp32 residual stream (tile = 128 features x up to BN tokens; a thread owns one feature): the tile
+// is written token-major into four 128-byte-swizzled boxes of 32 features, one per epilogue warp, and leaves as four
+// TMA add-reduces, out[token][feature] += acc + bias; tokens past the last row and features past the last column are
+// clipped by the tensor map.  (Per-element atomics from the registers -- 4224 a CTA, half a million a launch on 53 k
+// addresses under K splits -- took 3.5 us per launch.)
+template <int BN>
+__device__ __forceinline__ void epilogue_swap_reduce(uint32_t tmem_acc, int m0, int n0, int q, int lane, int rows_a,
+                                                     const float* __restrict__ bias, const CUtensorMap* map_out,
+                                                     uint8_t* stage_generic, uint32_t stage_u32) {
+  const int r = m0 + q * 32 + lane;
+  const float bv = (bias != nullptr && r < rows_a) ? bias[r] : 0.f;
+  uint8_t* box = stage_generic + q * (BN * 128);
+  const uint32_t chunk = (uint32_t)lane >> 2, within = ((uint32_t)lane & 3u) * 4u;
+#pragma unroll 1
+  for (int cc = 0; cc < BN / 32; ++cc) {
+    uint32_t v[32];
+    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), v);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const uint32_t t = (uint32_t)(cc * 32 + j);
+      *reinterpret_cast<float*>(box + t * 128u + ((chunk ^ (t & 7u)) << 4) + within) = __uint_as_float(v[j]) + bv;
+    }
+  }
+  fence_async_smem();
+  named_bar_sync(2, 128);
+  if (threadIdx.x == 64) {
+    for (int qq = 0; qq < 4; ++qq)
+      if (m0 + qq * 32 < rows_a) tma_reduce_add_2d(map_out, stage_u32 + (uint32_t)(qq * BN * 128), m0 + qq * 32, n0);
+    tma_commit_group();
+    tma_wait_group_read<0>();       // shared memory stays valid until the copies have read it
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // LM-head epilogues that also produce the rows' soft-max statistics (HeadStats): the logits are stored as by
 // EPI_STORE_F32, and every (token row, slice of the vocabulary) gets one pair (max z, sum exp(z - max)), z = logit *
@@ -704,6 +737,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       epilogue_vt<BN>(tmem_base, q, lane, bias_s, &maps_out.vt, stage_g, stage_u, n_store, sb * qd.d + (n0 - 2 * qd.d),
                       m0 - sb * qd.rows_per_seq, eg);
       if ((int)threadIdx.x == eg.first_tid) tma_wait_group_read<0>();
+    } else if (ready && SWAP && tma_out == 4) {
+      if constexpr (SWAP) epilogue_swap_reduce<BN>(tmem_base, m0, n0, q, lane, rows_a, bias, &maps_out.out, generic_base, base);
     } else if (ready) {
       epilogue_manual<BN, SWAP, SWAP>(tmem_base, m0, n0, q, lane, rows_a, rows_b, epi, bias, out, out_lo, ldc, split, qd, eg.c_begin,
                                       eg.c_end);
@@ -1342,6 +1377,12 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
     if (hilo && (e = get_tensor_map(A_lo, a_cap, K, K, bn, BK, &ml)) != cudaSuccess) return e;
     OutMaps none;
     none.out = ma; none.vt = ma;
+    // fp32 residual stream with 16-byte-aligned rows: the tile leaves as TMA add-reduces (see epilogue_swap_reduce)
+    int swap_tma = 0;
+    if (epi == EPI_RESIDUAL && (ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+      if ((e = get_tensor_map(out, M, N, ldc, bn, 32, &none.out, 4)) != cudaSuccess) return e;
+      swap_tma = 4;
+    }
     // many weight tiles (the LM heads): the persistent kernel keeps the weight stream going across tiles
     // (SDD_GEMM_PERSIST=0 switches it off)
     {
@@ -1355,8 +1396,8 @@ cudaError_t launch_gemm_tc(const __nv_bfloat16* A, long long a_cap, const __nv_b
                     : launch_persist_swap<64, false>(ma, mb, ml, none, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, skip, hs);
       }
     }
-    if (bn == 32) return launch_hl<32, true>(hilo, ma, mb, ml, none, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
-    return launch_hl<64, true>(hilo, ma, mb, ml, none, 0, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
+    if (bn == 32) return launch_hl<32, true>(hilo, ma, mb, ml, none, swap_tma, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
+    return launch_hl<64, true>(hilo, ma, mb, ml, none, swap_tma, N, M, K, epi, bias, out, out_lo, ldc, status, st, qd, splits, skip);
   }
   int bn = bn_hint == 512 ? 256 : bn_hint;       // 512: the CTA-pair kernel on 256 x 256 tiles
   const long long mt = (M + BM - 1) / BM;

@@ -47,24 +47,26 @@ def test_tc_gemm_matches_fp32_matmul(M, N, K, n_tile):
         for b in (bias, None):
             # fp32 outputs: a row stride that is not a multiple of 4 takes the hand-written epilogue, a multiple of 4
             # the TMA add-reduce (the CTA-pair cases use the latter)
-            ldc = N + (8 if epi in (0, 1) else (4 if n_tile == 512 else 3))
-            if epi in (0, 1):
-                out = torch.full((M, ldc), 7.0, device="cuda", dtype=torch.bfloat16)
-            else:
-                out = torch.randn(M, ldc, device="cuda", generator=g)
-            out0 = out[:, :N].float().clone()
-            sdd.sdd_debug_gemm_bf16(A, W, b, M, epi, out, n_tile, True, status)
-            torch.cuda.synchronize()
-            assert int(status.item()) == 0
-            ref = _ref(A, W, b, M, epi, out0)
-            got = out[:, :N].float()
-            tol = 2e-2 if epi in (0, 1) else 2e-3      # bf16 output rounding / fp32 accumulation order
-            err = (got - ref).abs().max().item()
-            scale = ref.abs().max().item()
-            assert err <= tol * max(1.0, scale), (epi, err, scale)
-            pad = out[:, N:].float()
-            if epi in (0, 1):
-                assert torch.all(pad == 7.0)            # nothing written past column N
+            ldcs = [N + (8 if epi in (0, 1) else (4 if n_tile == 512 else 3))]
+            if epi == 2 and M <= 64:
+                ldcs.append(N + 4)      # swapped orientation: the residual tile leaves by TMA add-reduce as well
+            for ldc in ldcs:
+                if epi in (0, 1):
+                    out = torch.full((M, ldc), 7.0, device="cuda", dtype=torch.bfloat16)
+                else:
+                    out = torch.randn(M, ldc, device="cuda", generator=g)
+                out0 = out[:, :N].float().clone()
+                pad0 = out[:, N:].float().clone()
+                sdd.sdd_debug_gemm_bf16(A, W, b, M, epi, out, n_tile, True, status)
+                torch.cuda.synchronize()
+                assert int(status.item()) == 0
+                ref = _ref(A, W, b, M, epi, out0)
+                got = out[:, :N].float()
+                tol = 2e-2 if epi in (0, 1) else 2e-3      # bf16 output rounding / fp32 accumulation order
+                err = (got - ref).abs().max().item()
+                scale = ref.abs().max().item()
+                assert err <= tol * max(1.0, scale), (epi, ldc, err, scale)
+                assert torch.equal(out[:, N:].float(), pad0)   # nothing written past column N
 
 
 def test_simt_and_tc_agree():
