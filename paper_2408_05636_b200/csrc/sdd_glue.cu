@@ -366,7 +366,7 @@ cudaError_t launch_layernorm(const float* h, const float* g, const float* b, T* 
   const dim3 grid((unsigned)((rows + 3) / 4));
   const uintptr_t al = reinterpret_cast<uintptr_t>(h) | reinterpret_cast<uintptr_t>(g) | reinterpret_cast<uintptr_t>(b) |
                        reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(out_lo);
-  if ((d & 3) == 0 && (al & 15u) == 0 && rows >= 64) {
+  if ((d & 3) == 0 && (al & 15u) == 0) {
     if (d <= 1024) launch_k(layernorm_vec_kernel<T, 8>, grid, dim3(128), 0, st, h, g, b, out, out_lo, rows, d, skip);
     else launch_k(layernorm_vec_kernel<T, 16>, grid, dim3(128), 0, st, h, g, b, out, out_lo, rows, d, skip);
   } else {
